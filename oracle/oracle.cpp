@@ -1,0 +1,168 @@
+// CPU oracle for the dense hot path: plain FP64 GEMM and naive three-pass
+// softmax attention over BF16-rounded inputs.
+//
+// THIS IS TEST INFRASTRUCTURE.  Only the tests, the smoke check and the
+// benchmark's cpu_baseline / reference legs may build, link or call it.  It
+// shares no code with the CUDA path and is deliberately slow and literal so a
+// reader can check it against the paper by eye.
+//
+// What it follows:
+//  * GEMM: the problem statement of Sec. 2 (A in R^{m x k}, B in R^{k x n},
+//    C in R^{m x n}) and the loop of Listing 2 (zero accumulator, sum over k of
+//    A-tile times B-tile, store).  Reading taken: C = A*B (the listing stores
+//    the loop result; prior C contents are ignored).
+//  * MHA forward: Algorithm 1 (FlashAttention-2 forward) computes exact softmax
+//    attention; the oracle is that definition written out per query row in three
+//    passes (scores and their max; exponentials and their sum; weighted sum of
+//    V), with the scale, causal mask, 1/l normalisation and log-sum-exp output
+//    the algorithm box leaves implicit.
+//
+// Inputs are BF16 bit patterns (uint16).  BF16 -> double is exact and every
+// product of two BF16 values is exact in double, so the only rounding is in the
+// FP64 summations.  Outputs stay in FP64 (never rounded to BF16).
+//
+// Pins (see tests/test_oracle_*.py): identity / permutation / all-ones /
+// single-non-zero / K-split additivity / exact rational brute force for GEMM;
+// constant-K mean-of-V, causal row 0, Nk = 1, rows summing to one, key
+// permutation invariance, split-merge identity, shift invariance, dominant key,
+// independent brute force for attention.  The causal alignment for Nq != Nk
+// (bottom-right) is a convention the paper does not state: parity unpinned by
+// the paper for that case.
+
+#include <algorithm>
+#include <cmath>
+#include <cstdint>
+#include <cstring>
+#include <limits>
+#include <thread>
+#include <vector>
+
+namespace {
+
+inline double bf16_to_double(uint16_t bits) {
+    uint32_t w = static_cast<uint32_t>(bits) << 16;
+    float f;
+    std::memcpy(&f, &w, sizeof f);
+    return static_cast<double>(f);
+}
+
+template <class F>
+void parallel_for(int64_t n, int nthreads, F&& body) {
+    if (nthreads <= 0) nthreads = static_cast<int>(std::thread::hardware_concurrency());
+    if (nthreads < 1) nthreads = 1;
+    if (n < nthreads) nthreads = static_cast<int>(std::max<int64_t>(n, 1));
+    if (nthreads == 1) {
+        for (int64_t i = 0; i < n; ++i) body(i);
+        return;
+    }
+    std::vector<std::thread> pool;
+    pool.reserve(nthreads);
+    for (int t = 0; t < nthreads; ++t)
+        pool.emplace_back([&, t] {
+            for (int64_t i = t; i < n; i += nthreads) body(i);
+        });
+    for (auto& th : pool) th.join();
+}
+
+}  // namespace
+
+extern "C" {
+
+int oracle_hardware_threads(void) {
+    int n = static_cast<int>(std::thread::hardware_concurrency());
+    return n < 1 ? 1 : n;
+}
+
+// C_out[r][j] = sum_{k<K} A[rows[r]][k] * B[k][j]      (Sec. 2, Listing 2)
+//
+// A: M x K row-major, pitch lda (elements); B: K x N row-major, pitch ldb.
+// rows: nrows row indices of C to compute, or NULL for all M rows (nrows
+// ignored).  C_out: dense (nrows or M) x N doubles.  Returns 0, or 1 on a bad
+// argument.
+int oracle_gemm(const uint16_t* A, const uint16_t* B, double* C_out,
+                int64_t M, int64_t N, int64_t K, int64_t lda, int64_t ldb,
+                const int64_t* rows, int64_t nrows, int nthreads) {
+    if (M < 0 || N < 0 || K < 0 || lda < K || ldb < N) return 1;
+    const int64_t R = rows ? nrows : M;
+    if (rows)
+        for (int64_t r = 0; r < R; ++r)
+            if (rows[r] < 0 || rows[r] >= M) return 1;
+    parallel_for(R, nthreads, [&](int64_t r) {
+        const int64_t i = rows ? rows[r] : r;
+        double* c = C_out + r * N;
+        for (int64_t j = 0; j < N; ++j) c[j] = 0.0;
+        for (int64_t k = 0; k < K; ++k) {
+            const double a = bf16_to_double(A[i * lda + k]);
+            const uint16_t* b = B + k * ldb;
+            for (int64_t j = 0; j < N; ++j) c[j] += a * bf16_to_double(b[j]);
+        }
+    });
+    return 0;
+}
+
+// Exact softmax attention for selected query rows (Algorithm 1, written as the
+// definition it reaches).
+//
+// Q: [B,H,Nq,D], K,V: [B,H,Nk,D], contiguous, D fastest, BF16 bits.
+// qrows: nrows flat query indices (b*H + h)*Nq + i, or NULL for all B*H*Nq.
+// O_out: nrows x D doubles; LSE_out: nrows doubles (natural log); P_out: NULL,
+// or nrows x Nk doubles receiving the normalised probabilities (0 where masked).
+// Key j is visible to query i iff j < Nk and (not causal or j <= i + (Nk - Nq)).
+//   pass 1: s_j = scale * sum_d Q[i][d] K[j][d] for visible j;  m = max_j s_j
+//   pass 2: e_j = exp(s_j - m);  l = sum_j e_j
+//   pass 3: O[i][d] = sum_j (e_j / l) V[j][d];  LSE[i] = m + ln l
+// `scale` is the FP32 value the GPU entry point receives, widened to double.
+int oracle_mha_fwd(const uint16_t* Q, const uint16_t* K, const uint16_t* V,
+                   double* O_out, double* LSE_out, double* P_out,
+                   int B, int H, int Nq, int Nk, int D, int causal, float scale,
+                   const int64_t* qrows, int64_t nrows, int nthreads) {
+    if (B < 0 || H < 0 || Nq < 0 || Nk < 1 || D < 1) return 1;
+    if (causal && Nq > Nk) return 1;
+    const int64_t total = static_cast<int64_t>(B) * H * Nq;
+    const int64_t R = qrows ? nrows : total;
+    if (qrows)
+        for (int64_t r = 0; r < R; ++r)
+            if (qrows[r] < 0 || qrows[r] >= total) return 1;
+    const double sc = static_cast<double>(scale);
+    parallel_for(R, nthreads, [&](int64_t r) {
+        const int64_t flat = qrows ? qrows[r] : r;
+        const int64_t bh = flat / Nq;
+        const int64_t i = flat % Nq;
+        const uint16_t* q = Q + flat * D;
+        const uint16_t* Kh = K + bh * Nk * D;
+        const uint16_t* Vh = V + bh * Nk * D;
+        const int64_t visible = causal ? std::min<int64_t>(Nk, i + (Nk - Nq) + 1) : Nk;
+        std::vector<double> s(static_cast<size_t>(visible));
+        std::vector<double> qd(static_cast<size_t>(D));
+        for (int d = 0; d < D; ++d) qd[d] = bf16_to_double(q[d]);
+        // pass 1
+        double m = -std::numeric_limits<double>::infinity();
+        for (int64_t j = 0; j < visible; ++j) {
+            double dot = 0.0;
+            for (int d = 0; d < D; ++d) dot += qd[d] * bf16_to_double(Kh[j * D + d]);
+            s[j] = sc * dot;
+            m = std::max(m, s[j]);
+        }
+        // pass 2
+        double l = 0.0;
+        for (int64_t j = 0; j < visible; ++j) {
+            s[j] = std::exp(s[j] - m);
+            l += s[j];
+        }
+        // pass 3
+        double* o = O_out + r * D;
+        for (int d = 0; d < D; ++d) o[d] = 0.0;
+        for (int64_t j = 0; j < visible; ++j) {
+            const double p = s[j] / l;
+            for (int d = 0; d < D; ++d) o[d] += p * bf16_to_double(Vh[j * D + d]);
+        }
+        LSE_out[r] = m + std::log(l);
+        if (P_out) {
+            double* p = P_out + r * Nk;
+            for (int64_t j = 0; j < Nk; ++j) p[j] = j < visible ? s[j] / l : 0.0;
+        }
+    });
+    return 0;
+}
+
+}  // extern "C"
