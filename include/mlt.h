@@ -1,0 +1,97 @@
+/*
+ * mlt.h -- C ABI of the B200 (sm_100a) dense hot path: BF16 GEMM with FP32
+ * accumulation and a FlashAttention-2 style multi-head-attention forward.
+ *
+ * Every pointer named "device" must be device memory of the CUDA device that
+ * is current on the calling thread.  `stream` is a cudaStream_t passed as
+ * void* (NULL = the legacy default stream).  All calls are asynchronous on
+ * `stream`, allocate no device memory, keep no pointer after returning, and
+ * return an mlt_status (never throw, never exit).  Argument validation runs
+ * before any CUDA call.  Outputs must not alias inputs.
+ *
+ * BF16 values are passed as their 16-bit patterns.
+ */
+#ifndef MLT_H_
+#define MLT_H_
+
+#include <stdint.h>
+
+#ifdef __cplusplus
+extern "C" {
+#endif
+
+typedef enum {
+    MLT_OK = 0,
+    MLT_ERR_INVALID_ARG = 1, /* NULL pointer, negative size, pitch < row width, causal with Nq > Nk, Nk == 0, scale <= 0 */
+    MLT_ERR_UNSUPPORTED = 2, /* head dimension other than 64 or 128; size beyond a TMA descriptor's range */
+    MLT_ERR_ALIGNMENT = 3,   /* base pointer not 16-byte aligned, or pitch not a multiple of 8 elements */
+    MLT_ERR_CUDA = 4,        /* a CUDA runtime / driver call failed */
+    MLT_ERR_ARCH = 5,        /* current device is not compute capability 10.x */
+    MLT_ERR_TIMEOUT = 6      /* a bounded device-side wait expired (reported by mlt_last_device_error) */
+} mlt_status;
+
+/*
+ * C = A * B  (paper Sec. 2: A in R^{m x k}, B in R^{k x n}, C in R^{m x n};
+ * Listing 2: zero-initialised accumulator, K loop of tile dots, one store).
+ * Reading taken: C is overwritten, its prior contents are ignored.
+ *
+ *   A  device, BF16, M x K row-major, A[i*lda + k]
+ *   B  device, BF16, K x N row-major, B[k*ldb + j]
+ *   C  device, BF16 out, M x N row-major, C[i*ldc + j]; products accumulate in
+ *      FP32 and are rounded once, to nearest even
+ *   lda, ldb, ldc  row pitches in ELEMENTS, each >= the row width and a multiple
+ *      of 8 (16-byte rows for the TMA descriptors); base pointers 16-byte aligned
+ *
+ * M == 0 or N == 0: MLT_OK, nothing launched.  K == 0: C is zero-filled.
+ * Any M, N, K otherwise (ragged tiles are zero-filled on load, clipped on store).
+ */
+int mlt_gemm(const void* A, const void* B, void* C,
+             int64_t M, int64_t N, int64_t K,
+             int64_t lda, int64_t ldb, int64_t ldc,
+             void* stream);
+
+/*
+ * O = softmax(scale * Q K^T [+ causal mask]) V,  LSE = log-sum-exp of the
+ * scaled, masked scores (natural log)  -- paper Sec. 2.5, Algorithm 1
+ * (FlashAttention-2 forward: per Q block, loop over K/V blocks, S = Q K_j^T,
+ * online softmax with running row max m and row sum l, O += P V_j, store O).
+ * The scale, the mask, the final 1/l and the LSE output are the benchmark
+ * configuration's; the algorithm box leaves them implicit.
+ *
+ *   Q      device, BF16, [B, H, Nq, D] contiguous (D fastest)
+ *   K, V   device, BF16, [B, H, Nk, D] contiguous
+ *   O      device, BF16 out, [B, H, Nq, D]
+ *   LSE    device, FP32 out, [B, H, Nq], or NULL to skip it
+ *   D      64 or 128
+ *   causal non-zero: key j is visible to query i iff j <= i + (Nk - Nq)
+ *          (bottom-right aligned; requires Nq <= Nk)
+ *   scale  multiplies the raw dot products (typically 1/sqrt(D)); must be finite and > 0
+ *
+ * B*H*Nq == 0: MLT_OK, nothing launched.  Nk == 0: MLT_ERR_INVALID_ARG.
+ * P is rounded to BF16 for the second product; S, m, l and O accumulate in FP32.
+ */
+int mlt_mha_fwd(const void* Q, const void* K, const void* V,
+                void* O, float* LSE,
+                int B, int H, int Nq, int Nk, int D,
+                int causal, float scale, void* stream);
+
+/*
+ * Device-side health word.  Kernels never trap: a wait that exceeds its bound
+ * records {code, barrier id, block} in a per-device status word and the kernel
+ * drains and returns.  This call synchronises the current device, reads and
+ * clears that word, and returns MLT_OK, MLT_ERR_TIMEOUT or MLT_ERR_CUDA.
+ * detail (host, may be NULL) receives 4 words: code, barrier id, block, aux.
+ * (Library addition; the paper has no counterpart.)
+ */
+int mlt_last_device_error(uint32_t* detail);
+
+/* Text for an mlt_status value (static storage). */
+const char* mlt_status_string(int status);
+
+/* Library version: major*10000 + minor*100 + patch. */
+int mlt_version(void);
+
+#ifdef __cplusplus
+}
+#endif
+#endif /* MLT_H_ */

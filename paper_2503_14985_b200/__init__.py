@@ -1,0 +1,8 @@
+"""B200 (sm_100a) dense hot path: BF16 GEMM and FlashAttention-2 style MHA forward.
+
+`binding` wraps the C ABI of include/mlt.h (libmlt.so, built by `build`);
+`inputs` holds the seeded synthetic workloads.  Nothing here computes on the CPU.
+"""
+from . import inputs  # noqa: F401
+from .binding import (MltError, gemm, gemm_raw, last_device_error, load, mha_fwd, mha_fwd_raw,  # noqa: F401
+                      status_string, version)

@@ -1,0 +1,219 @@
+// BF16 GEMM C = A * B with FP32 accumulation in tensor memory (paper Sec. 2,
+// Listing 2: per output tile, a K loop of tile dots into a zero-initialised
+// accumulator, then one store).
+//
+// One persistent CTA per SM, 6 warps with fixed roles:
+//   warp 0      TMA producer: A tile (BM x 64, K-major) and B tile (64 x BN, N contiguous) per stage
+//   warp 1      UMMA issuer (one elected lane) and owner of the tensor-memory allocation
+//   warps 2-5   epilogue: TMEM -> registers -> BF16 -> global, overlapped with the next tile's main loop
+// Tile 128 x BN x 64, kStages-deep smem ring guarded by full/empty mbarriers; two
+// accumulators in TMEM (2 x BN columns) guarded by acc_full/acc_empty mbarriers.
+#pragma once
+
+#include "ptx.cuh"
+
+namespace mlt {
+
+constexpr int kGemmBM = 128;
+constexpr int kGemmBK = 64;
+constexpr int kGemmThreads = 192;
+
+template <int BN, int kStages>
+struct GemmSmem {
+    static constexpr int kABytes = kGemmBM * kGemmBK * 2;  // 16 KB
+    static constexpr int kBBytes = kGemmBK * BN * 2;       // 64 rows x BN, as BN/64 boxes of 64 x 64
+    static constexpr int kStageBytes = kABytes + kBBytes;
+    static constexpr int kBarrierBytes = 256;
+    static constexpr int kTotal = kStages * kStageBytes + kBarrierBytes + 1024;  // + alignment slack
+};
+
+struct GemmParams {
+    __nv_bfloat16* C;
+    int64_t ldc;
+    int M, N, K;
+    int tiles_m, tiles_n;
+    int group_m;  // M-tiles per raster group
+};
+
+// tile index -> (tile_m, tile_n): groups of `group_m` M-tiles, M fastest inside a group, so that
+// the CTAs running at the same time share few A and B panels (L2 reuse).
+__device__ __forceinline__ void gemm_tile_coords(const GemmParams& p, int tile, int& tm, int& tn) {
+    const int per_group = p.group_m * p.tiles_n;
+    const int g = tile / per_group;
+    const int first_m = g * p.group_m;
+    const int rows = min(p.group_m, p.tiles_m - first_m);
+    const int r = tile - g * per_group;
+    tm = first_m + r % rows;
+    tn = r / rows;
+}
+
+template <int BN, int kStages>
+__global__ void __launch_bounds__(kGemmThreads, 1)
+gemm_bf16_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_constant__ CUtensorMap tmap_b,
+                 const GemmParams p) {
+    using L = GemmSmem<BN, kStages>;
+    extern __shared__ uint8_t smem_raw[];
+    uint8_t* smem = reinterpret_cast<uint8_t*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~uintptr_t(1023));
+    uint64_t* bars = reinterpret_cast<uint64_t*>(smem + kStages * L::kStageBytes);
+    uint64_t* full = bars;                     // [kStages]  TMA -> MMA
+    uint64_t* empty = bars + kStages;          // [kStages]  MMA -> TMA
+    uint64_t* acc_full = bars + 2 * kStages;   // [2]        MMA -> epilogue
+    uint64_t* acc_empty = acc_full + 2;        // [2]        epilogue -> MMA
+    uint32_t* tmem_base_slot = reinterpret_cast<uint32_t*>(acc_empty + 2);
+    volatile uint32_t* abort_flag = tmem_base_slot + 1;
+
+    const int warp = threadIdx.x >> 5;
+    const int lane = threadIdx.x & 31;
+    const int num_tiles = p.tiles_m * p.tiles_n;
+    const int num_kb = (p.K + kGemmBK - 1) / kGemmBK;
+    constexpr uint32_t kTmemCols = 2 * BN;  // 512 for BN = 256, 256 for BN = 128
+
+    if (threadIdx.x == 0) {
+        for (int s = 0; s < kStages; ++s) {
+            mbar_init(&full[s], 1);
+            mbar_init(&empty[s], 1);
+        }
+        for (int a = 0; a < 2; ++a) {
+            mbar_init(&acc_full[a], 1);
+            mbar_init(&acc_empty[a], 4);  // one arrive per epilogue warp
+        }
+        *abort_flag = 0;
+        fence_mbar_init();
+    }
+    if (warp == 0 && lane == 0) {
+        prefetch_tensormap(&tmap_a);
+        prefetch_tensormap(&tmap_b);
+    }
+    if (warp == 1) {
+        tmem_alloc(tmem_base_slot, kTmemCols);
+        tmem_relinquish();
+    }
+    tc_fence_before();
+    __syncthreads();
+    tc_fence_after();
+    const uint32_t tmem_base = *tmem_base_slot;
+
+    if (warp == 0) {
+        // ----------------------------- producer -----------------------------
+        if (lane == 0) {
+            int stage = 0;
+            uint32_t phase = 0;
+            bool ok = true;
+            for (int tile = blockIdx.x; tile < num_tiles && ok; tile += gridDim.x) {
+                int tm, tn;
+                gemm_tile_coords(p, tile, tm, tn);
+                const int m0 = tm * kGemmBM, n0 = tn * BN;
+                for (int kb = 0; kb < num_kb; ++kb) {
+                    ok = mbar_wait(&empty[stage], phase ^ 1, abort_flag, 0x100 + stage);
+                    if (!ok) break;
+                    uint8_t* sa = smem + stage * L::kStageBytes;
+                    uint8_t* sb = sa + L::kABytes;
+                    mbar_arrive_expect_tx(&full[stage], L::kStageBytes);
+                    tma_load_2d(sa, &tmap_a, &full[stage], kb * kGemmBK, m0);
+#pragma unroll
+                    for (int c = 0; c < BN / 64; ++c)
+                        tma_load_2d(sb + c * (kGemmBK * 128), &tmap_b, &full[stage], n0 + c * 64, kb * kGemmBK);
+                    if (++stage == kStages) { stage = 0; phase ^= 1; }
+                }
+            }
+        }
+    } else if (warp == 1) {
+        // ----------------------------- MMA issuer -----------------------------
+        if (lane == 0) {
+            constexpr uint32_t idesc = make_idesc_bf16(kGemmBM, BN, /*a_mn_major=*/false, /*b_mn_major=*/true);
+            int stage = 0;
+            uint32_t phase = 0;
+            int acc = 0;
+            uint32_t acc_phase = 0;
+            bool ok = true;
+            for (int tile = blockIdx.x; tile < num_tiles && ok; tile += gridDim.x) {
+                ok = mbar_wait(&acc_empty[acc], acc_phase ^ 1, abort_flag, 0x300 + acc);
+                if (!ok) break;
+                tc_fence_after();
+                const uint32_t d_tmem = tmem_base + acc * BN;
+                for (int kb = 0; kb < num_kb; ++kb) {
+                    ok = mbar_wait(&full[stage], phase, abort_flag, 0x200 + stage);
+                    if (!ok) break;
+                    tc_fence_after();
+                    const uint32_t sa = smem_u32(smem + stage * L::kStageBytes);
+                    const uint32_t sb = sa + L::kABytes;
+#pragma unroll
+                    for (int k = 0; k < kGemmBK / 16; ++k) {
+                        const uint64_t da = make_sdesc_sw128(sa + k * 32, 16, 1024);
+                        const uint64_t db = make_sdesc_sw128(sb + k * 2048, kGemmBK * 128, 1024);
+                        umma_ss(d_tmem, da, db, idesc, (kb | k) != 0);
+                    }
+                    umma_commit(&empty[stage]);  // frees the smem stage once these UMMAs have read it
+                    if (++stage == kStages) { stage = 0; phase ^= 1; }
+                }
+                if (ok) umma_commit(&acc_full[acc]);
+                if (++acc == 2) { acc = 0; acc_phase ^= 1; }
+            }
+        }
+    } else {
+        // ----------------------------- epilogue -----------------------------
+        const int quarter = warp & 3;  // TMEM lanes this warp may touch: 32*quarter .. +31
+        int acc = 0;
+        uint32_t acc_phase = 0;
+        bool ok = true;
+        for (int tile = blockIdx.x; tile < num_tiles && ok; tile += gridDim.x) {
+            int tm, tn;
+            gemm_tile_coords(p, tile, tm, tn);
+            const int row = tm * kGemmBM + quarter * 32 + lane;
+            const int n0 = tn * BN;
+            ok = __all_sync(0xffffffffu, mbar_wait(&acc_full[acc], acc_phase, abort_flag, 0x400 + acc));
+            if (!ok) break;
+            tc_fence_after();
+            const uint32_t t_row = tmem_base + (static_cast<uint32_t>(quarter * 32) << 16) + acc * BN;
+            __nv_bfloat16* crow = p.C + static_cast<int64_t>(row) * p.ldc;
+#pragma unroll 1
+            for (int c = 0; c < BN / 32; ++c) {
+                uint32_t v[32];
+                tmem_ld_32x32b_x32(t_row + c * 32, v);
+                tmem_wait_ld();
+                const int col0 = n0 + c * 32;
+                if (row < p.M) {
+#pragma unroll
+                    for (int q = 0; q < 4; ++q) {
+                        const int col = col0 + q * 8;
+                        uint4 out;
+                        out.x = pack_bf16x2(__uint_as_float(v[q * 8 + 0]), __uint_as_float(v[q * 8 + 1]));
+                        out.y = pack_bf16x2(__uint_as_float(v[q * 8 + 2]), __uint_as_float(v[q * 8 + 3]));
+                        out.z = pack_bf16x2(__uint_as_float(v[q * 8 + 4]), __uint_as_float(v[q * 8 + 5]));
+                        out.w = pack_bf16x2(__uint_as_float(v[q * 8 + 6]), __uint_as_float(v[q * 8 + 7]));
+                        if (col + 8 <= p.N) {
+                            *reinterpret_cast<uint4*>(crow + col) = out;
+                        } else if (col < p.N) {
+                            const __nv_bfloat16* e = reinterpret_cast<const __nv_bfloat16*>(&out);
+                            for (int j = 0; col + j < p.N; ++j) crow[col + j] = e[j];
+                        }
+                    }
+                }
+            }
+            tc_fence_before();
+            __syncwarp();
+            if (lane == 0) mbar_arrive(&acc_empty[acc]);
+            if (++acc == 2) { acc = 0; acc_phase ^= 1; }
+        }
+    }
+
+    // common exit: every role reaches this, also after an aborted wait
+    tc_fence_before();
+    __syncthreads();
+    if (warp == 1) {
+        __syncwarp();
+        tc_fence_after();
+        tmem_dealloc(tmem_base, kTmemCols);
+    }
+}
+
+// C[i][0..N) = 0 for K == 0 (BLAS convention for an empty sum).
+__global__ void gemm_zero_fill_kernel(__nv_bfloat16* C, int64_t ldc, int M, int N) {
+    const int64_t total = static_cast<int64_t>(M) * N;
+    for (int64_t i = blockIdx.x * static_cast<int64_t>(blockDim.x) + threadIdx.x; i < total;
+         i += static_cast<int64_t>(gridDim.x) * blockDim.x) {
+        C[(i / N) * ldc + (i % N)] = __float2bfloat16(0.0f);
+    }
+}
+
+}  // namespace mlt

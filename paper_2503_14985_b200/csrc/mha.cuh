@@ -1,0 +1,381 @@
+// Multi-head attention forward in the FlashAttention-2 form (paper Sec. 2.5,
+// Algorithm 1): per block of query rows, loop over K/V blocks; S = Q K_j^T on the
+// tensor cores, online softmax with running row max m and row sum l, O += P V_j on
+// the tensor cores, final O / l and LSE = m + ln l.
+//
+// A CTA owns 256 query rows of one (batch, head): two 128-row tiles that take turns
+// on the tensor pipe, so the exponentials of one tile overlap the products of the other.
+//   warps 0-3   softmax / O-rescale / epilogue of tile 0 (one thread per query row)
+//   warps 4-7   the same for tile 1
+//   warp  8     UMMA issuer (one lane) and owner of the tensor-memory allocation
+//   warp  9     TMA loader (one lane): both Q tiles once, then K_0, V_0, K_1, V_1, ... through a ring
+// Tensor memory (512 columns): S_0 | S_1 (128 FP32 columns each; the BF16 P of a tile
+// overwrites the first 64 columns of its S and is consumed from there as the A operand
+// of P V), then O_0 | O_1 (D FP32 columns each).
+#pragma once
+
+#include <math.h>
+
+#include "ptx.cuh"
+
+namespace mlt {
+
+constexpr int kMhaBlock = 128;   // query rows per tile and keys per K/V block
+constexpr int kMhaThreads = 320;
+constexpr float kLog2e = 1.4426950408889634f;
+constexpr float kRescaleThreshold = 8.0f;  // in log2 units: keep a stale max until it is off by more than 2^8
+
+template <int D>
+struct MhaSmem {
+    static constexpr int kTileBytes = kMhaBlock * D * 2;  // one Q, K or V tile: D/64 chunks of 128 rows x 128 B
+    static constexpr int kChunkBytes = kMhaBlock * 128;
+    static constexpr int kStages = (D == 128) ? 4 : 8;
+    static constexpr int kBarrierBytes = 256;
+    static constexpr int kTotal = 2 * kTileBytes + kStages * kTileBytes + kBarrierBytes + 1024;
+};
+
+struct MhaParams {
+    __nv_bfloat16* O;
+    float* LSE;  // may be null
+    int BH, Nq, Nk;
+    int causal;
+    float scale;
+    int num_pairs;   // 256-row query groups per head
+    int head_group;  // heads that share a span of consecutive block indices
+};
+
+// block index -> (pair, bh).  Heads are taken in groups; inside a group the query
+// position is the slow index and runs from the last rows to the first, so under a
+// causal mask the longest items are dispatched first, and the CTAs resident at any
+// time read the K/V of few heads (L2 reuse).
+__device__ __forceinline__ void mha_item(const MhaParams& p, int block, int& pair, int& bh) {
+    const int per_group = p.num_pairs * p.head_group;
+    const int g = block / per_group;
+    const int first = g * p.head_group;
+    const int heads = min(p.head_group, p.BH - first);
+    const int r = block - g * per_group;
+    pair = p.num_pairs - 1 - r / heads;
+    bh = first + r % heads;
+}
+
+template <int D>
+__global__ void __launch_bounds__(kMhaThreads, 1)
+mha_fwd_kernel(const __grid_constant__ CUtensorMap tmap_q, const __grid_constant__ CUtensorMap tmap_k,
+               const __grid_constant__ CUtensorMap tmap_v, const MhaParams p) {
+    using L = MhaSmem<D>;
+    constexpr int kStages = L::kStages;
+    constexpr int kChunks = D / 64;
+    extern __shared__ uint8_t smem_raw[];
+    uint8_t* smem = reinterpret_cast<uint8_t*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~uintptr_t(1023));
+    uint8_t* smem_q = smem;                        // [2][tile]
+    uint8_t* smem_kv = smem + 2 * L::kTileBytes;   // [kStages][tile]
+    uint64_t* bars = reinterpret_cast<uint64_t*>(smem_kv + kStages * L::kTileBytes);
+    uint64_t* q_full = bars;                  // [1]
+    uint64_t* kv_full = bars + 1;             // [kStages]
+    uint64_t* kv_empty = kv_full + kStages;   // [kStages]
+    uint64_t* s_full = kv_empty + kStages;    // [2]  UMMA -> softmax: S_t(j) complete
+    uint64_t* p_full = s_full + 2;            // [2]  softmax -> UMMA: P_t(j) in TMEM, O_t rescaled
+    uint64_t* o_full = p_full + 2;            // [2]  UMMA -> epilogue: O_t complete
+    uint32_t* tmem_base_slot = reinterpret_cast<uint32_t*>(o_full + 2);
+    volatile uint32_t* abort_flag = tmem_base_slot + 1;
+
+    const int warp = threadIdx.x >> 5;
+    const int lane = threadIdx.x & 31;
+
+    int pair, bh;
+    mha_item(p, blockIdx.x, pair, bh);
+    const int q_base = pair * 2 * kMhaBlock;
+    const int shift = p.Nk - p.Nq;  // bottom-right alignment of the causal mask
+    // number of K/V blocks each tile needs
+    int J[2];
+#pragma unroll
+    for (int t = 0; t < 2; ++t) {
+        const int q0 = q_base + t * kMhaBlock;
+        if (q0 >= p.Nq) {
+            J[t] = 0;
+        } else {
+            int last_key = p.Nk - 1;
+            if (p.causal) last_key = min(last_key, min(q0 + kMhaBlock, p.Nq) - 1 + shift);
+            J[t] = last_key / kMhaBlock + 1;
+        }
+    }
+    const int Jmax = max(J[0], J[1]);
+
+    if (threadIdx.x == 0) {
+        mbar_init(q_full, 1);
+        for (int s = 0; s < kStages; ++s) {
+            mbar_init(&kv_full[s], 1);
+            mbar_init(&kv_empty[s], 1);
+        }
+        for (int t = 0; t < 2; ++t) {
+            mbar_init(&s_full[t], 1);
+            mbar_init(&p_full[t], 4);  // one arrive per softmax warp
+            mbar_init(&o_full[t], 1);
+        }
+        *abort_flag = 0;
+        fence_mbar_init();
+    }
+    if (warp == 9 && lane == 0) {
+        prefetch_tensormap(&tmap_q);
+        prefetch_tensormap(&tmap_k);
+        prefetch_tensormap(&tmap_v);
+    }
+    if (warp == 8) {
+        tmem_alloc(tmem_base_slot, 512);
+        tmem_relinquish();
+    }
+    tc_fence_before();
+    __syncthreads();
+    tc_fence_after();
+    const uint32_t tmem_base = *tmem_base_slot;
+    constexpr uint32_t kColS = 0;      // S_t at kColS + t*128
+    constexpr uint32_t kColO = 256;    // O_t at kColO + t*D
+
+    if (warp == 9) {
+        // ------------------------------- loader -------------------------------
+        if (lane == 0) {
+            mbar_arrive_expect_tx(q_full, 2 * L::kTileBytes);
+#pragma unroll
+            for (int t = 0; t < 2; ++t)
+#pragma unroll
+                for (int c = 0; c < kChunks; ++c)
+                    tma_load_3d(smem_q + t * L::kTileBytes + c * L::kChunkBytes, &tmap_q, q_full, c * 64,
+                                q_base + t * kMhaBlock, bh);
+            int stage = 0;
+            uint32_t phase = 0;
+            bool ok = true;
+            for (int j = 0; j < Jmax && ok; ++j) {
+#pragma unroll
+                for (int kv = 0; kv < 2; ++kv) {
+                    ok = mbar_wait(&kv_empty[stage], phase ^ 1, abort_flag, 0x100 + stage);
+                    if (!ok) break;
+                    uint8_t* dst = smem_kv + stage * L::kTileBytes;
+                    mbar_arrive_expect_tx(&kv_full[stage], L::kTileBytes);
+#pragma unroll
+                    for (int c = 0; c < kChunks; ++c)
+                        tma_load_3d(dst + c * L::kChunkBytes, kv == 0 ? &tmap_k : &tmap_v, &kv_full[stage], c * 64,
+                                    j * kMhaBlock, bh);
+                    if (++stage == kStages) { stage = 0; phase ^= 1; }
+                }
+            }
+        }
+    } else if (warp == 8) {
+        // ------------------------------- UMMA issuer -------------------------------
+        if (lane == 0) {
+            constexpr uint32_t idesc_qk = make_idesc_bf16(kMhaBlock, kMhaBlock, false, false);
+            constexpr uint32_t idesc_pv = make_idesc_bf16(kMhaBlock, D, false, true);
+            int stage = 0;
+            uint32_t phase = 0;
+            bool ok = true;
+            // S_t = Q_t K^T over the D/16 k-steps of the tile in ring slot `slot`
+            auto issue_qk = [&](int t, int slot) {
+                const uint32_t q_addr = smem_u32(smem_q + t * L::kTileBytes);
+                const uint32_t k_addr = smem_u32(smem_kv + slot * L::kTileBytes);
+#pragma unroll
+                for (int kk = 0; kk < D / 16; ++kk) {
+                    const uint32_t off = (kk / 4) * L::kChunkBytes + (kk % 4) * 32;
+                    umma_ss(tmem_base + kColS + t * kMhaBlock, make_sdesc_sw128(q_addr + off, 16, 1024),
+                            make_sdesc_sw128(k_addr + off, 16, 1024), idesc_qk, kk != 0);
+                }
+                umma_commit(&s_full[t]);
+            };
+            // O_t (+)= P_t V over the 8 k-steps (16 keys each) of the tile in ring slot `slot`
+            auto issue_pv = [&](int t, int slot, bool first) {
+                const uint32_t v_addr = smem_u32(smem_kv + slot * L::kTileBytes);
+#pragma unroll
+                for (int kk = 0; kk < kMhaBlock / 16; ++kk)
+                    umma_ts(tmem_base + kColO + t * D, tmem_base + kColS + t * kMhaBlock + kk * 8,
+                            make_sdesc_sw128(v_addr + kk * 2048, L::kChunkBytes, 1024), idesc_pv, !(first && kk == 0));
+            };
+            if (Jmax > 0) {
+                ok = mbar_wait(q_full, 0, abort_flag, 0x200);
+                if (ok) ok = mbar_wait(&kv_full[stage], phase, abort_flag, 0x210 + stage);
+                if (ok) {
+                    tc_fence_after();
+                    for (int t = 0; t < 2; ++t)
+                        if (J[t] > 0) issue_qk(t, stage);
+                    umma_commit(&kv_empty[stage]);
+                    if (++stage == kStages) { stage = 0; phase ^= 1; }
+                }
+            }
+            for (int j = 0; j < Jmax && ok; ++j) {
+                const int vslot = stage;
+                ok = mbar_wait(&kv_full[vslot], phase, abort_flag, 0x220 + vslot);
+                if (!ok) break;
+                if (++stage == kStages) { stage = 0; phase ^= 1; }
+                const int kslot = stage;  // K_{j+1}, if there is one
+                bool k_ready = false;
+                for (int t = 0; t < 2 && ok; ++t) {
+                    if (j >= J[t]) continue;
+                    ok = mbar_wait(&p_full[t], j & 1, abort_flag, 0x230 + t);
+                    if (!ok) break;
+                    tc_fence_after();
+                    issue_pv(t, vslot, j == 0);
+                    if (j == J[t] - 1) umma_commit(&o_full[t]);
+                    if (j + 1 < J[t]) {
+                        if (!k_ready) {
+                            ok = mbar_wait(&kv_full[kslot], phase, abort_flag, 0x240 + kslot);
+                            if (!ok) break;
+                            tc_fence_after();
+                            k_ready = true;
+                        }
+                        issue_qk(t, kslot);
+                    }
+                }
+                if (!ok) break;
+                umma_commit(&kv_empty[vslot]);
+                if (j + 1 < Jmax) {
+                    umma_commit(&kv_empty[kslot]);
+                    if (++stage == kStages) { stage = 0; phase ^= 1; }
+                }
+            }
+        }
+    } else {
+        // ------------------- softmax, O rescale and epilogue of tile t -------------------
+        const int t = warp >> 2;
+        const int quarter = warp & 3;
+        const int row_in_tile = quarter * 32 + lane;
+        const int qi = q_base + t * kMhaBlock + row_in_tile;  // query index inside the head
+        const uint32_t lane_addr = tmem_base + (static_cast<uint32_t>(quarter * 32) << 16);
+        const uint32_t s_addr = lane_addr + kColS + t * kMhaBlock;
+        const uint32_t o_addr = lane_addr + kColO + t * D;
+        const float c = p.scale * kLog2e;
+        const int Jt = J[t];
+        const int limit = p.causal ? min(p.Nk - 1, qi + shift) : p.Nk - 1;  // last visible key of this row
+        float m_run = -INFINITY;  // reference max (raw score units); may lag the true max by < 2^8 in exp2 units
+        float l_run = 0.0f;
+        bool ok = true;
+
+        for (int j = 0; j < Jt; ++j) {
+            ok = __all_sync(0xffffffffu, mbar_wait(&s_full[t], j & 1, abort_flag, 0x300 + t));
+            if (!ok) break;
+            tc_fence_after();
+            uint32_t sr[128];
+#pragma unroll
+            for (int q = 0; q < 4; ++q) tmem_ld_32x32b_x32(s_addr + q * 32, *reinterpret_cast<uint32_t(*)[32]>(&sr[q * 32]));
+            tmem_wait_ld();
+            float* s = reinterpret_cast<float*>(sr);
+            const int j0 = j * kMhaBlock;
+            if (j0 + kMhaBlock - 1 > limit) {  // diagonal or tail block: mask keys beyond the row's last visible one
+#pragma unroll
+                for (int i = 0; i < 128; ++i)
+                    if (j0 + i > limit) s[i] = -INFINITY;
+            }
+            float mx = s[0];
+#pragma unroll
+            for (int i = 1; i < 128; ++i) mx = fmaxf(mx, s[i]);
+            // lazy rescale: move the reference max only when it is off by more than the threshold
+            float alpha = 1.0f;
+            bool moved = false;
+            if (j == 0) {
+                m_run = mx;
+            } else if ((mx - m_run) * c > kRescaleThreshold || (m_run == -INFINITY && mx > -INFINITY)) {
+                alpha = (m_run == -INFINITY) ? 0.0f : fast_exp2((m_run - mx) * c);
+                m_run = mx;
+                moved = true;
+            }
+            if (__any_sync(0xffffffffu, moved)) {
+                // S_t(j) complete implies every earlier UMMA, so P_t(j-1) V has landed in O_t
+#pragma unroll 1
+                for (int q = 0; q < D / 32; ++q) {
+                    uint32_t o[32];
+                    tmem_ld_32x32b_x32(o_addr + q * 32, o);
+                    tmem_wait_ld();
+#pragma unroll
+                    for (int i = 0; i < 32; ++i) o[i] = __float_as_uint(__uint_as_float(o[i]) * alpha);
+                    tmem_st_32x32b_x32(o_addr + q * 32, o);
+                }
+                l_run *= alpha;
+            }
+            const float neg_mc = (m_run == -INFINITY) ? 0.0f : -m_run * c;
+            float sum = 0.0f;
+            uint32_t pk[64];
+#pragma unroll
+            for (int i = 0; i < 64; ++i) {
+                const float p0 = fast_exp2(fmaf(s[2 * i], c, neg_mc));
+                const float p1 = fast_exp2(fmaf(s[2 * i + 1], c, neg_mc));
+                sum += p0 + p1;
+                pk[i] = pack_bf16x2(p0, p1);
+            }
+            l_run += sum;
+            tmem_st_32x32b_x32(s_addr, *reinterpret_cast<uint32_t(*)[32]>(&pk[0]));
+            tmem_st_32x32b_x32(s_addr + 32, *reinterpret_cast<uint32_t(*)[32]>(&pk[32]));
+            tmem_wait_st();
+            tc_fence_before();
+            __syncwarp();
+            if (lane == 0) mbar_arrive(&p_full[t]);
+        }
+
+        if (ok && Jt > 0) {
+            ok = __all_sync(0xffffffffu, mbar_wait(&o_full[t], 0, abort_flag, 0x400 + t));
+            if (ok) {
+                tc_fence_after();
+                const float inv_l = 1.0f / l_run;
+                const bool valid = qi < p.Nq;
+                __nv_bfloat16* orow = p.O + (static_cast<int64_t>(bh) * p.Nq + qi) * D;
+#pragma unroll 1
+                for (int q = 0; q < D / 32; ++q) {
+                    uint32_t o[32];
+                    tmem_ld_32x32b_x32(o_addr + q * 32, o);
+                    tmem_wait_ld();
+                    if (valid) {
+#pragma unroll
+                        for (int v = 0; v < 4; ++v) {
+                            uint4 out;
+                            out.x = pack_bf16x2(__uint_as_float(o[v * 8 + 0]) * inv_l, __uint_as_float(o[v * 8 + 1]) * inv_l);
+                            out.y = pack_bf16x2(__uint_as_float(o[v * 8 + 2]) * inv_l, __uint_as_float(o[v * 8 + 3]) * inv_l);
+                            out.z = pack_bf16x2(__uint_as_float(o[v * 8 + 4]) * inv_l, __uint_as_float(o[v * 8 + 5]) * inv_l);
+                            out.w = pack_bf16x2(__uint_as_float(o[v * 8 + 6]) * inv_l, __uint_as_float(o[v * 8 + 7]) * inv_l);
+                            *reinterpret_cast<uint4*>(orow + q * 32 + v * 8) = out;
+                        }
+                    }
+                }
+                if (valid && p.LSE) p.LSE[static_cast<int64_t>(bh) * p.Nq + qi] = m_run * p.scale + logf(l_run);
+            }
+        }
+    }
+
+    // common exit: every role reaches this, also after an aborted wait
+    tc_fence_before();
+    __syncthreads();
+    if (warp == 8) {
+        __syncwarp();
+        tc_fence_after();
+        tmem_dealloc(tmem_base, 512);
+    }
+}
+
+inline int mha_configure() {
+    if (cudaFuncSetAttribute(mha_fwd_kernel<64>, cudaFuncAttributeMaxDynamicSharedMemorySize, MhaSmem<64>::kTotal) !=
+        cudaSuccess)
+        return 1;
+    if (cudaFuncSetAttribute(mha_fwd_kernel<128>, cudaFuncAttributeMaxDynamicSharedMemorySize, MhaSmem<128>::kTotal) !=
+        cudaSuccess)
+        return 1;
+    return 0;
+}
+
+inline int mha_launch(const CUtensorMap& tq, const CUtensorMap& tk, const CUtensorMap& tv, __nv_bfloat16* O, float* LSE,
+                      int B, int H, int Nq, int Nk, int D, bool causal, float scale, int sm_count, cudaStream_t st) {
+    (void)sm_count;
+    MhaParams p;
+    p.O = O;
+    p.LSE = LSE;
+    p.BH = B * H;
+    p.Nq = Nq;
+    p.Nk = Nk;
+    p.causal = causal ? 1 : 0;
+    p.scale = scale;
+    p.num_pairs = (Nq + 2 * kMhaBlock - 1) / (2 * kMhaBlock);
+    p.head_group = 8;
+    const int64_t items = static_cast<int64_t>(p.num_pairs) * p.BH;
+    if (items > INT32_MAX) return 2;
+    const int grid = static_cast<int>(items);
+    if (D == 64)
+        mha_fwd_kernel<64><<<grid, kMhaThreads, MhaSmem<64>::kTotal, st>>>(tq, tk, tv, p);
+    else
+        mha_fwd_kernel<128><<<grid, kMhaThreads, MhaSmem<128>::kTotal, st>>>(tq, tk, tv, p);
+    return cudaGetLastError() == cudaSuccess ? 0 : 4;
+}
+
+}  // namespace mlt

@@ -1,0 +1,237 @@
+// Host side of the C ABI declared in include/mlt.h: argument validation, TMA
+// descriptor encoding, launch configuration.  All arithmetic of the hot path runs
+// in the kernels of gemm.cuh and mha.cuh.
+#include <cuda.h>
+#include <cuda_runtime.h>
+
+#include <atomic>
+#include <cstdint>
+#include <cstdlib>
+#include <cstring>
+#include <mutex>
+
+#include "../../include/mlt.h"
+#include "gemm.cuh"
+#include "mha.cuh"
+
+namespace {
+
+using namespace mlt;
+
+typedef CUresult (*EncodeTiledFn)(CUtensorMap*, CUtensorMapDataType, cuuint32_t, void*, const cuuint64_t*,
+                                  const cuuint64_t*, const cuuint32_t*, const cuuint32_t*, CUtensorMapInterleave,
+                                  CUtensorMapSwizzle, CUtensorMapL2promotion, CUtensorMapFloatOOBfill);
+
+struct DeviceInfo {
+    int sm_count = 0;
+    int cc_major = 0;
+    bool configured = false;
+};
+
+std::mutex g_mutex;
+EncodeTiledFn g_encode = nullptr;
+DeviceInfo g_devices[64];
+
+// Looks up cuTensorMapEncodeTiled through the runtime, so libcuda is not a link-time dependency.
+int get_encoder(EncodeTiledFn* out) {
+    std::lock_guard<std::mutex> lock(g_mutex);
+    if (!g_encode) {
+        void* fn = nullptr;
+        cudaDriverEntryPointQueryResult qres;
+        cudaError_t e = cudaGetDriverEntryPoint("cuTensorMapEncodeTiled", &fn, cudaEnableDefault, &qres);
+        if (e != cudaSuccess || qres != cudaDriverEntryPointSuccess || !fn) return MLT_ERR_CUDA;
+        g_encode = reinterpret_cast<EncodeTiledFn>(fn);
+    }
+    *out = g_encode;
+    return MLT_OK;
+}
+
+template <class Kernel>
+int set_smem(Kernel k, int bytes) {
+    return cudaFuncSetAttribute(k, cudaFuncAttributeMaxDynamicSharedMemorySize, bytes) == cudaSuccess ? MLT_OK
+                                                                                                     : MLT_ERR_CUDA;
+}
+
+// Once per device: capability check and the shared-memory opt-in of every kernel.
+int get_device(DeviceInfo* out) {
+    int dev = 0;
+    if (cudaGetDevice(&dev) != cudaSuccess || dev < 0 || dev >= 64) return MLT_ERR_CUDA;
+    std::lock_guard<std::mutex> lock(g_mutex);
+    DeviceInfo& d = g_devices[dev];
+    if (!d.configured) {
+        if (cudaDeviceGetAttribute(&d.cc_major, cudaDevAttrComputeCapabilityMajor, dev) != cudaSuccess ||
+            cudaDeviceGetAttribute(&d.sm_count, cudaDevAttrMultiProcessorCount, dev) != cudaSuccess)
+            return MLT_ERR_CUDA;
+        if (d.cc_major != 10) return MLT_ERR_ARCH;
+        if (set_smem(gemm_bf16_kernel<256, 4>, GemmSmem<256, 4>::kTotal) != MLT_OK ||
+            set_smem(gemm_bf16_kernel<128, 6>, GemmSmem<128, 6>::kTotal) != MLT_OK)
+            return MLT_ERR_CUDA;
+        if (mha_configure() != MLT_OK) return MLT_ERR_CUDA;
+        d.configured = true;
+    }
+    *out = d;
+    return MLT_OK;
+}
+
+// BF16 tensor map with 128-byte swizzle.  dims / strides innermost first; strides[0] is implicit.
+int encode_bf16(CUtensorMap* map, const void* base, int rank, const uint64_t* dims, const uint64_t* strides_bytes,
+                const uint32_t* box) {
+    EncodeTiledFn enc;
+    int rc = get_encoder(&enc);
+    if (rc != MLT_OK) return rc;
+    cuuint64_t gdim[5];
+    cuuint64_t gstride[5];
+    cuuint32_t gbox[5];
+    cuuint32_t estr[5];
+    for (int i = 0; i < rank; ++i) {
+        if (dims[i] == 0 || dims[i] > (1ull << 32)) return MLT_ERR_UNSUPPORTED;
+        gdim[i] = dims[i];
+        gbox[i] = box[i];
+        estr[i] = 1;
+        if (i > 0) {
+            if (strides_bytes[i - 1] >= (1ull << 40) || strides_bytes[i - 1] % 16) return MLT_ERR_UNSUPPORTED;
+            gstride[i - 1] = strides_bytes[i - 1];
+        }
+    }
+    CUresult r = enc(map, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, static_cast<cuuint32_t>(rank), const_cast<void*>(base),
+                     gdim, gstride, gbox, estr, CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B,
+                     CU_TENSOR_MAP_L2_PROMOTION_L2_256B, CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
+    return r == CUDA_SUCCESS ? MLT_OK : MLT_ERR_CUDA;
+}
+
+inline bool aligned16(const void* p) { return (reinterpret_cast<uintptr_t>(p) & 15u) == 0; }
+
+}  // namespace
+
+extern "C" {
+
+int mlt_version(void) { return 100; }
+
+const char* mlt_status_string(int status) {
+    switch (status) {
+        case MLT_OK: return "ok";
+        case MLT_ERR_INVALID_ARG: return "invalid argument";
+        case MLT_ERR_UNSUPPORTED: return "unsupported size or head dimension";
+        case MLT_ERR_ALIGNMENT: return "pointer not 16-byte aligned or pitch not a multiple of 8 elements";
+        case MLT_ERR_CUDA: return "CUDA runtime or driver call failed";
+        case MLT_ERR_ARCH: return "device is not compute capability 10.x (sm_100a required)";
+        case MLT_ERR_TIMEOUT: return "a bounded device-side wait expired";
+        default: return "unknown status";
+    }
+}
+
+int mlt_last_device_error(uint32_t* detail) {
+    if (cudaDeviceSynchronize() != cudaSuccess) return MLT_ERR_CUDA;
+    unsigned int host[4] = {0, 0, 0, 0};
+    if (cudaMemcpyFromSymbol(host, g_status, sizeof host) != cudaSuccess) return MLT_ERR_CUDA;
+    if (detail) std::memcpy(detail, host, sizeof host);
+    if (host[0] != 0) {
+        unsigned int zero[4] = {0, 0, 0, 0};
+        if (cudaMemcpyToSymbol(g_status, zero, sizeof zero) != cudaSuccess) return MLT_ERR_CUDA;
+        return host[0] == kStatusTimeout ? MLT_ERR_TIMEOUT : MLT_ERR_CUDA;
+    }
+    return MLT_OK;
+}
+
+int mlt_gemm(const void* A, const void* B, void* C, int64_t M, int64_t N, int64_t K, int64_t lda, int64_t ldb,
+             int64_t ldc, void* stream) {
+    // ---- validation (no CUDA call before this block has passed) ----
+    if (M < 0 || N < 0 || K < 0) return MLT_ERR_INVALID_ARG;
+    if (M == 0 || N == 0) return MLT_OK;
+    if (!C || ldc < N) return MLT_ERR_INVALID_ARG;
+    if (K > 0 && (!A || !B || lda < K || ldb < N)) return MLT_ERR_INVALID_ARG;
+    if (M > INT32_MAX - 256 || N > INT32_MAX - 256 || K > INT32_MAX - 256) return MLT_ERR_UNSUPPORTED;
+    if (!aligned16(C) || (ldc % 8) != 0) return MLT_ERR_ALIGNMENT;
+    if (K > 0 && (!aligned16(A) || !aligned16(B) || (lda % 8) != 0 || (ldb % 8) != 0)) return MLT_ERR_ALIGNMENT;
+
+    DeviceInfo dev;
+    int rc = get_device(&dev);
+    if (rc != MLT_OK) return rc;
+    cudaStream_t st = static_cast<cudaStream_t>(stream);
+
+    if (K == 0) {
+        const int64_t total = M * N;
+        const int blocks = static_cast<int>(std::min<int64_t>((total + 255) / 256, 4 * dev.sm_count));
+        gemm_zero_fill_kernel<<<blocks, 256, 0, st>>>(static_cast<__nv_bfloat16*>(C), ldc, static_cast<int>(M),
+                                                      static_cast<int>(N));
+        return cudaGetLastError() == cudaSuccess ? MLT_OK : MLT_ERR_CUDA;
+    }
+
+    // 128 x 256 tiles unless that leaves most SMs idle; then 128 x 128.
+    const int64_t tiles_m = (M + kGemmBM - 1) / kGemmBM;
+    const bool wide = tiles_m * ((N + 255) / 256) >= dev.sm_count;
+    const int bn = wide ? 256 : 128;
+    const int64_t tiles_n = (N + bn - 1) / bn;
+    if (tiles_m * tiles_n > INT32_MAX) return MLT_ERR_UNSUPPORTED;
+
+    CUtensorMap ta, tb;
+    {
+        const uint64_t dims[2] = {static_cast<uint64_t>(K), static_cast<uint64_t>(M)};
+        const uint64_t strides[1] = {static_cast<uint64_t>(lda) * 2};
+        const uint32_t box[2] = {kGemmBK, kGemmBM};
+        rc = encode_bf16(&ta, A, 2, dims, strides, box);
+        if (rc != MLT_OK) return rc;
+    }
+    {
+        const uint64_t dims[2] = {static_cast<uint64_t>(N), static_cast<uint64_t>(K)};
+        const uint64_t strides[1] = {static_cast<uint64_t>(ldb) * 2};
+        const uint32_t box[2] = {64, kGemmBK};
+        rc = encode_bf16(&tb, B, 2, dims, strides, box);
+        if (rc != MLT_OK) return rc;
+    }
+
+    GemmParams p;
+    p.C = static_cast<__nv_bfloat16*>(C);
+    p.ldc = ldc;
+    p.M = static_cast<int>(M);
+    p.N = static_cast<int>(N);
+    p.K = static_cast<int>(K);
+    p.tiles_m = static_cast<int>(tiles_m);
+    p.tiles_n = static_cast<int>(tiles_n);
+    p.group_m = 16;
+    const int grid = static_cast<int>(std::min<int64_t>(tiles_m * tiles_n, dev.sm_count));
+    if (wide)
+        gemm_bf16_kernel<256, 4><<<grid, kGemmThreads, GemmSmem<256, 4>::kTotal, st>>>(ta, tb, p);
+    else
+        gemm_bf16_kernel<128, 6><<<grid, kGemmThreads, GemmSmem<128, 6>::kTotal, st>>>(ta, tb, p);
+    return cudaGetLastError() == cudaSuccess ? MLT_OK : MLT_ERR_CUDA;
+}
+
+int mlt_mha_fwd(const void* Q, const void* K, const void* V, void* O, float* LSE, int B, int H, int Nq, int Nk, int D,
+                int causal, float scale, void* stream) {
+    if (B < 0 || H < 0 || Nq < 0 || Nk < 0) return MLT_ERR_INVALID_ARG;
+    if (static_cast<int64_t>(B) * H * Nq == 0) return MLT_OK;
+    if (Nk == 0) return MLT_ERR_INVALID_ARG;
+    if (!Q || !K || !V || !O) return MLT_ERR_INVALID_ARG;
+    if (causal && Nq > Nk) return MLT_ERR_INVALID_ARG;
+    if (!(scale > 0.0f) || scale > 3.0e38f) return MLT_ERR_INVALID_ARG;  // zero, negative, NaN or infinite
+    if (D != 64 && D != 128) return MLT_ERR_UNSUPPORTED;
+    if (static_cast<int64_t>(B) * H > INT32_MAX / 2) return MLT_ERR_UNSUPPORTED;
+    if (!aligned16(Q) || !aligned16(K) || !aligned16(V) || !aligned16(O)) return MLT_ERR_ALIGNMENT;
+
+    DeviceInfo dev;
+    int rc = get_device(&dev);
+    if (rc != MLT_OK) return rc;
+
+    CUtensorMap tq, tk, tv;
+    const uint64_t bh = static_cast<uint64_t>(B) * H;
+    const uint32_t box[3] = {64, kMhaBlock, 1};
+    {
+        const uint64_t dims[3] = {static_cast<uint64_t>(D), static_cast<uint64_t>(Nq), bh};
+        const uint64_t strides[2] = {static_cast<uint64_t>(D) * 2, static_cast<uint64_t>(Nq) * D * 2};
+        rc = encode_bf16(&tq, Q, 3, dims, strides, box);
+        if (rc != MLT_OK) return rc;
+    }
+    {
+        const uint64_t dims[3] = {static_cast<uint64_t>(D), static_cast<uint64_t>(Nk), bh};
+        const uint64_t strides[2] = {static_cast<uint64_t>(D) * 2, static_cast<uint64_t>(Nk) * D * 2};
+        rc = encode_bf16(&tk, K, 3, dims, strides, box);
+        if (rc != MLT_OK) return rc;
+        rc = encode_bf16(&tv, V, 3, dims, strides, box);
+        if (rc != MLT_OK) return rc;
+    }
+    return mha_launch(tq, tk, tv, static_cast<__nv_bfloat16*>(O), LSE, B, H, Nq, Nk, D, causal != 0, scale,
+                      dev.sm_count, static_cast<cudaStream_t>(stream));
+}
+
+}  // extern "C"

@@ -1,0 +1,55 @@
+"""The C-ABI library: loads without a GPU, exports every declared symbol, validates before touching CUDA."""
+import ctypes
+import os
+import re
+
+import pytest
+
+import __graft_entry__ as entry
+from paper_2503_14985_b200 import binding
+
+ROOT = os.path.dirname(os.path.dirname(os.path.abspath(__file__)))
+
+
+@pytest.fixture(scope="module")
+def lib():
+    entry.build()
+    return binding.load()
+
+
+def test_header_symbols_are_exported(lib):
+    header = open(os.path.join(ROOT, "include", "mlt.h")).read()
+    declared = set(re.findall(r"^(?:int|const char\*)\s+(mlt_[a-z_0-9]+)\s*\(", header, flags=re.M))
+    assert declared >= set(binding.EXPORTS)
+    for name in declared:
+        assert hasattr(lib, name), f"{name} declared in mlt.h but not exported"
+
+
+def test_version_and_status_strings(lib):
+    assert binding.version() >= 100
+    texts = {binding.status_string(i) for i in range(7)}
+    assert len(texts) == 7 and "unknown status" not in texts
+    assert binding.status_string(99) == "unknown status"
+
+
+def test_validation_precedes_cuda(lib):
+    # none of these may reach a CUDA call (there may be no GPU here): the status must be the validation one
+    assert binding.gemm_raw(0, 0, 0, -1, 1, 1, 8, 8, 8) == 1
+    assert binding.gemm_raw(0, 0, 0, 0, 8, 8, 8, 8, 8) == 0
+    assert binding.gemm_raw(16, 16, 0, 4, 4, 4, 8, 8, 8) == 1
+    assert binding.gemm_raw(16, 16, 16, 4, 4, 4, 8, 8, 2) == 1
+    assert binding.gemm_raw(16, 16, 16, 4, 4, 4, 8, 8, 12) == 3
+    assert binding.gemm_raw(16, 16, 18, 4, 4, 4, 8, 8, 8) == 3
+    assert binding.mha_fwd_raw(16, 16, 16, 16, 0, 1, 1, 8, 8, 80, 0, 1.0) == 2
+    assert binding.mha_fwd_raw(16, 16, 16, 16, 0, 1, 1, 9, 8, 64, 1, 1.0) == 1
+    assert binding.mha_fwd_raw(16, 16, 16, 16, 0, 0, 4, 9, 8, 64, 0, 1.0) == 0
+    assert binding.mha_fwd_raw(16, 16, 16, 16, 0, 1, 1, 8, 8, 64, 0, float("nan")) == 1
+
+
+def test_product_does_not_import_oracle():
+    pkg = os.path.join(ROOT, "paper_2503_14985_b200")
+    for dirpath, _, files in os.walk(pkg):
+        for f in files:
+            if f.endswith((".py", ".cu", ".cuh", ".h")):
+                text = open(os.path.join(dirpath, f)).read()
+                assert "import oracle" not in text and "from oracle" not in text and "oracle/" not in text, f
