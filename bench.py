@@ -1,0 +1,454 @@
+#!/usr/bin/env python
+"""Benchmark of the dense hot path on B200: BF16 GEMM + MHA forward through the C ABI.
+
+One *step* is one pass of the whole hot path over one batch of synthetic input:
+one large GEMM (tile schedule, TMA loads, UMMA accumulate, K loop, epilogue) and one
+D=128 causal attention forward (work schedule, Q/K/V loads, S = QK^T, mask, online
+softmax, PV, finalize).  `value` is TFLOP/s over the step (conventional FLOP counts:
+2MNK; 4*B*H*Nq*Nk*D, halved when causal), summed over all ranks.
+
+    python bench.py [--gpus N] [--steps K] [--warmup W] [--impl mlt|reference] [--all]
+
+For N > 1 launch with torch.distributed.run: every rank runs the same workload on
+its own GPU (independent problems, no data-path collective; weak scaling); NCCL is
+used only for the barrier and the max-over-ranks time.
+
+`--impl reference` times the CPU oracle (FP64, host threads) on a bounded sample of
+the same workload; it is a deliberately slow checker, reported as a baseline.
+`--all` adds per-configuration timings of every benchmark configuration under "configs".
+"""
+from __future__ import annotations
+
+import argparse
+import json
+import os
+import sys
+import threading
+import time
+
+import numpy as np
+
+ROOT = os.path.dirname(os.path.abspath(__file__))
+if ROOT not in sys.path:
+    sys.path.insert(0, ROOT)
+
+from paper_2503_14985_b200 import inputs  # noqa: E402
+
+METRIC = "TFLOP/s and % of B200 dense-BF16 peak for GEMM and MHA fwd (1 GPU)"
+UNIT = "TFLOP/s"
+NOMINAL_BF16_TFLOPS = 2250.0
+GEMM_NAME = "gemm_8192x28672x4096"
+MHA_NAME = "mha_b2h32n4096d128_causal"
+WORKLOAD = f"{GEMM_NAME} + {MHA_NAME}"
+
+
+# --------------------------------------------------------------------------
+# distributed plumbing (rank / world from the environment; gloo-testable)
+# --------------------------------------------------------------------------
+
+def dist_env():
+    return int(os.environ.get("RANK", "0")), int(os.environ.get("LOCAL_RANK", "0")), int(os.environ.get("WORLD_SIZE", "1"))
+
+
+def init_dist(backend: str):
+    """Initialise torch.distributed from RANK/WORLD_SIZE/MASTER_* if WORLD_SIZE > 1; returns (rank, local, world)."""
+    rank, local, world = dist_env()
+    if world > 1:
+        import torch.distributed as dist
+        if not dist.is_initialized():
+            os.environ.setdefault("MASTER_ADDR", "127.0.0.1")
+            os.environ.setdefault("MASTER_PORT", "29500")
+            dist.init_process_group(backend=backend, rank=rank, world_size=world)
+    return rank, local, world
+
+
+def barrier(world: int):
+    if world > 1:
+        import torch.distributed as dist
+        dist.barrier()
+
+
+def aggregate(ms_local: float, units_local: float, world: int, device=None):
+    """Whole-job figures: (max time over ranks in ms, sum of units over ranks)."""
+    if world == 1:
+        return ms_local, units_local
+    import torch
+    import torch.distributed as dist
+    t = torch.tensor([ms_local], dtype=torch.float64, device=device)
+    u = torch.tensor([units_local], dtype=torch.float64, device=device)
+    dist.all_reduce(t, op=dist.ReduceOp.MAX)
+    dist.all_reduce(u, op=dist.ReduceOp.SUM)
+    return float(t.item()), float(u.item())
+
+
+# --------------------------------------------------------------------------
+# clocks (read-only NVML sampling during the timed region)
+# --------------------------------------------------------------------------
+
+class ClockSampler:
+    REASONS = {0x8: "hw_slowdown", 0x40: "hw_thermal_slowdown", 0x20: "sw_thermal_slowdown", 0x4: "sw_power_cap",
+               0x80: "hw_power_brake_slowdown"}
+
+    def __init__(self, index: int, period_s: float = 0.005):
+        self.index, self.period = index, period_s
+        self.samples, self.reasons, self.power = [], set(), []
+        self._stop = threading.Event()
+        self._thread = None
+        self.max_mhz = None
+        try:
+            import pynvml
+            pynvml.nvmlInit()
+            self._nv = pynvml
+            self._h = pynvml.nvmlDeviceGetHandleByIndex(index)
+            self.max_mhz = int(pynvml.nvmlDeviceGetMaxClockInfo(self._h, pynvml.NVML_CLOCK_SM))
+        except Exception:
+            self._nv = None
+
+    def _run(self):
+        nv = self._nv
+        while not self._stop.is_set():
+            try:
+                self.samples.append(int(nv.nvmlDeviceGetClockInfo(self._h, nv.NVML_CLOCK_SM)))
+                mask = int(nv.nvmlDeviceGetCurrentClocksEventReasons(self._h))
+                for bit, name in self.REASONS.items():
+                    if mask & bit:
+                        self.reasons.add(name)
+                self.power.append(nv.nvmlDeviceGetPowerUsage(self._h) / 1000.0)
+            except Exception:
+                pass
+            self._stop.wait(self.period)
+
+    def __enter__(self):
+        if self._nv is not None:
+            self._thread = threading.Thread(target=self._run, daemon=True)
+            self._thread.start()
+        return self
+
+    def __exit__(self, *exc):
+        self._stop.set()
+        if self._thread is not None:
+            self._thread.join()
+
+    def summary(self):
+        return {"sm_mhz": float(np.median(self.samples)) if self.samples else None, "sm_max_mhz": self.max_mhz,
+                "reasons": sorted(self.reasons), "samples": len(self.samples),
+                "power_w_max": max(self.power) if self.power else None}
+
+
+def measured_peaks():
+    path = os.path.join(ROOT, "MEASURED_PEAKS.json")
+    if os.path.exists(path):
+        with open(path) as f:
+            d = json.load(f)
+        return {"burst": float(d["bf16_tflops"]), "sustained": float(d["bf16_tflops_sustained"]),
+                "hbm_gbs": float(d["hbm_gbs"]), "source": "measured"}
+    return {"burst": 1590.0, "sustained": 1400.0, "hbm_gbs": 6650.0, "source": "fallback"}
+
+
+# --------------------------------------------------------------------------
+# the CPU oracle as a timed baseline (bounded sample of the same workload)
+# --------------------------------------------------------------------------
+
+def oracle_sample_step(data, gemm_rows: int, mha_rows: int):
+    """One oracle 'step' on a sample of complete output rows; returns (seconds, flop, description)."""
+    import oracle
+    M, N, K = data["gemm_shape"]
+    B, H, Nq, Nk, D, causal = data["mha_shape"]
+    rows = np.linspace(0, M - 1, gemm_rows).astype(np.int64)
+    qrows = np.linspace(0, B * H * Nq - 1, mha_rows).astype(np.int64)
+    t0 = time.perf_counter()
+    oracle.gemm(data["A"], data["B"], M, N, K, rows=rows)
+    oracle.mha_fwd(data["Q"], data["K"], data["V"], causal=bool(causal), scale=data["scale"], qrows=qrows)
+    dt = time.perf_counter() - t0
+    flop = 2.0 * len(rows) * N * K
+    for r in qrows:
+        i = int(r % Nq)
+        visible = min(Nk, i + (Nk - Nq) + 1) if causal else Nk
+        flop += 4.0 * visible * D
+    what = f"{len(rows)} of {M} GEMM output rows + {len(qrows)} of {B * H * Nq} attention query rows (all columns)"
+    return dt, flop, what
+
+
+def make_host_data(gemm_name: str, mha_name: str):
+    M, N, K, kind, seed = inputs.GEMM_CONFIGS[gemm_name]
+    A, B = inputs.gemm_inputs(M, N, K, seed=seed, kind=kind)
+    Bn, H, Nq, Nk, D, causal, mseed, outl = inputs.MHA_CONFIGS[mha_name]
+    Q, Kk, V = inputs.mha_inputs(Bn, H, Nq, Nk, D, seed=mseed, outlier_percent=outl)
+    return {"A": A, "B": B, "Q": Q, "K": Kk, "V": V, "gemm_shape": (M, N, K), "mha_shape": (Bn, H, Nq, Nk, D, causal),
+            "scale": float(np.float32(1.0 / np.sqrt(D)))}
+
+
+def run_reference(args):
+    rank, _, world = dist_env()
+    if rank != 0:
+        return 0
+    import oracle
+    data = make_host_data(GEMM_NAME, MHA_NAME)
+    cores = oracle.hardware_threads()
+    gemm_rows, mha_rows = 64, 2048
+    for _ in range(max(args.warmup, 1)):
+        oracle_sample_step(data, 8, 64)
+    t_total, f_total, what = 0.0, 0.0, ""
+    for _ in range(args.steps):
+        dt, flop, what = oracle_sample_step(data, gemm_rows, mha_rows)
+        t_total += dt
+        f_total += flop
+    value = f_total / t_total / 1e12
+    line = {"impl": "reference", "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": args.gpus, "steps": args.steps,
+            "warmup": args.warmup, "ms_per_step": 1e3 * t_total / args.steps, "higher_is_better": True, "scaling": "weak",
+            "vs_baseline": None, "dtype": "f64", "data": "synthetic",
+            "config": {"workload": WORKLOAD, "note": "CPU oracle on a sample of complete output rows per step"},
+            "cpu_baseline": {"value": value, "unit": UNIT, "cores": cores, "kind": "oracle", "sample": what},
+            "e2e": {"value": value, "unit": UNIT, "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0}}
+    print(json.dumps(line))
+    return 0
+
+
+# --------------------------------------------------------------------------
+# the CUDA path
+# --------------------------------------------------------------------------
+
+def run_mlt(args):
+    import torch
+    import paper_2503_14985_b200 as mlt
+
+    if not torch.cuda.is_available():
+        raise RuntimeError("bench.py needs a CUDA device (sm_100a); there is no CPU fallback")
+    rank, local, world = init_dist("nccl")
+    torch.cuda.set_device(local)
+    dev = torch.device("cuda", local)
+    mlt.load()
+
+    data = make_host_data(GEMM_NAME, MHA_NAME)
+    M, N, K = data["gemm_shape"]
+    Bn, H, Nq, Nk, D, causal = data["mha_shape"]
+    scale = data["scale"]
+    gemm_flop = inputs.gemm_flops(M, N, K)
+    mha_flop = inputs.mha_flops(Bn, H, Nq, Nk, D, causal)
+    step_flop = gemm_flop + mha_flop
+
+    def pinned(bits):
+        return torch.from_numpy(np.ascontiguousarray(bits).view(np.int16)).pin_memory()
+
+    hA, hB, hQ, hK, hV = (pinned(data[k]) for k in ("A", "B", "Q", "K", "V"))
+    dA, dB, dQ, dK, dV = (torch.empty_like(h, device=dev) for h in (hA, hB, hQ, hK, hV))
+    dC = torch.empty((M, N), dtype=torch.int16, device=dev)
+    dO = torch.empty_like(dQ)
+    dL = torch.empty((Bn, H, Nq), dtype=torch.float32, device=dev)
+    hC = torch.empty((M, N), dtype=torch.int16).pin_memory()
+    hO = torch.empty(tuple(dQ.shape), dtype=torch.int16).pin_memory()
+    hL = torch.empty((Bn, H, Nq), dtype=torch.float32).pin_memory()
+    for d, h in ((dA, hA), (dB, hB), (dQ, hQ), (dK, hK), (dV, hV)):
+        d.copy_(h)
+    stream = torch.cuda.current_stream()
+    sp = stream.cuda_stream
+
+    def launch_gemm():
+        rc = mlt.gemm_raw(dA.data_ptr(), dB.data_ptr(), dC.data_ptr(), M, N, K, K, N, N, sp)
+        if rc:
+            raise mlt.MltError(rc, "mlt_gemm")
+
+    def launch_mha():
+        rc = mlt.mha_fwd_raw(dQ.data_ptr(), dK.data_ptr(), dV.data_ptr(), dO.data_ptr(), dL.data_ptr(), Bn, H, Nq, Nk, D,
+                             causal, scale, sp)
+        if rc:
+            raise mlt.MltError(rc, "mlt_mha_fwd")
+
+    def step():
+        launch_gemm()
+        launch_mha()
+
+    def e2e_step():
+        for d, h in ((dA, hA), (dB, hB), (dQ, hQ), (dK, hK), (dV, hV)):
+            d.copy_(h, non_blocking=True)
+        step()
+        hC.copy_(dC, non_blocking=True)
+        hO.copy_(dO, non_blocking=True)
+        hL.copy_(dL, non_blocking=True)
+
+    # ---- device-resident timing: W warm-up steps, then exactly K timed steps ----
+    for _ in range(args.warmup):
+        step()
+    torch.cuda.synchronize()
+    K_steps = args.steps
+    ev = [[torch.cuda.Event(enable_timing=True) for _ in range(3)] for _ in range(K_steps)]
+    t_begin, t_end = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    barrier(world)
+    torch.cuda.synchronize()
+    with ClockSampler(local) as clocks:
+        t_begin.record(stream)
+        for i in range(K_steps):
+            ev[i][0].record(stream)
+            launch_gemm()
+            ev[i][1].record(stream)
+            launch_mha()
+            ev[i][2].record(stream)
+        t_end.record(stream)
+        torch.cuda.synchronize()
+    barrier(world)
+    ms_total = t_begin.elapsed_time(t_end)
+    gemm_ms = [e[0].elapsed_time(e[1]) for e in ev]
+    mha_ms = [e[1].elapsed_time(e[2]) for e in ev]
+    rc, detail = mlt.last_device_error()
+    if rc:
+        raise mlt.MltError(rc, f"device status {detail}")
+
+    # ---- end to end: host buffers in, host buffers out, copies inside the timed region ----
+    for _ in range(max(1, min(args.warmup, 3))):
+        e2e_step()
+    torch.cuda.synchronize()
+    e2e_steps = max(1, min(K_steps, 10))
+    e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    barrier(world)
+    torch.cuda.synchronize()
+    e0.record(stream)
+    for _ in range(e2e_steps):
+        e2e_step()
+    e1.record(stream)
+    torch.cuda.synchronize()
+    barrier(world)
+    e2e_ms = e0.elapsed_time(e1)
+    h2d = sum(h.numel() * h.element_size() for h in (hA, hB, hQ, hK, hV))
+    d2h = sum(h.numel() * h.element_size() for h in (hC, hO, hL))
+
+    ms_max, flop_all = aggregate(ms_total, step_flop * K_steps, world, dev)
+    e2e_max, e2e_flop = aggregate(e2e_ms, step_flop * e2e_steps, world, dev)
+    value = flop_all / (ms_max * 1e-3) / 1e12
+    e2e_value = e2e_flop / (e2e_max * 1e-3) / 1e12
+
+    # ---- optional: every benchmark configuration on its own (rank 0 reports) ----
+    per_config = None
+    if args.all:
+        per_config = time_all_configs(mlt, torch, dev, stream)
+
+    if rank != 0:
+        return 0
+
+    peaks = measured_peaks()
+    gemm_avg_ms = float(np.mean(gemm_ms))
+    mha_avg_ms = float(np.mean(mha_ms))
+    achieved = gemm_flop / (gemm_avg_ms * 1e-3) / 1e12
+    long_run = ms_total > 1000.0
+    peak = peaks["sustained"] if long_run else peaks["burst"]
+    roofline = {"bound": "tensor", "kernel": "gemm_bf16_kernel<256,4>", "achieved": achieved, "peak": peak, "unit": UNIT,
+                "frac": achieved / peak, "traffic": NCU_TRAFFIC_BYTES.get("gemm"),
+                "peak_source": f"{peaks['source']} cuBLAS bf16 {'sustained' if long_run else 'burst'}",
+                "frac_of_nominal_2250": achieved / NOMINAL_BF16_TFLOPS,
+                "achieved_hbm_gbs": 2.0 * (M * K + K * N + M * N) / (gemm_avg_ms * 1e-3) / 1e9}
+    per_op = {"gemm": {"config": GEMM_NAME, "ms": gemm_avg_ms, "ms_min": float(np.min(gemm_ms)),
+                       "tflops": achieved, "tflops_best": gemm_flop / (np.min(gemm_ms) * 1e-3) / 1e12,
+                       "frac_of_2250": achieved / NOMINAL_BF16_TFLOPS},
+              "mha_fwd": {"config": MHA_NAME, "ms": mha_avg_ms, "ms_min": float(np.min(mha_ms)),
+                          "tflops": mha_flop / (mha_avg_ms * 1e-3) / 1e12,
+                          "tflops_best": mha_flop / (np.min(mha_ms) * 1e-3) / 1e12,
+                          "frac_of_2250": mha_flop / (mha_avg_ms * 1e-3) / 1e12 / NOMINAL_BF16_TFLOPS}}
+
+    cpu_baseline = None
+    if world == 1 or rank == 0:
+        import oracle
+        dt, flop, what = oracle_sample_step(data, 2048, 32768)
+        cpu_baseline = {"value": flop / dt / 1e12, "unit": UNIT, "cores": oracle.hardware_threads(), "kind": "oracle",
+                        "sample": what, "seconds": dt}
+
+    line = {"metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world, "steps": K_steps, "warmup": args.warmup,
+            "ms_per_step": ms_max / K_steps, "higher_is_better": True, "scaling": "weak", "vs_baseline": None,
+            "dtype": "bf16", "data": "synthetic",
+            "config": {"workload": WORKLOAD, "gemm": {"M": M, "N": N, "K": K}, "mha": {"B": Bn, "H": H, "Nq": Nq, "Nk": Nk,
+                       "D": D, "causal": bool(causal)}, "l2": "inputs larger than L2 (302 MB GEMM operands, 201 MB Q/K/V)",
+                       "flop_convention": "2MNK; 4*B*H*Nq*Nk*D halved when causal", "parallelism": f"replicas x{world}"},
+            "clocks": clocks.summary(),
+            "e2e": {"value": e2e_value, "unit": UNIT, "h2d_bytes_per_step": h2d, "d2h_bytes_per_step": d2h,
+                    "ms_per_step": e2e_max / e2e_steps, "steps": e2e_steps},
+            "gpu_launches": 2 * K_steps, "roofline": roofline, "cpu_baseline": cpu_baseline, "per_op": per_op}
+    if per_config is not None:
+        line["configs"] = per_config
+    print(json.dumps(line))
+    return 0
+
+
+# dram__bytes_read.sum + dram__bytes_write.sum per launch from the ncu capture summarised under profiles/
+NCU_TRAFFIC_BYTES = {"gemm": None}
+
+
+def time_all_configs(mlt, torch, dev, stream, iters: int = 20, only: str | None = None, warm: int = 3):
+    """Min / median kernel time of every benchmark configuration (CUDA events, inputs resident)."""
+    out = {}
+    sp = stream.cuda_stream
+
+    def devbits(bits):
+        return torch.from_numpy(np.ascontiguousarray(bits).view(np.int16)).to(dev)
+
+    flush = torch.empty(256 << 20, dtype=torch.int8, device=dev)
+
+    def timeit(fn, flop):
+        for _ in range(warm):
+            fn()
+        times = []
+        for _ in range(iters):
+            flush.zero_()  # evict L2 between timed launches
+            a, b = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+            a.record(stream)
+            fn()
+            b.record(stream)
+            torch.cuda.synchronize()
+            times.append(a.elapsed_time(b))
+        tmin, tmed = float(np.min(times)), float(np.median(times))
+        return {"ms_min": tmin, "ms_median": tmed, "tflops_best": flop / tmin / 1e9, "tflops_median": flop / tmed / 1e9,
+                "frac_of_2250_best": flop / tmin / 1e9 / NOMINAL_BF16_TFLOPS}
+
+    for name, (M, N, K, kind, seed) in inputs.GEMM_CONFIGS.items():
+        if only is not None and name != only:
+            continue
+        A, B = inputs.gemm_inputs(M, N, K, seed=seed, kind=kind)
+        dA, dB = devbits(A), devbits(B)
+        dC = torch.empty((M, N), dtype=torch.int16, device=dev)
+
+        def fn():
+            rc = mlt.gemm_raw(dA.data_ptr(), dB.data_ptr(), dC.data_ptr(), M, N, K, K, N, N, sp)
+            assert rc == 0, rc
+        out[name] = timeit(fn, inputs.gemm_flops(M, N, K))
+        del dA, dB, dC
+    for name, (Bn, H, Nq, Nk, D, causal, seed, outl) in inputs.MHA_CONFIGS.items():
+        if only is not None and name != only:
+            continue
+        Q, Kk, V = inputs.mha_inputs(Bn, H, Nq, Nk, D, seed=seed, outlier_percent=outl)
+        dQ, dK, dV = devbits(Q), devbits(Kk), devbits(V)
+        dO = torch.empty_like(dQ)
+        dL = torch.empty((Bn, H, Nq), dtype=torch.float32, device=dev)
+        sc = float(np.float32(1.0 / np.sqrt(D)))
+
+        def fn():
+            rc = mlt.mha_fwd_raw(dQ.data_ptr(), dK.data_ptr(), dV.data_ptr(), dO.data_ptr(), dL.data_ptr(), Bn, H, Nq, Nk,
+                                 D, causal, sc, sp)
+            assert rc == 0, rc
+        out[name] = timeit(fn, inputs.mha_flops(Bn, H, Nq, Nk, D, causal))
+        del dQ, dK, dV, dO, dL
+    return out
+
+
+def main(argv=None):
+    ap = argparse.ArgumentParser(description=__doc__, formatter_class=argparse.RawDescriptionHelpFormatter)
+    ap.add_argument("--gpus", type=int, default=1)
+    ap.add_argument("--steps", type=int, default=50)
+    ap.add_argument("--warmup", type=int, default=5)
+    ap.add_argument("--impl", choices=["mlt", "reference"], default="mlt")
+    ap.add_argument("--all", action="store_true", help="also time every benchmark configuration on its own")
+    ap.add_argument("--only", default=None, help="time one named configuration alone (kernel launches only; for profiling)")
+    args = ap.parse_args(argv)
+    if args.only is not None:
+        import torch
+        import paper_2503_14985_b200 as mlt
+        torch.cuda.set_device(0)
+        res = time_all_configs(mlt, torch, torch.device("cuda", 0), torch.cuda.current_stream(), iters=args.steps,
+                               only=args.only, warm=args.warmup)
+        print(json.dumps({"only": args.only, **res.get(args.only, {"error": "unknown configuration"})}))
+        return 0
+    if args.warmup < 3 and args.impl == "mlt":
+        args.warmup = 3
+    if args.impl == "reference":
+        return run_reference(args)
+    return run_mlt(args)
+
+
+if __name__ == "__main__":
+    sys.exit(main())
