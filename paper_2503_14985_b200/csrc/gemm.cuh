@@ -184,8 +184,9 @@ gemm_bf16_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_consta
                         if (col + 8 <= p.N) {
                             *reinterpret_cast<uint4*>(crow + col) = out;
                         } else if (col < p.N) {
-                            const __nv_bfloat16* e = reinterpret_cast<const __nv_bfloat16*>(&out);
-                            for (int j = 0; col + j < p.N; ++j) crow[col + j] = e[j];
+                            const uint32_t w[4] = {out.x, out.y, out.z, out.w};
+                            for (int j = 0; col + j < p.N; ++j)
+                                crow[col + j] = __ushort_as_bfloat16(static_cast<unsigned short>(w[j >> 1] >> ((j & 1) * 16)));
                         }
                     }
                 }
@@ -204,6 +205,195 @@ gemm_bf16_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_consta
         __syncwarp();
         tc_fence_after();
         tmem_dealloc(tmem_base, kTmemCols);
+    }
+}
+
+// ---------------------------------------------------------------------------
+// CTA-pair variant for large problems: a cluster of two CTAs owns a 256 x 256 tile.
+// Each CTA loads its own 128 rows of A and its own 128 columns of B (no multicast);
+// the leader CTA (cluster rank 0) issues cta_group::2 UMMAs that read both CTAs'
+// shared memory and write both CTAs' tensor memory (rows 0-127 / 128-255 of the tile).
+// Compared with two independent 128 x 256 tiles this cuts the L2 -> SM operand traffic
+// per FLOP by a third and the shared-memory reads of B by half.
+//   full[s]       in the leader: both CTAs' TMA loads count bytes on it
+//   empty[s]      in each CTA: the leader's commit arrives on both
+//   acc_full[a]   in each CTA: the leader's commit arrives on both
+//   acc_empty[a]  in the leader: the epilogue warps of both CTAs arrive on it (8 arrivals)
+// ---------------------------------------------------------------------------
+constexpr int kPairBM = 256;
+constexpr int kPairBN = 256;
+
+template <int kStages>
+struct GemmPairSmem {
+    static constexpr int kABytes = 128 * kGemmBK * 2;  // this CTA's 128 rows of A
+    static constexpr int kBBytes = kGemmBK * 128 * 2;  // this CTA's 128 columns of B: 2 boxes of 64 x 64
+    static constexpr int kStageBytes = kABytes + kBBytes;
+    static constexpr int kTotal = kStages * kStageBytes + 256 + 1024;
+};
+
+template <int kStages>
+__global__ void __cluster_dims__(2, 1, 1) __launch_bounds__(kGemmThreads, 1)
+gemm_bf16_pair_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_constant__ CUtensorMap tmap_b,
+                      const GemmParams p) {
+    using L = GemmPairSmem<kStages>;
+    extern __shared__ uint8_t smem_raw[];
+    uint8_t* smem = reinterpret_cast<uint8_t*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~uintptr_t(1023));
+    uint64_t* bars = reinterpret_cast<uint64_t*>(smem + kStages * L::kStageBytes);
+    uint64_t* full = bars;
+    uint64_t* empty = bars + kStages;
+    uint64_t* acc_full = bars + 2 * kStages;
+    uint64_t* acc_empty = acc_full + 2;
+    uint32_t* tmem_base_slot = reinterpret_cast<uint32_t*>(acc_empty + 2);
+    volatile uint32_t* abort_flag = tmem_base_slot + 1;
+
+    const int warp = threadIdx.x >> 5;
+    const int lane = threadIdx.x & 31;
+    const uint32_t rank = cluster_ctarank();
+    const bool leader = rank == 0;
+    const int cluster_id = blockIdx.x >> 1;
+    const int num_clusters = gridDim.x >> 1;
+    const int num_tiles = p.tiles_m * p.tiles_n;
+    const int num_kb = (p.K + kGemmBK - 1) / kGemmBK;
+    constexpr uint32_t kTmemCols = 512;  // two 256-column accumulators
+
+    if (threadIdx.x == 0) {
+        for (int s = 0; s < kStages; ++s) {
+            mbar_init(&full[s], 1);
+            mbar_init(&empty[s], 1);
+        }
+        for (int a = 0; a < 2; ++a) {
+            mbar_init(&acc_full[a], 1);
+            mbar_init(&acc_empty[a], 8);  // 4 epilogue warps in each of the two CTAs
+        }
+        *abort_flag = 0;
+        fence_mbar_init();
+    }
+    if (warp == 0 && lane == 0) {
+        prefetch_tensormap(&tmap_a);
+        prefetch_tensormap(&tmap_b);
+    }
+    if (warp == 1) {
+        tmem_alloc_pair(tmem_base_slot, kTmemCols);
+        tmem_relinquish_pair();
+    }
+    tc_fence_before();
+    cluster_sync_all();  // barrier inits and allocations of both CTAs are visible to both
+    tc_fence_after();
+    const uint32_t tmem_base = *tmem_base_slot;
+
+    if (warp == 0) {
+        // ----------------------------- producer (both CTAs) -----------------------------
+        if (lane == 0) {
+            int stage = 0;
+            uint32_t phase = 0;
+            bool ok = true;
+            for (int tile = cluster_id; tile < num_tiles && ok; tile += num_clusters) {
+                int tm, tn;
+                gemm_tile_coords(p, tile, tm, tn);
+                const int m0 = tm * kPairBM + static_cast<int>(rank) * 128;
+                const int n0 = tn * kPairBN + static_cast<int>(rank) * 128;
+                for (int kb = 0; kb < num_kb; ++kb) {
+                    ok = mbar_wait(&empty[stage], phase ^ 1, abort_flag, 0x100 + stage);
+                    if (!ok) break;
+                    uint8_t* sa = smem + stage * L::kStageBytes;
+                    uint8_t* sb = sa + L::kABytes;
+                    if (leader) mbar_arrive_expect_tx(&full[stage], 2 * L::kStageBytes);
+                    const uint32_t bar = map_to_cta(smem_u32(&full[stage]), 0);
+                    tma_load_2d_pair(sa, &tmap_a, bar, kb * kGemmBK, m0);
+                    tma_load_2d_pair(sb, &tmap_b, bar, n0, kb * kGemmBK);
+                    tma_load_2d_pair(sb + kGemmBK * 128, &tmap_b, bar, n0 + 64, kb * kGemmBK);
+                    if (++stage == kStages) { stage = 0; phase ^= 1; }
+                }
+            }
+        }
+    } else if (warp == 1) {
+        // ----------------------------- UMMA issuer (leader CTA only) -----------------------------
+        if (leader && lane == 0) {
+            constexpr uint32_t idesc = make_idesc_bf16(kPairBM, kPairBN, /*a_mn_major=*/false, /*b_mn_major=*/true);
+            int stage = 0;
+            uint32_t phase = 0;
+            int acc = 0;
+            uint32_t acc_phase = 0;
+            bool ok = true;
+            for (int tile = cluster_id; tile < num_tiles && ok; tile += num_clusters) {
+                ok = mbar_wait(&acc_empty[acc], acc_phase ^ 1, abort_flag, 0x300 + acc);
+                if (!ok) break;
+                tc_fence_after();
+                const uint32_t d_tmem = tmem_base + acc * kPairBN;
+                for (int kb = 0; kb < num_kb; ++kb) {
+                    ok = mbar_wait(&full[stage], phase, abort_flag, 0x200 + stage);
+                    if (!ok) break;
+                    tc_fence_after();
+                    const uint32_t sa = smem_u32(smem + stage * L::kStageBytes);
+                    const uint32_t sb = sa + L::kABytes;
+#pragma unroll
+                    for (int k = 0; k < kGemmBK / 16; ++k) {
+                        const uint64_t da = make_sdesc_sw128(sa + k * 32, 16, 1024);
+                        const uint64_t db = make_sdesc_sw128(sb + k * 2048, kGemmBK * 128, 1024);
+                        umma_ss_pair(d_tmem, da, db, idesc, (kb | k) != 0);
+                    }
+                    umma_commit_pair(&empty[stage], 3);
+                    if (++stage == kStages) { stage = 0; phase ^= 1; }
+                }
+                if (ok) umma_commit_pair(&acc_full[acc], 3);
+                if (++acc == 2) { acc = 0; acc_phase ^= 1; }
+            }
+        }
+    } else {
+        // ----------------------------- epilogue (both CTAs, own 128 rows) -----------------------------
+        const int quarter = warp & 3;
+        int acc = 0;
+        uint32_t acc_phase = 0;
+        bool ok = true;
+        for (int tile = cluster_id; tile < num_tiles && ok; tile += num_clusters) {
+            int tm, tn;
+            gemm_tile_coords(p, tile, tm, tn);
+            const int row = tm * kPairBM + static_cast<int>(rank) * 128 + quarter * 32 + lane;
+            const int n0 = tn * kPairBN;
+            ok = __all_sync(0xffffffffu, mbar_wait(&acc_full[acc], acc_phase, abort_flag, 0x400 + acc));
+            if (!ok) break;
+            tc_fence_after();
+            const uint32_t t_row = tmem_base + (static_cast<uint32_t>(quarter * 32) << 16) + acc * kPairBN;
+            __nv_bfloat16* crow = p.C + static_cast<int64_t>(row) * p.ldc;
+#pragma unroll 1
+            for (int c = 0; c < kPairBN / 32; ++c) {
+                uint32_t v[32];
+                tmem_ld_32x32b_x32(t_row + c * 32, v);
+                tmem_wait_ld();
+                const int col0 = n0 + c * 32;
+                if (row < p.M) {
+#pragma unroll
+                    for (int q = 0; q < 4; ++q) {
+                        const int col = col0 + q * 8;
+                        uint4 out;
+                        out.x = pack_bf16x2(__uint_as_float(v[q * 8 + 0]), __uint_as_float(v[q * 8 + 1]));
+                        out.y = pack_bf16x2(__uint_as_float(v[q * 8 + 2]), __uint_as_float(v[q * 8 + 3]));
+                        out.z = pack_bf16x2(__uint_as_float(v[q * 8 + 4]), __uint_as_float(v[q * 8 + 5]));
+                        out.w = pack_bf16x2(__uint_as_float(v[q * 8 + 6]), __uint_as_float(v[q * 8 + 7]));
+                        if (col + 8 <= p.N) {
+                            *reinterpret_cast<uint4*>(crow + col) = out;
+                        } else if (col < p.N) {
+                            const uint32_t w[4] = {out.x, out.y, out.z, out.w};
+                            for (int j = 0; col + j < p.N; ++j)
+                                crow[col + j] = __ushort_as_bfloat16(static_cast<unsigned short>(w[j >> 1] >> ((j & 1) * 16)));
+                        }
+                    }
+                }
+            }
+            tc_fence_before();
+            __syncwarp();
+            if (lane == 0) mbar_arrive_cluster(map_to_cta(smem_u32(&acc_empty[acc]), 0));
+            if (++acc == 2) { acc = 0; acc_phase ^= 1; }
+        }
+    }
+
+    // common exit: no CTA of the pair leaves while its peer may still touch its memory
+    tc_fence_before();
+    cluster_sync_all();
+    if (warp == 1) {
+        __syncwarp();
+        tc_fence_after();
+        tmem_dealloc_pair(tmem_base, kTmemCols);
     }
 }
 

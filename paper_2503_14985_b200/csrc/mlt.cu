@@ -64,7 +64,8 @@ int get_device(DeviceInfo* out) {
             return MLT_ERR_CUDA;
         if (d.cc_major != 10) return MLT_ERR_ARCH;
         if (set_smem(gemm_bf16_kernel<256, 4>, GemmSmem<256, 4>::kTotal) != MLT_OK ||
-            set_smem(gemm_bf16_kernel<128, 6>, GemmSmem<128, 6>::kTotal) != MLT_OK)
+            set_smem(gemm_bf16_kernel<128, 6>, GemmSmem<128, 6>::kTotal) != MLT_OK ||
+            set_smem(gemm_bf16_pair_kernel<6>, GemmPairSmem<6>::kTotal) != MLT_OK)
             return MLT_ERR_CUDA;
         if (mha_configure() != MLT_OK) return MLT_ERR_CUDA;
         d.configured = true;
@@ -97,6 +98,15 @@ int encode_bf16(CUtensorMap* map, const void* base, int rank, const uint64_t* di
                      gdim, gstride, gbox, estr, CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B,
                      CU_TENSOR_MAP_L2_PROMOTION_L2_256B, CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
     return r == CUDA_SUCCESS ? MLT_OK : MLT_ERR_CUDA;
+}
+
+// Debug only: MLT_FORCE_VARIANT=0|1|2 pins the GEMM tile variant (pair 256x256, 128x256, 128x128).
+int forced_variant() {
+    static const int v = [] {
+        const char* e = std::getenv("MLT_FORCE_VARIANT");
+        return e ? std::atoi(e) : -1;
+    }();
+    return v;
 }
 
 inline bool aligned16(const void* p) { return (reinterpret_cast<uintptr_t>(p) & 15u) == 0; }
@@ -157,10 +167,21 @@ int mlt_gemm(const void* A, const void* B, void* C, int64_t M, int64_t N, int64_
         return cudaGetLastError() == cudaSuccess ? MLT_OK : MLT_ERR_CUDA;
     }
 
-    // 128 x 256 tiles unless that leaves most SMs idle; then 128 x 128.
-    const int64_t tiles_m = (M + kGemmBM - 1) / kGemmBM;
-    const bool wide = tiles_m * ((N + 255) / 256) >= dev.sm_count;
-    const int bn = wide ? 256 : 128;
+    // Tile shape by problem size: CTA pairs on 256 x 256 tiles when there is at least one tile per pair of SMs,
+    // else 128 x 256 tiles, else (most SMs would idle) 128 x 128 tiles.
+    const int64_t pair_tiles = ((M + kPairBM - 1) / kPairBM) * ((N + kPairBN - 1) / kPairBN);
+    const int64_t tiles_m128 = (M + kGemmBM - 1) / kGemmBM;
+    int variant;  // 0: pair 256x256, 1: 128x256, 2: 128x128
+    if (pair_tiles >= dev.sm_count / 2 && forced_variant() != 1 && forced_variant() != 2)
+        variant = 0;
+    else if (tiles_m128 * ((N + 255) / 256) >= dev.sm_count && forced_variant() != 2)
+        variant = 1;
+    else
+        variant = 2;
+    if (forced_variant() >= 0 && forced_variant() <= 2) variant = forced_variant();
+    const int bm = variant == 0 ? kPairBM : kGemmBM;
+    const int bn = variant == 2 ? 128 : 256;
+    const int64_t tiles_m = (M + bm - 1) / bm;
     const int64_t tiles_n = (N + bn - 1) / bn;
     if (tiles_m * tiles_n > INT32_MAX) return MLT_ERR_UNSUPPORTED;
 
@@ -168,7 +189,7 @@ int mlt_gemm(const void* A, const void* B, void* C, int64_t M, int64_t N, int64_
     {
         const uint64_t dims[2] = {static_cast<uint64_t>(K), static_cast<uint64_t>(M)};
         const uint64_t strides[1] = {static_cast<uint64_t>(lda) * 2};
-        const uint32_t box[2] = {kGemmBK, kGemmBM};
+        const uint32_t box[2] = {kGemmBK, 128};
         rc = encode_bf16(&ta, A, 2, dims, strides, box);
         if (rc != MLT_OK) return rc;
     }
@@ -188,12 +209,18 @@ int mlt_gemm(const void* A, const void* B, void* C, int64_t M, int64_t N, int64_
     p.K = static_cast<int>(K);
     p.tiles_m = static_cast<int>(tiles_m);
     p.tiles_n = static_cast<int>(tiles_n);
-    p.group_m = 16;
-    const int grid = static_cast<int>(std::min<int64_t>(tiles_m * tiles_n, dev.sm_count));
-    if (wide)
-        gemm_bf16_kernel<256, 4><<<grid, kGemmThreads, GemmSmem<256, 4>::kTotal, st>>>(ta, tb, p);
-    else
-        gemm_bf16_kernel<128, 6><<<grid, kGemmThreads, GemmSmem<128, 6>::kTotal, st>>>(ta, tb, p);
+    if (variant == 0) {
+        p.group_m = 8;
+        const int clusters = static_cast<int>(std::min<int64_t>(tiles_m * tiles_n, dev.sm_count / 2));
+        gemm_bf16_pair_kernel<6><<<2 * clusters, kGemmThreads, GemmPairSmem<6>::kTotal, st>>>(ta, tb, p);
+    } else {
+        p.group_m = 16;
+        const int grid = static_cast<int>(std::min<int64_t>(tiles_m * tiles_n, dev.sm_count));
+        if (variant == 1)
+            gemm_bf16_kernel<256, 4><<<grid, kGemmThreads, GemmSmem<256, 4>::kTotal, st>>>(ta, tb, p);
+        else
+            gemm_bf16_kernel<128, 6><<<grid, kGemmThreads, GemmSmem<128, 6>::kTotal, st>>>(ta, tb, p);
+    }
     return cudaGetLastError() == cudaSuccess ? MLT_OK : MLT_ERR_CUDA;
 }
 

@@ -39,8 +39,9 @@ def ld_for(width, extra):
     return (width + 7) // 8 * 8 + extra
 
 
+# the last three are large enough for the CTA-pair (256 x 256) kernel, with ragged edges in M, N and K
 SHAPES = [(128, 256, 64), (1, 8, 8), (8, 8, 16), (129, 257, 72), (300, 520, 1000), (512, 512, 512),
-          (2048, 1024, 8), (130, 2500, 200), (4100, 300, 136)]
+          (2048, 1024, 8), (130, 2500, 200), (4100, 300, 136), (2100, 2300, 520), (1281, 6152, 72), (19000, 264, 136)]
 
 
 @pytest.mark.parametrize("extra", [0, 8, 64])
@@ -53,7 +54,7 @@ def test_parity_small_and_ragged(M, N, K, extra):
     check_gemm(C, ref, f"{M}x{N}x{K}+{extra}")
 
 
-@pytest.mark.parametrize("M,N,K", [(256, 512, 256), (129, 257, 200), (384, 640, 1024)])
+@pytest.mark.parametrize("M,N,K", [(256, 512, 256), (129, 257, 200), (384, 640, 1024), (2176, 2312, 200), (4096, 4096, 256)])
 def test_bit_exact_on_small_integers(M, N, K):
     # entries in {-1,0,1}: every partial sum is an exact small integer; |c| <= 256 is BF16-representable
     A, B = inputs.gemm_inputs(M, N, K, seed=7, kind="ternary", lda=ld_for(K, 0), ldb=ld_for(N, 0))
@@ -133,7 +134,7 @@ def test_argument_errors_do_not_launch():
     x = torch.zeros(64, 64, dtype=torch.bfloat16, device="cuda")
     p = x.data_ptr()
     assert mlt.gemm_raw(p, p, p + 2, 8, 8, 8, 64, 64, 64) == 3          # C not 16-byte aligned
-    assert mlt.gemm_raw(p, p, p, 8, 8, 8, 257 - 1 + 1, 64, 64) == 3     # lda = 257: not a multiple of 8
+    assert mlt.gemm_raw(p, p, p, 8, 8, 8, 257, 64, 64) == 3     # lda = 257: not a multiple of 8
     assert mlt.gemm_raw(p, p, p, 8, 8, 16, 8, 64, 64) == 1              # lda < K
     assert mlt.gemm_raw(0, p, p, 8, 8, 8, 64, 64, 64) == 1              # NULL A
     assert mlt.gemm_raw(p, p, p, -1, 8, 8, 64, 64, 64) == 1
