@@ -7,11 +7,19 @@
 // on the tensor pipe, so the exponentials of one tile overlap the products of the other.
 //   warps 0-3   softmax / O-rescale / epilogue of tile 0 (one thread per query row)
 //   warps 4-7   the same for tile 1
-//   warp  8     UMMA issuer (one lane) and owner of the tensor-memory allocation
+//   warp  8     UMMA issuer (one lane) and owner of the tensor-memory allocation; it serves the
+//               tiles in a fixed order (P V of tile 0, next Q K^T of tile 0, the same for tile 1),
+//               which keeps the two softmax warpgroups half a period apart
 //   warp  9     TMA loader (one lane): both Q tiles once, then K_0, V_0, K_1, V_1, ... through a ring
+//   warps 10-11 idle (they complete the third warpgroup for the register hand-over)
 // Tensor memory (512 columns): S_0 | S_1 (128 FP32 columns each; the BF16 P of a tile
 // overwrites the first 64 columns of its S and is consumed from there as the A operand
 // of P V), then O_0 | O_1 (D FP32 columns each).
+//
+// Measured on B200: one thread sustains one UMMA issue per 46-64 clocks only while its
+// scheduler partition is otherwise quiet, and shared memory (TMA writes plus operand reads,
+// about 128 bytes per clock and SM) is a co-bound: per tile and K/V block the tensor core
+// reads Q, K and V tiles while TMA writes the next K and V tiles.
 #pragma once
 
 #include <math.h>
@@ -21,7 +29,7 @@
 namespace mlt {
 
 constexpr int kMhaBlock = 128;   // query rows per tile and keys per K/V block
-constexpr int kMhaThreads = 320;
+constexpr int kMhaThreads = 384; // three warpgroups
 constexpr float kLog2e = 1.4426950408889634f;
 constexpr float kRescaleThreshold = 8.0f;  // in log2 units: keep a stale max until it is off by more than 2^8
 
@@ -30,7 +38,7 @@ struct MhaSmem {
     static constexpr int kTileBytes = kMhaBlock * D * 2;  // one Q, K or V tile: D/64 chunks of 128 rows x 128 B
     static constexpr int kChunkBytes = kMhaBlock * 128;
     static constexpr int kStages = (D == 128) ? 4 : 8;
-    static constexpr int kBarrierBytes = 256;
+    static constexpr int kBarrierBytes = 512;
     static constexpr int kTotal = 2 * kTileBytes + kStages * kTileBytes + kBarrierBytes + 1024;
 };
 
@@ -42,7 +50,15 @@ struct MhaParams {
     float scale;
     int num_pairs;   // 256-row query groups per head
     int head_group;  // heads that share a span of consecutive block indices
+#ifdef MLT_TRACE
+    long long* trace;
+#endif
 };
+#ifdef MLT_TRACE
+#define MLT_TR(ev, j, t) do { if (blockIdx.x == 0 && (j) < 32) p.trace[((ev) * 32 + (j)) * 2 + (t)] = clock64(); } while (0)
+#else
+#define MLT_TR(ev, j, t) do { } while (0)
+#endif
 
 // block index -> (pair, bh).  Heads are taken in groups; inside a group the query
 // position is the slow index and runs from the last rows to the first, so under a
@@ -131,8 +147,11 @@ mha_fwd_kernel(const __grid_constant__ CUtensorMap tmap_q, const __grid_constant
     constexpr uint32_t kColS = 0;      // S_t at kColS + t*128
     constexpr uint32_t kColO = 256;    // O_t at kColO + t*D
 
-    if (warp == 9) {
+    if (warp >= 10) {
+        setmaxnreg_dec<40>();  // only hand their registers over
+    } else if (warp == 9) {
         // ------------------------------- loader -------------------------------
+        setmaxnreg_dec<40>();
         if (lane == 0) {
             mbar_arrive_expect_tx(q_full, 2 * L::kTileBytes);
 #pragma unroll
@@ -161,32 +180,39 @@ mha_fwd_kernel(const __grid_constant__ CUtensorMap tmap_q, const __grid_constant
         }
     } else if (warp == 8) {
         // ------------------------------- UMMA issuer -------------------------------
+        setmaxnreg_dec<40>();
         if (lane == 0) {
             constexpr uint32_t idesc_qk = make_idesc_bf16(kMhaBlock, kMhaBlock, false, false);
             constexpr uint32_t idesc_pv = make_idesc_bf16(kMhaBlock, D, false, true);
-            int stage = 0;
-            uint32_t phase = 0;
-            bool ok = true;
+            // descriptor low words: Q tiles fixed, K/V per ring slot; K steps add small constants
+            const uint32_t q_lo[2] = {sdesc_lo(smem_u32(smem_q), 16), sdesc_lo(smem_u32(smem_q + L::kTileBytes), 16)};
+            const uint32_t kv_lo0 = sdesc_lo(smem_u32(smem_kv), 16);
+            const uint32_t v_lbo = (static_cast<uint32_t>(L::kChunkBytes) >> 4) << 16;  // V is MN-major: chunk pitch
             // S_t = Q_t K^T over the D/16 k-steps of the tile in ring slot `slot`
             auto issue_qk = [&](int t, int slot) {
-                const uint32_t q_addr = smem_u32(smem_q + t * L::kTileBytes);
-                const uint32_t k_addr = smem_u32(smem_kv + slot * L::kTileBytes);
+                const uint32_t d = tmem_base + kColS + t * kMhaBlock;
+                const uint32_t a0 = q_lo[t];
+                const uint32_t b0 = kv_lo0 + slot * (L::kTileBytes >> 4);
+                umma_ss_lo<false>(d, a0, b0, idesc_qk);
 #pragma unroll
-                for (int kk = 0; kk < D / 16; ++kk) {
-                    const uint32_t off = (kk / 4) * L::kChunkBytes + (kk % 4) * 32;
-                    umma_ss(tmem_base + kColS + t * kMhaBlock, make_sdesc_sw128(q_addr + off, 16, 1024),
-                            make_sdesc_sw128(k_addr + off, 16, 1024), idesc_qk, kk != 0);
+                for (int kk = 1; kk < D / 16; ++kk) {
+                    const uint32_t off = ((kk / 4) * L::kChunkBytes + (kk % 4) * 32) >> 4;
+                    umma_ss_lo<true>(d, a0 + off, b0 + off, idesc_qk);
                 }
                 umma_commit(&s_full[t]);
             };
             // O_t (+)= P_t V over the 8 k-steps (16 keys each) of the tile in ring slot `slot`
             auto issue_pv = [&](int t, int slot, bool first) {
-                const uint32_t v_addr = smem_u32(smem_kv + slot * L::kTileBytes);
+                const uint32_t d = tmem_base + kColO + t * D;
+                const uint32_t a0 = tmem_base + kColS + t * kMhaBlock;
+                const uint32_t b0 = (kv_lo0 & 0xFFFFu) + slot * (L::kTileBytes >> 4) + v_lbo;
+                umma_ts_lo(d, a0, b0, idesc_pv, first ? 0u : 1u);
 #pragma unroll
-                for (int kk = 0; kk < kMhaBlock / 16; ++kk)
-                    umma_ts(tmem_base + kColO + t * D, tmem_base + kColS + t * kMhaBlock + kk * 8,
-                            make_sdesc_sw128(v_addr + kk * 2048, L::kChunkBytes, 1024), idesc_pv, !(first && kk == 0));
+                for (int kk = 1; kk < kMhaBlock / 16; ++kk) umma_ts_lo(d, a0 + kk * 8, b0 + kk * (2048 >> 4), idesc_pv, 1u);
             };
+            int stage = 0;
+            uint32_t phase = 0;
+            bool ok = true;
             if (Jmax > 0) {
                 ok = mbar_wait(q_full, 0, abort_flag, 0x200);
                 if (ok) ok = mbar_wait(&kv_full[stage], phase, abort_flag, 0x210 + stage);
@@ -209,6 +235,7 @@ mha_fwd_kernel(const __grid_constant__ CUtensorMap tmap_q, const __grid_constant
                     if (j >= J[t]) continue;
                     ok = mbar_wait(&p_full[t], j & 1, abort_flag, 0x230 + t);
                     if (!ok) break;
+                    MLT_TR(0, j, t);
                     tc_fence_after();
                     issue_pv(t, vslot, j == 0);
                     if (j == J[t] - 1) umma_commit(&o_full[t]);
@@ -221,6 +248,7 @@ mha_fwd_kernel(const __grid_constant__ CUtensorMap tmap_q, const __grid_constant
                         }
                         issue_qk(t, kslot);
                     }
+                    MLT_TR(1, j, t);
                 }
                 if (!ok) break;
                 umma_commit(&kv_empty[vslot]);
@@ -232,6 +260,7 @@ mha_fwd_kernel(const __grid_constant__ CUtensorMap tmap_q, const __grid_constant
         }
     } else {
         // ------------------- softmax, O rescale and epilogue of tile t -------------------
+        setmaxnreg_inc<232>();
         const int t = warp >> 2;
         const int quarter = warp & 3;
         const int row_in_tile = quarter * 32 + lane;
@@ -249,61 +278,82 @@ mha_fwd_kernel(const __grid_constant__ CUtensorMap tmap_q, const __grid_constant
         for (int j = 0; j < Jt; ++j) {
             ok = __all_sync(0xffffffffu, mbar_wait(&s_full[t], j & 1, abort_flag, 0x300 + t));
             if (!ok) break;
+            if (threadIdx.x == t * 128) MLT_TR(2, j, t);
             tc_fence_after();
-            uint32_t sr[128];
+            uint32_t s[4][32];  // this thread's row of S: 4 chunks of 32 keys
 #pragma unroll
-            for (int q = 0; q < 4; ++q) tmem_ld_32x32b_x32(s_addr + q * 32, *reinterpret_cast<uint32_t(*)[32]>(&sr[q * 32]));
+            for (int q = 0; q < 4; ++q) tmem_ld_32x32b_x32(s_addr + q * 32, s[q]);
             tmem_wait_ld();
-            float* s = reinterpret_cast<float*>(sr);
+            if (threadIdx.x == t * 128) MLT_TR(3, j, t);
             const int j0 = j * kMhaBlock;
             if (j0 + kMhaBlock - 1 > limit) {  // diagonal or tail block: mask keys beyond the row's last visible one
 #pragma unroll
-                for (int i = 0; i < 128; ++i)
-                    if (j0 + i > limit) s[i] = -INFINITY;
-            }
-            float mx = s[0];
+                for (int q = 0; q < 4; ++q)
 #pragma unroll
-            for (int i = 1; i < 128; ++i) mx = fmaxf(mx, s[i]);
+                    for (int i = 0; i < 32; ++i)
+                        if (j0 + q * 32 + i > limit) s[q][i] = 0xFF800000u;  // -inf
+            }
+            // row max over four independent chains (short dependency paths)
+            float mx[4];
+#pragma unroll
+            for (int q = 0; q < 4; ++q) {
+                mx[q] = fmaxf(__uint_as_float(s[q][0]), __uint_as_float(s[q][1]));
+#pragma unroll
+                for (int i = 2; i < 32; i += 2)
+                    mx[q] = fmaxf(mx[q], fmaxf(__uint_as_float(s[q][i]), __uint_as_float(s[q][i + 1])));
+            }
+            const float mxr = fmaxf(fmaxf(mx[0], mx[1]), fmaxf(mx[2], mx[3]));
             // lazy rescale: move the reference max only when it is off by more than the threshold
             float alpha = 1.0f;
             bool moved = false;
             if (j == 0) {
-                m_run = mx;
-            } else if ((mx - m_run) * c > kRescaleThreshold || (m_run == -INFINITY && mx > -INFINITY)) {
-                alpha = (m_run == -INFINITY) ? 0.0f : fast_exp2((m_run - mx) * c);
-                m_run = mx;
+                m_run = mxr;
+            } else if ((mxr - m_run) * c > kRescaleThreshold || (m_run == -INFINITY && mxr > -INFINITY)) {
+                alpha = (m_run == -INFINITY) ? 0.0f : fast_exp2((m_run - mxr) * c);
+                m_run = mxr;
                 moved = true;
             }
             if (__any_sync(0xffffffffu, moved)) {
-                // S_t(j) complete implies every earlier UMMA, so P_t(j-1) V has landed in O_t
+                // S_t(j) complete implies every earlier UMMA of this tile, so P_t(j-1) V has landed in O_t
 #pragma unroll 1
-                for (int q = 0; q < D / 32; ++q) {
-                    uint32_t o[32];
-                    tmem_ld_32x32b_x32(o_addr + q * 32, o);
+                for (int q = 0; q < D / 16; ++q) {
+                    uint32_t o[16];
+                    tmem_ld_32x32b_x16(o_addr + q * 16, o);
                     tmem_wait_ld();
 #pragma unroll
-                    for (int i = 0; i < 32; ++i) o[i] = __float_as_uint(__uint_as_float(o[i]) * alpha);
-                    tmem_st_32x32b_x32(o_addr + q * 32, o);
+                    for (int i = 0; i < 16; ++i) o[i] = __float_as_uint(__uint_as_float(o[i]) * alpha);
+                    tmem_st_32x32b_x16(o_addr + q * 16, o);
                 }
                 l_run *= alpha;
             }
             const float neg_mc = (m_run == -INFINITY) ? 0.0f : -m_run * c;
-            float sum = 0.0f;
-            uint32_t pk[64];
+            // p = 2^(s*c - m*c) with packed FP32 FMAs; P goes back to TMEM 32 keys at a time
+            const float2 c2 = make_float2(c, c), n2 = make_float2(neg_mc, neg_mc);
+            float2 acc0 = make_float2(0.0f, 0.0f), acc1 = make_float2(0.0f, 0.0f);
 #pragma unroll
-            for (int i = 0; i < 64; ++i) {
-                const float p0 = fast_exp2(fmaf(s[2 * i], c, neg_mc));
-                const float p1 = fast_exp2(fmaf(s[2 * i + 1], c, neg_mc));
-                sum += p0 + p1;
-                pk[i] = pack_bf16x2(p0, p1);
+            for (int q = 0; q < 4; ++q) {
+                uint32_t pk[16];
+#pragma unroll
+                for (int i = 0; i < 16; i += 2) {
+                    float2 x0 = ffma2(make_float2(__uint_as_float(s[q][2 * i]), __uint_as_float(s[q][2 * i + 1])), c2, n2);
+                    float2 x1 = ffma2(make_float2(__uint_as_float(s[q][2 * i + 2]), __uint_as_float(s[q][2 * i + 3])), c2, n2);
+                    x0.x = fast_exp2(x0.x);
+                    x0.y = fast_exp2(x0.y);
+                    x1.x = fast_exp2(x1.x);
+                    x1.y = fast_exp2(x1.y);
+                    acc0 = fadd2(acc0, x0);
+                    acc1 = fadd2(acc1, x1);
+                    pk[i] = pack_bf16x2(x0.x, x0.y);
+                    pk[i + 1] = pack_bf16x2(x1.x, x1.y);
+                }
+                tmem_st_32x32b_x16(s_addr + q * 16, pk);
             }
-            l_run += sum;
-            tmem_st_32x32b_x32(s_addr, *reinterpret_cast<uint32_t(*)[32]>(&pk[0]));
-            tmem_st_32x32b_x32(s_addr + 32, *reinterpret_cast<uint32_t(*)[32]>(&pk[32]));
             tmem_wait_st();
             tc_fence_before();
             __syncwarp();
             if (lane == 0) mbar_arrive(&p_full[t]);
+            l_run += (acc0.x + acc0.y) + (acc1.x + acc1.y);
+            if (threadIdx.x == t * 128) MLT_TR(4, j, t);
         }
 
         if (ok && Jt > 0) {
@@ -314,19 +364,19 @@ mha_fwd_kernel(const __grid_constant__ CUtensorMap tmap_q, const __grid_constant
                 const bool valid = qi < p.Nq;
                 __nv_bfloat16* orow = p.O + (static_cast<int64_t>(bh) * p.Nq + qi) * D;
 #pragma unroll 1
-                for (int q = 0; q < D / 32; ++q) {
-                    uint32_t o[32];
-                    tmem_ld_32x32b_x32(o_addr + q * 32, o);
+                for (int q = 0; q < D / 16; ++q) {
+                    uint32_t o[16];
+                    tmem_ld_32x32b_x16(o_addr + q * 16, o);
                     tmem_wait_ld();
                     if (valid) {
 #pragma unroll
-                        for (int v = 0; v < 4; ++v) {
+                        for (int v = 0; v < 2; ++v) {
                             uint4 out;
                             out.x = pack_bf16x2(__uint_as_float(o[v * 8 + 0]) * inv_l, __uint_as_float(o[v * 8 + 1]) * inv_l);
                             out.y = pack_bf16x2(__uint_as_float(o[v * 8 + 2]) * inv_l, __uint_as_float(o[v * 8 + 3]) * inv_l);
                             out.z = pack_bf16x2(__uint_as_float(o[v * 8 + 4]) * inv_l, __uint_as_float(o[v * 8 + 5]) * inv_l);
                             out.w = pack_bf16x2(__uint_as_float(o[v * 8 + 6]) * inv_l, __uint_as_float(o[v * 8 + 7]) * inv_l);
-                            *reinterpret_cast<uint4*>(orow + q * 32 + v * 8) = out;
+                            *reinterpret_cast<uint4*>(orow + q * 16 + v * 8) = out;
                         }
                     }
                 }
@@ -344,6 +394,11 @@ mha_fwd_kernel(const __grid_constant__ CUtensorMap tmap_q, const __grid_constant
         tmem_dealloc(tmem_base, 512);
     }
 }
+
+#ifdef MLT_TRACE
+static long long* g_trace_ptr = nullptr;
+extern "C" void mlt_debug_set_trace(long long* ptr) { g_trace_ptr = ptr; }
+#endif
 
 inline int mha_configure() {
     if (cudaFuncSetAttribute(mha_fwd_kernel<64>, cudaFuncAttributeMaxDynamicSharedMemorySize, MhaSmem<64>::kTotal) !=
@@ -368,6 +423,9 @@ inline int mha_launch(const CUtensorMap& tq, const CUtensorMap& tk, const CUtens
     p.scale = scale;
     p.num_pairs = (Nq + 2 * kMhaBlock - 1) / (2 * kMhaBlock);
     p.head_group = 8;
+#ifdef MLT_TRACE
+    p.trace = g_trace_ptr;
+#endif
     const int64_t items = static_cast<int64_t>(p.num_pairs) * p.BH;
     if (items > INT32_MAX) return 2;
     const int grid = static_cast<int>(items);
