@@ -109,6 +109,11 @@ int forced_variant() {
     return v;
 }
 
+int debug_env_int(const char* name, int fallback) {
+    const char* e = std::getenv(name);
+    return e && std::atoi(e) > 0 ? std::atoi(e) : fallback;
+}
+
 inline bool aligned16(const void* p) { return (reinterpret_cast<uintptr_t>(p) & 15u) == 0; }
 
 }  // namespace
@@ -210,7 +215,8 @@ int mlt_gemm(const void* A, const void* B, void* C, int64_t M, int64_t N, int64_
     p.tiles_m = static_cast<int>(tiles_m);
     p.tiles_n = static_cast<int>(tiles_n);
     if (variant == 0) {
-        p.group_m = 8;
+        // M-tiles per raster group: wide problems re-read B once per group, so fewer, taller groups pay
+        p.group_m = debug_env_int("MLT_GEMM_GROUP_M", tiles_n >= 32 ? 16 : 8);
         const int clusters = static_cast<int>(std::min<int64_t>(tiles_m * tiles_n, dev.sm_count / 2));
         gemm_bf16_pair_kernel<6><<<2 * clusters, kGemmThreads, GemmPairSmem<6>::kTotal, st>>>(ta, tb, p);
     } else {
