@@ -119,34 +119,41 @@ gemm_bf16_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_consta
         }
     } else if (warp == 1) {
         // ----------------------------- MMA issuer -----------------------------
-        if (lane == 0) {
+        // The whole warp runs the loop (uniform control flow keeps descriptors in the uniform datapath);
+        // one elected lane executes the tcgen05 instructions.
+        {
+            const bool leader = elect_one();
             constexpr uint32_t idesc = make_idesc_bf16(kGemmBM, BN, /*a_mn_major=*/false, /*b_mn_major=*/true);
+            const uint32_t a_lo0 = sdesc_lo(smem_u32(smem), 16);
+            const uint32_t b_lo0 = sdesc_lo(smem_u32(smem + L::kABytes), kGemmBK * 128);
             int stage = 0;
             uint32_t phase = 0;
             int acc = 0;
             uint32_t acc_phase = 0;
             bool ok = true;
             for (int tile = blockIdx.x; tile < num_tiles && ok; tile += gridDim.x) {
-                ok = mbar_wait(&acc_empty[acc], acc_phase ^ 1, abort_flag, 0x300 + acc);
+                ok = __all_sync(0xffffffffu, mbar_wait(&acc_empty[acc], acc_phase ^ 1, abort_flag, 0x300 + acc));
                 if (!ok) break;
                 tc_fence_after();
                 const uint32_t d_tmem = tmem_base + acc * BN;
                 for (int kb = 0; kb < num_kb; ++kb) {
-                    ok = mbar_wait(&full[stage], phase, abort_flag, 0x200 + stage);
+                    ok = __all_sync(0xffffffffu, mbar_wait(&full[stage], phase, abort_flag, 0x200 + stage));
                     if (!ok) break;
                     tc_fence_after();
-                    const uint32_t sa = smem_u32(smem + stage * L::kStageBytes);
-                    const uint32_t sb = sa + L::kABytes;
+                    const uint32_t a_lo = a_lo0 + stage * (L::kStageBytes >> 4);
+                    const uint32_t b_lo = b_lo0 + stage * (L::kStageBytes >> 4);
+                    if (leader) {
+                        umma_ss_lo_dyn(d_tmem, a_lo, b_lo, idesc, kb != 0);
 #pragma unroll
-                    for (int k = 0; k < kGemmBK / 16; ++k) {
-                        const uint64_t da = make_sdesc_sw128(sa + k * 32, 16, 1024);
-                        const uint64_t db = make_sdesc_sw128(sb + k * 2048, kGemmBK * 128, 1024);
-                        umma_ss(d_tmem, da, db, idesc, (kb | k) != 0);
+                        for (int k = 1; k < kGemmBK / 16; ++k)
+                            umma_ss_lo<true>(d_tmem, a_lo + k * (32 >> 4), b_lo + k * (2048 >> 4), idesc);
+                        umma_commit(&empty[stage]);  // frees the smem stage once these UMMAs have read it
                     }
-                    umma_commit(&empty[stage]);  // frees the smem stage once these UMMAs have read it
+                    __syncwarp();
                     if (++stage == kStages) { stage = 0; phase ^= 1; }
                 }
-                if (ok) umma_commit(&acc_full[acc]);
+                if (ok && leader) umma_commit(&acc_full[acc]);
+                __syncwarp();
                 if (++acc == 2) { acc = 0; acc_phase ^= 1; }
             }
         }
@@ -308,34 +315,39 @@ gemm_bf16_pair_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_c
         }
     } else if (warp == 1) {
         // ----------------------------- UMMA issuer (leader CTA only) -----------------------------
-        if (leader && lane == 0) {
+        if (leader) {
+            // whole warp, uniform control flow; one elected lane executes the tcgen05 instructions
+            const bool issuer = elect_one();
             constexpr uint32_t idesc = make_idesc_bf16(kPairBM, kPairBN, /*a_mn_major=*/false, /*b_mn_major=*/true);
+            const uint32_t a_lo0 = sdesc_lo(smem_u32(smem), 16);
+            const uint32_t b_lo0 = sdesc_lo(smem_u32(smem + L::kABytes), kGemmBK * 128);
             int stage = 0;
             uint32_t phase = 0;
             int acc = 0;
             uint32_t acc_phase = 0;
             bool ok = true;
             for (int tile = cluster_id; tile < num_tiles && ok; tile += num_clusters) {
-                ok = mbar_wait(&acc_empty[acc], acc_phase ^ 1, abort_flag, 0x300 + acc);
+                ok = __all_sync(0xffffffffu, mbar_wait(&acc_empty[acc], acc_phase ^ 1, abort_flag, 0x300 + acc));
                 if (!ok) break;
                 tc_fence_after();
                 const uint32_t d_tmem = tmem_base + acc * kPairBN;
                 for (int kb = 0; kb < num_kb; ++kb) {
-                    ok = mbar_wait(&full[stage], phase, abort_flag, 0x200 + stage);
+                    ok = __all_sync(0xffffffffu, mbar_wait(&full[stage], phase, abort_flag, 0x200 + stage));
                     if (!ok) break;
                     tc_fence_after();
-                    const uint32_t sa = smem_u32(smem + stage * L::kStageBytes);
-                    const uint32_t sb = sa + L::kABytes;
+                    const uint32_t a_lo = a_lo0 + stage * (L::kStageBytes >> 4);
+                    const uint32_t b_lo = b_lo0 + stage * (L::kStageBytes >> 4);
+                    if (issuer) {
 #pragma unroll
-                    for (int k = 0; k < kGemmBK / 16; ++k) {
-                        const uint64_t da = make_sdesc_sw128(sa + k * 32, 16, 1024);
-                        const uint64_t db = make_sdesc_sw128(sb + k * 2048, kGemmBK * 128, 1024);
-                        umma_ss_pair(d_tmem, da, db, idesc, (kb | k) != 0);
+                        for (int k = 0; k < kGemmBK / 16; ++k)
+                            umma_ss_pair_lo(d_tmem, a_lo + k * (32 >> 4), b_lo + k * (2048 >> 4), idesc, (kb | k) != 0);
+                        umma_commit_pair(&empty[stage], 3);
                     }
-                    umma_commit_pair(&empty[stage], 3);
+                    __syncwarp();
                     if (++stage == kStages) { stage = 0; phase ^= 1; }
                 }
-                if (ok) umma_commit_pair(&acc_full[acc], 3);
+                if (ok && issuer) umma_commit_pair(&acc_full[acc], 3);
+                __syncwarp();
                 if (++acc == 2) { acc = 0; acc_phase ^= 1; }
             }
         }

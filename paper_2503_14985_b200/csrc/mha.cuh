@@ -180,80 +180,94 @@ mha_fwd_kernel(const __grid_constant__ CUtensorMap tmap_q, const __grid_constant
         }
     } else if (warp == 8) {
         // ------------------------------- UMMA issuer -------------------------------
+        // The whole warp runs this code (uniform control flow keeps addresses and descriptors in the uniform
+        // datapath: an issue costs about 20 clocks instead of about 46 from a single divergent lane); one
+        // elected lane executes the tcgen05 instructions.
         setmaxnreg_dec<40>();
-        if (lane == 0) {
+        {
+            const bool leader = elect_one();
             constexpr uint32_t idesc_qk = make_idesc_bf16(kMhaBlock, kMhaBlock, false, false);
             constexpr uint32_t idesc_pv = make_idesc_bf16(kMhaBlock, D, false, true);
             // descriptor low words: Q tiles fixed, K/V per ring slot; K steps add small constants
-            const uint32_t q_lo[2] = {sdesc_lo(smem_u32(smem_q), 16), sdesc_lo(smem_u32(smem_q + L::kTileBytes), 16)};
+            const uint32_t q_lo0 = sdesc_lo(smem_u32(smem_q), 16);
             const uint32_t kv_lo0 = sdesc_lo(smem_u32(smem_kv), 16);
             const uint32_t v_lbo = (static_cast<uint32_t>(L::kChunkBytes) >> 4) << 16;  // V is MN-major: chunk pitch
             // S_t = Q_t K^T over the D/16 k-steps of the tile in ring slot `slot`
             auto issue_qk = [&](int t, int slot) {
                 const uint32_t d = tmem_base + kColS + t * kMhaBlock;
-                const uint32_t a0 = q_lo[t];
+                const uint32_t a0 = q_lo0 + t * (L::kTileBytes >> 4);
                 const uint32_t b0 = kv_lo0 + slot * (L::kTileBytes >> 4);
-                umma_ss_lo<false>(d, a0, b0, idesc_qk);
+                if (leader) {
+                    umma_ss_lo<false>(d, a0, b0, idesc_qk);
 #pragma unroll
-                for (int kk = 1; kk < D / 16; ++kk) {
-                    const uint32_t off = ((kk / 4) * L::kChunkBytes + (kk % 4) * 32) >> 4;
-                    umma_ss_lo<true>(d, a0 + off, b0 + off, idesc_qk);
+                    for (int kk = 1; kk < D / 16; ++kk) {
+                        const uint32_t off = ((kk / 4) * L::kChunkBytes + (kk % 4) * 32) >> 4;
+                        umma_ss_lo<true>(d, a0 + off, b0 + off, idesc_qk);
+                    }
+                    umma_commit(&s_full[t]);
                 }
-                umma_commit(&s_full[t]);
+                __syncwarp();
             };
             // O_t (+)= P_t V over the 8 k-steps (16 keys each) of the tile in ring slot `slot`
             auto issue_pv = [&](int t, int slot, bool first) {
                 const uint32_t d = tmem_base + kColO + t * D;
                 const uint32_t a0 = tmem_base + kColS + t * kMhaBlock;
                 const uint32_t b0 = (kv_lo0 & 0xFFFFu) + slot * (L::kTileBytes >> 4) + v_lbo;
-                umma_ts_lo(d, a0, b0, idesc_pv, first ? 0u : 1u);
+                if (leader) {
+                    umma_ts_lo(d, a0, b0, idesc_pv, first ? 0u : 1u);
 #pragma unroll
-                for (int kk = 1; kk < kMhaBlock / 16; ++kk) umma_ts_lo(d, a0 + kk * 8, b0 + kk * (2048 >> 4), idesc_pv, 1u);
+                    for (int kk = 1; kk < kMhaBlock / 16; ++kk)
+                        umma_ts_lo(d, a0 + kk * 8, b0 + kk * (2048 >> 4), idesc_pv, 1u);
+                }
+                __syncwarp();
+            };
+            auto wait_all = [&](uint64_t* bar, uint32_t parity, uint32_t id) {
+                return __all_sync(0xffffffffu, mbar_wait(bar, parity, abort_flag, id)) != 0;
             };
             int stage = 0;
             uint32_t phase = 0;
             bool ok = true;
             if (Jmax > 0) {
-                ok = mbar_wait(q_full, 0, abort_flag, 0x200);
-                if (ok) ok = mbar_wait(&kv_full[stage], phase, abort_flag, 0x210 + stage);
+                ok = wait_all(q_full, 0, 0x200);
+                if (ok) ok = wait_all(&kv_full[stage], phase, 0x210 + stage);
                 if (ok) {
                     tc_fence_after();
                     for (int t = 0; t < 2; ++t)
                         if (J[t] > 0) issue_qk(t, stage);
-                    umma_commit(&kv_empty[stage]);
+                    if (leader) umma_commit(&kv_empty[stage]);
                     if (++stage == kStages) { stage = 0; phase ^= 1; }
                 }
             }
             for (int j = 0; j < Jmax && ok; ++j) {
                 const int vslot = stage;
-                ok = mbar_wait(&kv_full[vslot], phase, abort_flag, 0x220 + vslot);
+                ok = wait_all(&kv_full[vslot], phase, 0x220 + vslot);
                 if (!ok) break;
                 if (++stage == kStages) { stage = 0; phase ^= 1; }
                 const int kslot = stage;  // K_{j+1}, if there is one
                 bool k_ready = false;
                 for (int t = 0; t < 2 && ok; ++t) {
                     if (j >= J[t]) continue;
-                    ok = mbar_wait(&p_full[t], j & 1, abort_flag, 0x230 + t);
+                    ok = wait_all(&p_full[t], j & 1, 0x230 + t);
                     if (!ok) break;
-                    MLT_TR(0, j, t);
+                    if (leader) MLT_TR(0, j, t);
                     tc_fence_after();
                     issue_pv(t, vslot, j == 0);
-                    if (j == J[t] - 1) umma_commit(&o_full[t]);
+                    if (j == J[t] - 1 && leader) umma_commit(&o_full[t]);
                     if (j + 1 < J[t]) {
                         if (!k_ready) {
-                            ok = mbar_wait(&kv_full[kslot], phase, abort_flag, 0x240 + kslot);
+                            ok = wait_all(&kv_full[kslot], phase, 0x240 + kslot);
                             if (!ok) break;
                             tc_fence_after();
                             k_ready = true;
                         }
                         issue_qk(t, kslot);
                     }
-                    MLT_TR(1, j, t);
+                    if (leader) MLT_TR(1, j, t);
                 }
                 if (!ok) break;
-                umma_commit(&kv_empty[vslot]);
+                if (leader) umma_commit(&kv_empty[vslot]);
                 if (j + 1 < Jmax) {
-                    umma_commit(&kv_empty[kslot]);
+                    if (leader) umma_commit(&kv_empty[kslot]);
                     if (++stage == kStages) { stage = 0; phase ^= 1; }
                 }
             }
@@ -293,66 +307,92 @@ mha_fwd_kernel(const __grid_constant__ CUtensorMap tmap_q, const __grid_constant
                     for (int i = 0; i < 32; ++i)
                         if (j0 + q * 32 + i > limit) s[q][i] = 0xFF800000u;  // -inf
             }
-            // row max over four independent chains (short dependency paths)
-            float mx[4];
+            // One pass: p = 2^((s - m_ref)*c) against the reference max of the previous blocks while the
+            // row max of this block is taken on the side (ALU pipe, off the MUFU-bound path).  Software
+            // pipelined by hand: the exponentials of the next four keys are issued before the current four
+            // are summed and packed.  Only if the block max beats the reference by more than the threshold
+            // (or there is no reference yet) are O and l rescaled and the pass repeated with the new max.
+            float mx[4] = {-INFINITY, -INFINITY, -INFINITY, -INFINITY};
+            float2 acc0, acc1;
+            auto exp_pass = [&](float neg_mc, bool with_max) {
+                const float2 c2 = make_float2(c, c), n2 = make_float2(neg_mc, neg_mc);
+                acc0 = make_float2(0.0f, 0.0f);
+                acc1 = make_float2(0.0f, 0.0f);
+                float2 xa = ffma2(make_float2(__uint_as_float(s[0][0]), __uint_as_float(s[0][1])), c2, n2);
+                float2 xb = ffma2(make_float2(__uint_as_float(s[0][2]), __uint_as_float(s[0][3])), c2, n2);
+                xa.x = fast_exp2(xa.x);
+                xa.y = fast_exp2(xa.y);
+                xb.x = fast_exp2(xb.x);
+                xb.y = fast_exp2(xb.y);
 #pragma unroll
-            for (int q = 0; q < 4; ++q) {
-                mx[q] = fmaxf(__uint_as_float(s[q][0]), __uint_as_float(s[q][1]));
+                for (int q = 0; q < 4; ++q) {
+                    uint32_t pk[16];
 #pragma unroll
-                for (int i = 2; i < 32; i += 2)
-                    mx[q] = fmaxf(mx[q], fmaxf(__uint_as_float(s[q][i]), __uint_as_float(s[q][i + 1])));
-            }
-            const float mxr = fmaxf(fmaxf(mx[0], mx[1]), fmaxf(mx[2], mx[3]));
-            // lazy rescale: move the reference max only when it is off by more than the threshold
-            float alpha = 1.0f;
-            bool moved = false;
+                    for (int i = 0; i < 32; i += 4) {
+                        const int e = q * 32 + i + 4;  // first key of the next group
+                        float2 ya = xa, yb = xb;
+                        if (e < 128) {
+                            ya = ffma2(make_float2(__uint_as_float(s[e >> 5][e & 31]), __uint_as_float(s[e >> 5][(e & 31) + 1])), c2, n2);
+                            yb = ffma2(make_float2(__uint_as_float(s[e >> 5][(e & 31) + 2]), __uint_as_float(s[e >> 5][(e & 31) + 3])), c2, n2);
+                            ya.x = fast_exp2(ya.x);
+                            ya.y = fast_exp2(ya.y);
+                            yb.x = fast_exp2(yb.x);
+                            yb.y = fast_exp2(yb.y);
+                        }
+                        if (with_max)
+                            mx[(i >> 2) & 3] = fmaxf(mx[(i >> 2) & 3],
+                                                     fmaxf(fmaxf(__uint_as_float(s[q][i]), __uint_as_float(s[q][i + 1])),
+                                                           fmaxf(__uint_as_float(s[q][i + 2]), __uint_as_float(s[q][i + 3]))));
+                        acc0 = fadd2(acc0, xa);
+                        acc1 = fadd2(acc1, xb);
+                        pk[i >> 1] = pack_bf16x2(xa.x, xa.y);
+                        pk[(i >> 1) + 1] = pack_bf16x2(xb.x, xb.y);
+                        xa = ya;
+                        xb = yb;
+                    }
+                    tmem_st_32x32b_x16(s_addr + q * 16, pk);
+                }
+            };
+            bool moved;
             if (j == 0) {
-                m_run = mxr;
-            } else if ((mxr - m_run) * c > kRescaleThreshold || (m_run == -INFINITY && mxr > -INFINITY)) {
-                alpha = (m_run == -INFINITY) ? 0.0f : fast_exp2((m_run - mxr) * c);
-                m_run = mxr;
-                moved = true;
-            }
-            if (__any_sync(0xffffffffu, moved)) {
-                // S_t(j) complete implies every earlier UMMA of this tile, so P_t(j-1) V has landed in O_t
+                // no reference yet: take the row max first
+#pragma unroll
+                for (int q = 0; q < 4; ++q)
+#pragma unroll
+                    for (int i = 0; i < 32; i += 4)
+                        mx[(i >> 2) & 3] = fmaxf(mx[(i >> 2) & 3],
+                                                 fmaxf(fmaxf(__uint_as_float(s[q][i]), __uint_as_float(s[q][i + 1])),
+                                                       fmaxf(__uint_as_float(s[q][i + 2]), __uint_as_float(s[q][i + 3]))));
+                m_run = fmaxf(fmaxf(mx[0], mx[1]), fmaxf(mx[2], mx[3]));
+                moved = false;
+                exp_pass((m_run == -INFINITY) ? 0.0f : -m_run * c, false);
+            } else {
+                exp_pass((m_run == -INFINITY) ? 0.0f : -m_run * c, true);
+                const float mxr = fmaxf(fmaxf(mx[0], mx[1]), fmaxf(mx[2], mx[3]));
+                moved = (mxr - m_run) * c > kRescaleThreshold || (m_run == -INFINITY && mxr > -INFINITY);
+                if (__any_sync(0xffffffffu, moved)) {
+                    // rare: rescale O_t and l by 2^((m_old - m_new)*c) (1 for rows whose reference stays) and redo P.
+                    // S_t(j) complete implies every earlier UMMA, so P_t(j-1) V has landed in O_t.
+                    const float alpha = !moved ? 1.0f : (m_run == -INFINITY ? 0.0f : fast_exp2((m_run - mxr) * c));
+                    if (moved) m_run = mxr;
 #pragma unroll 1
-                for (int q = 0; q < D / 16; ++q) {
-                    uint32_t o[16];
-                    tmem_ld_32x32b_x16(o_addr + q * 16, o);
-                    tmem_wait_ld();
+                    for (int q = 0; q < D / 16; ++q) {
+                        uint32_t o[16];
+                        tmem_ld_32x32b_x16(o_addr + q * 16, o);
+                        tmem_wait_ld();
 #pragma unroll
-                    for (int i = 0; i < 16; ++i) o[i] = __float_as_uint(__uint_as_float(o[i]) * alpha);
-                    tmem_st_32x32b_x16(o_addr + q * 16, o);
+                        for (int i = 0; i < 16; ++i) o[i] = __float_as_uint(__uint_as_float(o[i]) * alpha);
+                        tmem_st_32x32b_x16(o_addr + q * 16, o);
+                    }
+                    l_run *= alpha;
+                    exp_pass((m_run == -INFINITY) ? 0.0f : -m_run * c, false);
                 }
-                l_run *= alpha;
             }
-            const float neg_mc = (m_run == -INFINITY) ? 0.0f : -m_run * c;
-            // p = 2^(s*c - m*c) with packed FP32 FMAs; P goes back to TMEM 32 keys at a time
-            const float2 c2 = make_float2(c, c), n2 = make_float2(neg_mc, neg_mc);
-            float2 acc0 = make_float2(0.0f, 0.0f), acc1 = make_float2(0.0f, 0.0f);
-#pragma unroll
-            for (int q = 0; q < 4; ++q) {
-                uint32_t pk[16];
-#pragma unroll
-                for (int i = 0; i < 16; i += 2) {
-                    float2 x0 = ffma2(make_float2(__uint_as_float(s[q][2 * i]), __uint_as_float(s[q][2 * i + 1])), c2, n2);
-                    float2 x1 = ffma2(make_float2(__uint_as_float(s[q][2 * i + 2]), __uint_as_float(s[q][2 * i + 3])), c2, n2);
-                    x0.x = fast_exp2(x0.x);
-                    x0.y = fast_exp2(x0.y);
-                    x1.x = fast_exp2(x1.x);
-                    x1.y = fast_exp2(x1.y);
-                    acc0 = fadd2(acc0, x0);
-                    acc1 = fadd2(acc1, x1);
-                    pk[i] = pack_bf16x2(x0.x, x0.y);
-                    pk[i + 1] = pack_bf16x2(x1.x, x1.y);
-                }
-                tmem_st_32x32b_x16(s_addr + q * 16, pk);
-            }
+            l_run += (acc0.x + acc0.y) + (acc1.x + acc1.y);
             tmem_wait_st();
             tc_fence_before();
             __syncwarp();
             if (lane == 0) mbar_arrive(&p_full[t]);
-            l_run += (acc0.x + acc0.y) + (acc1.x + acc1.y);
             if (threadIdx.x == t * 128) MLT_TR(4, j, t);
         }
 
