@@ -31,7 +31,7 @@ namespace mlt {
 constexpr int kMhaBlock = 128;   // query rows per tile and keys per K/V block
 constexpr int kMhaThreads = 384; // three warpgroups
 constexpr float kLog2e = 1.4426950408889634f;
-constexpr float kRescaleThreshold = 8.0f;  // in log2 units: keep a stale max until it is off by more than 2^8
+constexpr float kRescaleThreshold = 64.0f;  // in log2 units: the reference max may lag by up to 2^64 (FP32 and BF16 share the exponent range)
 
 template <int D>
 struct MhaSmem {
