@@ -30,7 +30,7 @@ def build(force: bool = False) -> str:
         if stale:
             tmp = _LIB + f".tmp{os.getpid()}"
             cmd = ["g++", "-O3", "-march=native", "-std=c++17", "-fPIC", "-shared", "-pthread",
-                   "-fno-fast-math", "-o", tmp, _SRC]
+                   "-fno-fast-math", "-ffp-contract=off", "-o", tmp, _SRC]
             try:
                 subprocess.run(cmd, check=True, capture_output=True, text=True)
             except subprocess.CalledProcessError as e:  # pragma: no cover
