@@ -31,7 +31,7 @@ namespace mlt {
 constexpr int kMhaBlock = 128;   // query rows per tile and keys per K/V block
 constexpr int kMhaThreads = 384; // three warpgroups
 constexpr float kLog2e = 1.4426950408889634f;
-constexpr float kRescaleThreshold = 64.0f;  // in log2 units: the reference max may lag by up to 2^64 (FP32 and BF16 share the exponent range)
+constexpr float kRescaleLimit = 18446744073709551616.0f;  // 2^64: a block sum at or above it forces a new reference max
 
 template <int D>
 struct MhaSmem {
@@ -117,7 +117,10 @@ mha_fwd_kernel(const __grid_constant__ CUtensorMap tmap_q, const __grid_constant
     }
     const int Jmax = max(J[0], J[1]);
 
-    if (threadIdx.x == 0) {
+    // The loader lane initialises the barriers and issues the first loads (Q and the first K/V tiles: the ring
+    // is empty, nothing to wait for) before the CTA-wide sync, so they overlap the tensor-memory allocation.
+    int pre_tiles = 0;  // ring tiles already requested (K_0, V_0, K_1, ...)
+    if (warp == 9 && lane == 0) {
         mbar_init(q_full, 1);
         for (int s = 0; s < kStages; ++s) {
             mbar_init(&kv_full[s], 1);
@@ -130,11 +133,28 @@ mha_fwd_kernel(const __grid_constant__ CUtensorMap tmap_q, const __grid_constant
         }
         *abort_flag = 0;
         fence_mbar_init();
-    }
-    if (warp == 9 && lane == 0) {
         prefetch_tensormap(&tmap_q);
         prefetch_tensormap(&tmap_k);
         prefetch_tensormap(&tmap_v);
+        // K_0 first: with Q it is all the first product needs
+        pre_tiles = min(2 * Jmax, kStages);
+        for (int i = 0; i < pre_tiles; ++i) {
+            if (i == 1) {
+                mbar_arrive_expect_tx(q_full, 2 * L::kTileBytes);
+#pragma unroll
+                for (int t = 0; t < 2; ++t)
+#pragma unroll
+                    for (int c = 0; c < kChunks; ++c)
+                        tma_load_3d(smem_q + t * L::kTileBytes + c * L::kChunkBytes, &tmap_q, q_full, c * 64,
+                                    q_base + t * kMhaBlock, bh);
+            }
+            uint8_t* dst = smem_kv + i * L::kTileBytes;
+            mbar_arrive_expect_tx(&kv_full[i], L::kTileBytes);
+#pragma unroll
+            for (int c = 0; c < kChunks; ++c)
+                tma_load_3d(dst + c * L::kChunkBytes, (i & 1) == 0 ? &tmap_k : &tmap_v, &kv_full[i], c * 64,
+                            (i >> 1) * kMhaBlock, bh);
+        }
     }
     if (warp == 8) {
         tmem_alloc(tmem_base_slot, 512);
@@ -153,29 +173,19 @@ mha_fwd_kernel(const __grid_constant__ CUtensorMap tmap_q, const __grid_constant
         // ------------------------------- loader -------------------------------
         setmaxnreg_dec<40>();
         if (lane == 0) {
-            mbar_arrive_expect_tx(q_full, 2 * L::kTileBytes);
-#pragma unroll
-            for (int t = 0; t < 2; ++t)
+            int stage = pre_tiles == kStages ? 0 : pre_tiles;
+            uint32_t phase = pre_tiles == kStages ? 1 : 0;
+            bool ok = true;
+            for (int i = pre_tiles; i < 2 * Jmax && ok; ++i) {
+                ok = mbar_wait(&kv_empty[stage], phase ^ 1, abort_flag, 0x100 + stage);
+                if (!ok) break;
+                uint8_t* dst = smem_kv + stage * L::kTileBytes;
+                mbar_arrive_expect_tx(&kv_full[stage], L::kTileBytes);
 #pragma unroll
                 for (int c = 0; c < kChunks; ++c)
-                    tma_load_3d(smem_q + t * L::kTileBytes + c * L::kChunkBytes, &tmap_q, q_full, c * 64,
-                                q_base + t * kMhaBlock, bh);
-            int stage = 0;
-            uint32_t phase = 0;
-            bool ok = true;
-            for (int j = 0; j < Jmax && ok; ++j) {
-#pragma unroll
-                for (int kv = 0; kv < 2; ++kv) {
-                    ok = mbar_wait(&kv_empty[stage], phase ^ 1, abort_flag, 0x100 + stage);
-                    if (!ok) break;
-                    uint8_t* dst = smem_kv + stage * L::kTileBytes;
-                    mbar_arrive_expect_tx(&kv_full[stage], L::kTileBytes);
-#pragma unroll
-                    for (int c = 0; c < kChunks; ++c)
-                        tma_load_3d(dst + c * L::kChunkBytes, kv == 0 ? &tmap_k : &tmap_v, &kv_full[stage], c * 64,
-                                    j * kMhaBlock, bh);
-                    if (++stage == kStages) { stage = 0; phase ^= 1; }
-                }
+                    tma_load_3d(dst + c * L::kChunkBytes, (i & 1) == 0 ? &tmap_k : &tmap_v, &kv_full[stage], c * 64,
+                                (i >> 1) * kMhaBlock, bh);
+                if (++stage == kStages) { stage = 0; phase ^= 1; }
             }
         }
     } else if (warp == 8) {
@@ -307,55 +317,14 @@ mha_fwd_kernel(const __grid_constant__ CUtensorMap tmap_q, const __grid_constant
                     for (int i = 0; i < 32; ++i)
                         if (j0 + q * 32 + i > limit) s[q][i] = 0xFF800000u;  // -inf
             }
-            // One pass: p = 2^((s - m_ref)*c) against the reference max of the previous blocks while the
-            // row max of this block is taken on the side (ALU pipe, off the MUFU-bound path).  Software
-            // pipelined by hand: the exponentials of the next four keys are issued before the current four
-            // are summed and packed.  Only if the block max beats the reference by more than the threshold
-            // (or there is no reference yet) are O and l rescaled and the pass repeated with the new max.
-            float mx[4] = {-INFINITY, -INFINITY, -INFINITY, -INFINITY};
+            // One pass: p = 2^((s - m_ref)*c) against a reference max m_ref taken from an earlier block.  Any
+            // reference gives the same O / l and the same m_ref*scale + ln l as long as nothing overflows (FP32
+            // and BF16 share the exponent range), so the row max is not taken at all on the fast path.  Only if
+            // the block's sum reaches 2^64 (or is not finite) is the true row max taken, O and l rescaled to it
+            // and the pass repeated; the first block of a row takes its max first.
             float2 acc0, acc1;
-            auto exp_pass = [&](float neg_mc, bool with_max) {
-                const float2 c2 = make_float2(c, c), n2 = make_float2(neg_mc, neg_mc);
-                acc0 = make_float2(0.0f, 0.0f);
-                acc1 = make_float2(0.0f, 0.0f);
-                float2 xa = ffma2(make_float2(__uint_as_float(s[0][0]), __uint_as_float(s[0][1])), c2, n2);
-                float2 xb = ffma2(make_float2(__uint_as_float(s[0][2]), __uint_as_float(s[0][3])), c2, n2);
-                xa.x = fast_exp2(xa.x);
-                xa.y = fast_exp2(xa.y);
-                xb.x = fast_exp2(xb.x);
-                xb.y = fast_exp2(xb.y);
-#pragma unroll
-                for (int q = 0; q < 4; ++q) {
-                    uint32_t pk[16];
-#pragma unroll
-                    for (int i = 0; i < 32; i += 4) {
-                        const int e = q * 32 + i + 4;  // first key of the next group
-                        float2 ya = xa, yb = xb;
-                        if (e < 128) {
-                            ya = ffma2(make_float2(__uint_as_float(s[e >> 5][e & 31]), __uint_as_float(s[e >> 5][(e & 31) + 1])), c2, n2);
-                            yb = ffma2(make_float2(__uint_as_float(s[e >> 5][(e & 31) + 2]), __uint_as_float(s[e >> 5][(e & 31) + 3])), c2, n2);
-                            ya.x = fast_exp2(ya.x);
-                            ya.y = fast_exp2(ya.y);
-                            yb.x = fast_exp2(yb.x);
-                            yb.y = fast_exp2(yb.y);
-                        }
-                        if (with_max)
-                            mx[(i >> 2) & 3] = fmaxf(mx[(i >> 2) & 3],
-                                                     fmaxf(fmaxf(__uint_as_float(s[q][i]), __uint_as_float(s[q][i + 1])),
-                                                           fmaxf(__uint_as_float(s[q][i + 2]), __uint_as_float(s[q][i + 3]))));
-                        acc0 = fadd2(acc0, xa);
-                        acc1 = fadd2(acc1, xb);
-                        pk[i >> 1] = pack_bf16x2(xa.x, xa.y);
-                        pk[(i >> 1) + 1] = pack_bf16x2(xb.x, xb.y);
-                        xa = ya;
-                        xb = yb;
-                    }
-                    tmem_st_32x32b_x16(s_addr + q * 16, pk);
-                }
-            };
-            bool moved;
-            if (j == 0) {
-                // no reference yet: take the row max first
+            auto row_max = [&]() {
+                float mx[4] = {-INFINITY, -INFINITY, -INFINITY, -INFINITY};
 #pragma unroll
                 for (int q = 0; q < 4; ++q)
 #pragma unroll
@@ -363,18 +332,48 @@ mha_fwd_kernel(const __grid_constant__ CUtensorMap tmap_q, const __grid_constant
                         mx[(i >> 2) & 3] = fmaxf(mx[(i >> 2) & 3],
                                                  fmaxf(fmaxf(__uint_as_float(s[q][i]), __uint_as_float(s[q][i + 1])),
                                                        fmaxf(__uint_as_float(s[q][i + 2]), __uint_as_float(s[q][i + 3]))));
-                m_run = fmaxf(fmaxf(mx[0], mx[1]), fmaxf(mx[2], mx[3]));
-                moved = false;
-                exp_pass((m_run == -INFINITY) ? 0.0f : -m_run * c, false);
+                return fmaxf(fmaxf(mx[0], mx[1]), fmaxf(mx[2], mx[3]));
+            };
+            auto exp_pass = [&](float neg_mc) {
+                const float2 c2 = make_float2(c, c), n2 = make_float2(neg_mc, neg_mc);
+                acc0 = make_float2(0.0f, 0.0f);
+                acc1 = make_float2(0.0f, 0.0f);
+                uint32_t pk[16];
+#pragma unroll
+                for (int w = 0; w < 8; ++w) {  // waves of 16 keys
+#pragma unroll
+                    for (int i = 0; i < 8; i += 2) {
+                        const int k = w * 16 + 2 * i;
+                        float2 x0 = ffma2(make_float2(__uint_as_float(s[k >> 5][k & 31]), __uint_as_float(s[k >> 5][(k & 31) + 1])), c2, n2);
+                        float2 x1 = ffma2(make_float2(__uint_as_float(s[k >> 5][(k & 31) + 2]), __uint_as_float(s[k >> 5][(k & 31) + 3])), c2, n2);
+                        x0.x = fast_exp2(x0.x);
+                        x0.y = fast_exp2(x0.y);
+                        x1.x = fast_exp2(x1.x);
+                        x1.y = fast_exp2(x1.y);
+                        acc0 = fadd2(acc0, x0);
+                        acc1 = fadd2(acc1, x1);
+                        pk[(w & 1) * 8 + i] = pack_bf16x2(x0.x, x0.y);
+                        pk[(w & 1) * 8 + i + 1] = pack_bf16x2(x1.x, x1.y);
+                    }
+                    if (w & 1) tmem_st_32x32b_x16(s_addr + (w >> 1) * 16, pk);
+                }
+            };
+            if (j == 0) {
+                m_run = row_max();  // no reference yet
+                exp_pass((m_run == -INFINITY) ? 0.0f : -m_run * c);
             } else {
-                exp_pass((m_run == -INFINITY) ? 0.0f : -m_run * c, true);
-                const float mxr = fmaxf(fmaxf(mx[0], mx[1]), fmaxf(mx[2], mx[3]));
-                moved = (mxr - m_run) * c > kRescaleThreshold || (m_run == -INFINITY && mxr > -INFINITY);
+                exp_pass((m_run == -INFINITY) ? 0.0f : -m_run * c);
+                const float blk = (acc0.x + acc0.y) + (acc1.x + acc1.y);
+                const bool moved = !(blk < kRescaleLimit);  // also catches inf and NaN
                 if (__any_sync(0xffffffffu, moved)) {
                     // rare: rescale O_t and l by 2^((m_old - m_new)*c) (1 for rows whose reference stays) and redo P.
                     // S_t(j) complete implies every earlier UMMA, so P_t(j-1) V has landed in O_t.
-                    const float alpha = !moved ? 1.0f : (m_run == -INFINITY ? 0.0f : fast_exp2((m_run - mxr) * c));
-                    if (moved) m_run = mxr;
+                    float alpha = 1.0f;
+                    if (moved) {
+                        const float mxr = fmaxf(row_max(), m_run);
+                        alpha = m_run == -INFINITY ? 0.0f : fast_exp2((m_run - mxr) * c);
+                        m_run = mxr;
+                    }
 #pragma unroll 1
                     for (int q = 0; q < D / 16; ++q) {
                         uint32_t o[16];
@@ -385,7 +384,7 @@ mha_fwd_kernel(const __grid_constant__ CUtensorMap tmap_q, const __grid_constant
                         tmem_st_32x32b_x16(o_addr + q * 16, o);
                     }
                     l_run *= alpha;
-                    exp_pass((m_run == -INFINITY) ? 0.0f : -m_run * c, false);
+                    exp_pass((m_run == -INFINITY) ? 0.0f : -m_run * c);
                 }
             }
             l_run += (acc0.x + acc0.y) + (acc1.x + acc1.y);
@@ -402,23 +401,35 @@ mha_fwd_kernel(const __grid_constant__ CUtensorMap tmap_q, const __grid_constant
                 tc_fence_after();
                 const float inv_l = 1.0f / l_run;
                 const bool valid = qi < p.Nq;
-                __nv_bfloat16* orow = p.O + (static_cast<int64_t>(bh) * p.Nq + qi) * D;
+                // O / l -> BF16 into the tile's Q region (no product reads it any more), 16-byte chunks XOR-swizzled
+                // by row; then each warp writes its own 32 rows out row-major, 512 contiguous bytes per instruction.
+                constexpr int kRowChunks = D / 8;  // 16-byte chunks per row
+                uint8_t* stage_o = smem_q + t * L::kTileBytes;
 #pragma unroll 1
                 for (int q = 0; q < D / 16; ++q) {
                     uint32_t o[16];
                     tmem_ld_32x32b_x16(o_addr + q * 16, o);
                     tmem_wait_ld();
-                    if (valid) {
 #pragma unroll
-                        for (int v = 0; v < 2; ++v) {
-                            uint4 out;
-                            out.x = pack_bf16x2(__uint_as_float(o[v * 8 + 0]) * inv_l, __uint_as_float(o[v * 8 + 1]) * inv_l);
-                            out.y = pack_bf16x2(__uint_as_float(o[v * 8 + 2]) * inv_l, __uint_as_float(o[v * 8 + 3]) * inv_l);
-                            out.z = pack_bf16x2(__uint_as_float(o[v * 8 + 4]) * inv_l, __uint_as_float(o[v * 8 + 5]) * inv_l);
-                            out.w = pack_bf16x2(__uint_as_float(o[v * 8 + 6]) * inv_l, __uint_as_float(o[v * 8 + 7]) * inv_l);
-                            *reinterpret_cast<uint4*>(orow + q * 16 + v * 8) = out;
-                        }
+                    for (int v = 0; v < 2; ++v) {
+                        uint4 out;
+                        out.x = pack_bf16x2(__uint_as_float(o[v * 8 + 0]) * inv_l, __uint_as_float(o[v * 8 + 1]) * inv_l);
+                        out.y = pack_bf16x2(__uint_as_float(o[v * 8 + 2]) * inv_l, __uint_as_float(o[v * 8 + 3]) * inv_l);
+                        out.z = pack_bf16x2(__uint_as_float(o[v * 8 + 4]) * inv_l, __uint_as_float(o[v * 8 + 5]) * inv_l);
+                        out.w = pack_bf16x2(__uint_as_float(o[v * 8 + 6]) * inv_l, __uint_as_float(o[v * 8 + 7]) * inv_l);
+                        const int chunk = (q * 2 + v) ^ (row_in_tile & (kRowChunks - 1));
+                        *reinterpret_cast<uint4*>(stage_o + row_in_tile * (D * 2) + chunk * 16) = out;
                     }
+                }
+                __syncwarp();
+                constexpr int kRowsPerStore = 32 / kRowChunks;
+                __nv_bfloat16* obase = p.O + (static_cast<int64_t>(bh) * p.Nq + q_base + t * kMhaBlock) * D;
+#pragma unroll 4
+                for (int r0 = 0; r0 < 32; r0 += kRowsPerStore) {
+                    const int rr = quarter * 32 + r0 + lane / kRowChunks;
+                    const int cc = lane % kRowChunks;
+                    const uint4 v = *reinterpret_cast<const uint4*>(stage_o + rr * (D * 2) + ((cc ^ (rr & (kRowChunks - 1))) * 16));
+                    if (q_base + t * kMhaBlock + rr < p.Nq) *reinterpret_cast<uint4*>(obase + rr * D + cc * 8) = v;
                 }
                 if (valid && p.LSE) p.LSE[static_cast<int64_t>(bh) * p.Nq + qi] = m_run * p.scale + logf(l_run);
             }
