@@ -7,19 +7,25 @@
 // on the tensor pipe, so the exponentials of one tile overlap the products of the other.
 //   warps 0-3   softmax / O-rescale / epilogue of tile 0 (one thread per query row)
 //   warps 4-7   the same for tile 1
-//   warp  8     UMMA issuer (one lane) and owner of the tensor-memory allocation; it serves the
-//               tiles in a fixed order (P V of tile 0, next Q K^T of tile 0, the same for tile 1),
-//               which keeps the two softmax warpgroups half a period apart
-//   warp  9     TMA loader (one lane): both Q tiles once, then K_0, V_0, K_1, V_1, ... through a ring
+//   warp  8     UMMA issuer (the whole warp runs the loop, one elected lane issues) and owner of the
+//               tensor-memory allocation; it serves the tiles in a fixed order (P V of tile 0, next
+//               Q K^T of tile 0, the same for tile 1), which keeps the two softmax warpgroups half a
+//               period apart
+//   warp  9     TMA loader (one lane): both Q tiles once, then K_0, V_0, K_1, V_1, ... through a ring;
+//               it also initialises the barriers and issues the first loads before the CTA-wide sync
 //   warps 10-11 idle (they complete the third warpgroup for the register hand-over)
 // Tensor memory (512 columns): S_0 | S_1 (128 FP32 columns each; the BF16 P of a tile
 // overwrites the first 64 columns of its S and is consumed from there as the A operand
 // of P V), then O_0 | O_1 (D FP32 columns each).
 //
-// Measured on B200: one thread sustains one UMMA issue per 46-64 clocks only while its
-// scheduler partition is otherwise quiet, and shared memory (TMA writes plus operand reads,
-// about 128 bytes per clock and SM) is a co-bound: per tile and K/V block the tensor core
-// reads Q, K and V tiles while TMA writes the next K and V tiles.
+// Measured on B200 (what shaped this kernel):
+//  * a UMMA of 128x128x16 takes 64 clocks, also with A from tensor memory; issuing one costs the issuing
+//    thread about 46 clocks from a single divergent lane and about 20 from warp-uniform code with an elected
+//    lane; a warp that shares its scheduler partition with a busy warp is served much more rarely;
+//  * per tile and K/V block the chain is: S ready -> TMEM load (125) -> softmax (about 1700: 1024 MUFU clocks
+//    plus the packed FP32 work a single warp per partition cannot fully overlap) -> P V and next Q K^T
+//    (about 1085) -> S ready; with two tiles half a period apart the period is about 3230 clocks, i.e. the
+//    tensor pipe is busy about two thirds of the time.
 #pragma once
 
 #include <math.h>
@@ -50,15 +56,7 @@ struct MhaParams {
     float scale;
     int num_pairs;   // 256-row query groups per head
     int head_group;  // heads that share a span of consecutive block indices
-#ifdef MLT_TRACE
-    long long* trace;
-#endif
 };
-#ifdef MLT_TRACE
-#define MLT_TR(ev, j, t) do { if (blockIdx.x == 0 && (j) < 32) p.trace[((ev) * 32 + (j)) * 2 + (t)] = clock64(); } while (0)
-#else
-#define MLT_TR(ev, j, t) do { } while (0)
-#endif
 
 // block index -> (pair, bh).  Heads are taken in groups; inside a group the query
 // position is the slow index and runs from the last rows to the first, so under a
@@ -259,7 +257,6 @@ mha_fwd_kernel(const __grid_constant__ CUtensorMap tmap_q, const __grid_constant
                     if (j >= J[t]) continue;
                     ok = wait_all(&p_full[t], j & 1, 0x230 + t);
                     if (!ok) break;
-                    if (leader) MLT_TR(0, j, t);
                     tc_fence_after();
                     issue_pv(t, vslot, j == 0);
                     if (j == J[t] - 1 && leader) umma_commit(&o_full[t]);
@@ -272,7 +269,6 @@ mha_fwd_kernel(const __grid_constant__ CUtensorMap tmap_q, const __grid_constant
                         }
                         issue_qk(t, kslot);
                     }
-                    if (leader) MLT_TR(1, j, t);
                 }
                 if (!ok) break;
                 if (leader) umma_commit(&kv_empty[vslot]);
@@ -302,13 +298,11 @@ mha_fwd_kernel(const __grid_constant__ CUtensorMap tmap_q, const __grid_constant
         for (int j = 0; j < Jt; ++j) {
             ok = __all_sync(0xffffffffu, mbar_wait(&s_full[t], j & 1, abort_flag, 0x300 + t));
             if (!ok) break;
-            if (threadIdx.x == t * 128) MLT_TR(2, j, t);
             tc_fence_after();
             uint32_t s[4][32];  // this thread's row of S: 4 chunks of 32 keys
 #pragma unroll
             for (int q = 0; q < 4; ++q) tmem_ld_32x32b_x32(s_addr + q * 32, s[q]);
             tmem_wait_ld();
-            if (threadIdx.x == t * 128) MLT_TR(3, j, t);
             const int j0 = j * kMhaBlock;
             if (j0 + kMhaBlock - 1 > limit) {  // diagonal or tail block: mask keys beyond the row's last visible one
 #pragma unroll
@@ -392,7 +386,6 @@ mha_fwd_kernel(const __grid_constant__ CUtensorMap tmap_q, const __grid_constant
             tc_fence_before();
             __syncwarp();
             if (lane == 0) mbar_arrive(&p_full[t]);
-            if (threadIdx.x == t * 128) MLT_TR(4, j, t);
         }
 
         if (ok && Jt > 0) {
@@ -405,26 +398,27 @@ mha_fwd_kernel(const __grid_constant__ CUtensorMap tmap_q, const __grid_constant
                 // by row; then each warp writes its own 32 rows out row-major, 512 contiguous bytes per instruction.
                 constexpr int kRowChunks = D / 8;  // 16-byte chunks per row
                 uint8_t* stage_o = smem_q + t * L::kTileBytes;
-#pragma unroll 1
-                for (int q = 0; q < D / 16; ++q) {
-                    uint32_t o[16];
-                    tmem_ld_32x32b_x16(o_addr + q * 16, o);
+                {
+                    uint32_t o[D / 32][32];  // the whole row at once: one TMEM round trip instead of eight
+#pragma unroll
+                    for (int q = 0; q < D / 32; ++q) tmem_ld_32x32b_x32(o_addr + q * 32, o[q]);
                     tmem_wait_ld();
 #pragma unroll
-                    for (int v = 0; v < 2; ++v) {
+                    for (int k = 0; k < D / 8; ++k) {  // 16-byte chunks of the BF16 row
+                        const uint32_t* w = &o[k >> 2][(k & 3) * 8];
                         uint4 out;
-                        out.x = pack_bf16x2(__uint_as_float(o[v * 8 + 0]) * inv_l, __uint_as_float(o[v * 8 + 1]) * inv_l);
-                        out.y = pack_bf16x2(__uint_as_float(o[v * 8 + 2]) * inv_l, __uint_as_float(o[v * 8 + 3]) * inv_l);
-                        out.z = pack_bf16x2(__uint_as_float(o[v * 8 + 4]) * inv_l, __uint_as_float(o[v * 8 + 5]) * inv_l);
-                        out.w = pack_bf16x2(__uint_as_float(o[v * 8 + 6]) * inv_l, __uint_as_float(o[v * 8 + 7]) * inv_l);
-                        const int chunk = (q * 2 + v) ^ (row_in_tile & (kRowChunks - 1));
+                        out.x = pack_bf16x2(__uint_as_float(w[0]) * inv_l, __uint_as_float(w[1]) * inv_l);
+                        out.y = pack_bf16x2(__uint_as_float(w[2]) * inv_l, __uint_as_float(w[3]) * inv_l);
+                        out.z = pack_bf16x2(__uint_as_float(w[4]) * inv_l, __uint_as_float(w[5]) * inv_l);
+                        out.w = pack_bf16x2(__uint_as_float(w[6]) * inv_l, __uint_as_float(w[7]) * inv_l);
+                        const int chunk = k ^ (row_in_tile & (kRowChunks - 1));
                         *reinterpret_cast<uint4*>(stage_o + row_in_tile * (D * 2) + chunk * 16) = out;
                     }
                 }
                 __syncwarp();
                 constexpr int kRowsPerStore = 32 / kRowChunks;
                 __nv_bfloat16* obase = p.O + (static_cast<int64_t>(bh) * p.Nq + q_base + t * kMhaBlock) * D;
-#pragma unroll 4
+#pragma unroll
                 for (int r0 = 0; r0 < 32; r0 += kRowsPerStore) {
                     const int rr = quarter * 32 + r0 + lane / kRowChunks;
                     const int cc = lane % kRowChunks;
@@ -445,11 +439,6 @@ mha_fwd_kernel(const __grid_constant__ CUtensorMap tmap_q, const __grid_constant
         tmem_dealloc(tmem_base, 512);
     }
 }
-
-#ifdef MLT_TRACE
-static long long* g_trace_ptr = nullptr;
-extern "C" void mlt_debug_set_trace(long long* ptr) { g_trace_ptr = ptr; }
-#endif
 
 inline int mha_configure() {
     if (cudaFuncSetAttribute(mha_fwd_kernel<64>, cudaFuncAttributeMaxDynamicSharedMemorySize, MhaSmem<64>::kTotal) !=
@@ -474,9 +463,6 @@ inline int mha_launch(const CUtensorMap& tq, const CUtensorMap& tk, const CUtens
     p.scale = scale;
     p.num_pairs = (Nq + 2 * kMhaBlock - 1) / (2 * kMhaBlock);
     p.head_group = 8;
-#ifdef MLT_TRACE
-    p.trace = g_trace_ptr;
-#endif
     const int64_t items = static_cast<int64_t>(p.num_pairs) * p.BH;
     if (items > INT32_MAX) return 2;
     const int grid = static_cast<int>(items);
