@@ -49,6 +49,9 @@ def _load():
         lib.oracle_mha_fwd.argtypes = [p, p, p, p, p, p, i32, i32, i32, i32, i32, i32, ctypes.c_float, p, i64, i32]
         lib.oracle_mha_fwd.restype = i32
         lib.oracle_hardware_threads.restype = i32
+        lib.oracle_paged_attn_decode.argtypes = [p, p, p, p, p, p, p, i32, i32, i32, i32, i32, i32, i32,
+                                                 ctypes.c_float, i32]
+        lib.oracle_paged_attn_decode.restype = i32
         _lib = lib
     return _lib
 
@@ -121,3 +124,32 @@ def mha_fwd(Q: np.ndarray, K: np.ndarray, V: np.ndarray, *, causal: bool, scale,
         if rc != 0:
             raise ValueError("oracle_mha_fwd: invalid argument")
     return (O, LSE, P) if return_probs else (O, LSE)
+
+
+def paged_attn_decode(Q: np.ndarray, K_cache: np.ndarray, V_cache: np.ndarray, block_table: np.ndarray,
+                      seq_lens: np.ndarray, *, scale, nthreads: int = 0):
+    """Paged-attention decode in FP64 (Sec. 3.2 / 4.3): softmax attention of one query token per sequence over
+    the keys and values its block table points to.
+
+    Q: [num_seqs, H, D]; K_cache, V_cache: [num_blocks, H_kv, block_size, D] uint16 BF16 bits;
+    block_table: [num_seqs, max_blocks] int32; seq_lens: [num_seqs] int32.  Returns (O [num_seqs, H, D], LSE [num_seqs, H]).
+    """
+    Q = np.ascontiguousarray(_u16(Q))
+    K_cache = np.ascontiguousarray(_u16(K_cache))
+    V_cache = np.ascontiguousarray(_u16(V_cache))
+    block_table = np.ascontiguousarray(block_table, dtype=np.int32)
+    seq_lens = np.ascontiguousarray(seq_lens, dtype=np.int32)
+    S, H, D = Q.shape
+    NB, H_kv, bs, D2 = K_cache.shape
+    if D2 != D or V_cache.shape != K_cache.shape or block_table.shape[0] != S or seq_lens.shape != (S,):
+        raise ValueError("shape mismatch")
+    O = np.empty((S, H, D), dtype=np.float64)
+    LSE = np.empty((S, H), dtype=np.float64)
+    if S > 0:
+        rc = _load().oracle_paged_attn_decode(Q.ctypes.data, K_cache.ctypes.data, V_cache.ctypes.data,
+                                              block_table.ctypes.data, seq_lens.ctypes.data, O.ctypes.data,
+                                              LSE.ctypes.data, S, H, H_kv, D, bs, block_table.shape[1], NB,
+                                              float(np.float32(scale)), nthreads)
+        if rc != 0:
+            raise ValueError("oracle_paged_attn_decode: invalid argument")
+    return O, LSE

@@ -21,6 +21,8 @@
 // product of two BF16 values is exact in double, so the only rounding is in the
 // FP64 summations.  Outputs stay in FP64 (never rounded to BF16).
 //
+// Paged-attention decode (Sec. 3.2 / 4.3) is the same definition over keys gathered through a block table.
+//
 // Pins (see tests/test_oracle_*.py): identity / permutation / all-ones /
 // single-non-zero / K-split additivity / exact rational brute force for GEMM;
 // constant-K mean-of-V, causal row 0, Nk = 1, rows summing to one, key
@@ -161,6 +163,65 @@ int oracle_mha_fwd(const uint16_t* Q, const uint16_t* K, const uint16_t* V,
             double* p = P_out + r * Nk;
             for (int64_t j = 0; j < Nk; ++j) p[j] = j < visible ? s[j] / l : 0.0;
         }
+    });
+    return 0;
+}
+
+// Paged-attention decode (Sec. 3.2 and 4.3: one query token per sequence, the request's keys and values live
+// in fixed-size cache blocks reached through a block table; Listing 6 gives the per-block loop, which reaches
+// plain softmax attention over the sequence's tokens).  Written as the definition: gather the sequence's keys and
+// values through the table, then the same three passes as oracle_mha_fwd with a single query row.
+//
+// Q: [num_seqs, H, D]; K_cache, V_cache: [num_blocks, H_kv, block_size, D] (D fastest), BF16 bits.
+// block_table: [num_seqs, max_blocks] physical block of logical block b of a sequence; seq_lens: [num_seqs].
+// Query head h reads KV head h / (H / H_kv).  Token i of a sequence sits in logical block i / block_size at
+// offset i % block_size.  O_out: [num_seqs, H, D] doubles; LSE_out: [num_seqs, H] (natural log).
+// A sequence of length 0 gives O = 0 and LSE = -inf.  Returns 0, or 1 on a bad argument.
+int oracle_paged_attn_decode(const uint16_t* Q, const uint16_t* K_cache, const uint16_t* V_cache,
+                             const int32_t* block_table, const int32_t* seq_lens, double* O_out, double* LSE_out,
+                             int num_seqs, int H, int H_kv, int D, int block_size, int max_blocks, int num_blocks,
+                             float scale, int nthreads) {
+    if (num_seqs < 0 || H < 1 || H_kv < 1 || H % H_kv != 0 || D < 1 || block_size < 1 || max_blocks < 0) return 1;
+    for (int s = 0; s < num_seqs; ++s) {
+        if (seq_lens[s] < 0 || seq_lens[s] > static_cast<int64_t>(max_blocks) * block_size) return 1;
+        const int used = (seq_lens[s] + block_size - 1) / block_size;
+        for (int b = 0; b < used; ++b)
+            if (block_table[static_cast<int64_t>(s) * max_blocks + b] < 0 ||
+                block_table[static_cast<int64_t>(s) * max_blocks + b] >= num_blocks)
+                return 1;
+    }
+    const double sc = static_cast<double>(scale);
+    const int group = H / H_kv;
+    parallel_for(static_cast<int64_t>(num_seqs) * H, nthreads, [&](int64_t r) {
+        const int s = static_cast<int>(r / H), h = static_cast<int>(r % H), kvh = h / group;
+        const int len = seq_lens[s];
+        const uint16_t* q = Q + r * D;
+        auto row = [&](const uint16_t* cache, int i) {
+            const int64_t blk = block_table[static_cast<int64_t>(s) * max_blocks + i / block_size];
+            return cache + ((blk * H_kv + kvh) * block_size + i % block_size) * D;
+        };
+        std::vector<double> e(static_cast<size_t>(len));
+        double m = -std::numeric_limits<double>::infinity();
+        for (int i = 0; i < len; ++i) {  // pass 1: scores and their max
+            const uint16_t* k = row(K_cache, i);
+            double dot = 0.0;
+            for (int d = 0; d < D; ++d) dot += bf16_to_double(q[d]) * bf16_to_double(k[d]);
+            e[i] = sc * dot;
+            m = std::max(m, e[i]);
+        }
+        double l = 0.0;
+        for (int i = 0; i < len; ++i) {  // pass 2: exponentials and their sum
+            e[i] = std::exp(e[i] - m);
+            l += e[i];
+        }
+        double* o = O_out + r * D;
+        for (int d = 0; d < D; ++d) o[d] = 0.0;
+        for (int i = 0; i < len; ++i) {  // pass 3: weighted sum of the values
+            const uint16_t* v = row(V_cache, i);
+            const double p = e[i] / l;
+            for (int d = 0; d < D; ++d) o[d] += p * bf16_to_double(v[d]);
+        }
+        LSE_out[r] = len > 0 ? m + std::log(l) : -std::numeric_limits<double>::infinity();
     });
     return 0;
 }

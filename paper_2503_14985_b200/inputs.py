@@ -163,6 +163,52 @@ def mha_inputs(B: int, H: int, Nq: int, Nk: int, D: int, *, seed: int, outlier_p
     return one(TENSOR_Q, Nq, True), one(TENSOR_K, Nk, True), one(TENSOR_V, Nk, outlier_v)
 
 
+TENSOR_PAGED_Q, TENSOR_PAGED_K, TENSOR_PAGED_V = 3, 4, 5
+
+
+def paged_inputs(num_seqs: int, H: int, H_kv: int, D: int, block_size: int, *, seed: int, min_len: int, max_len: int,
+                 spare_blocks: int = 3):
+    """A paged KV cache with a mix of sequence lengths, and one query token per sequence.
+
+    Returns Q [num_seqs, H, D], K_cache and V_cache [num_blocks, H_kv, block_size, D] (uint16 BF16 bits, N(0,1)),
+    block_table [num_seqs, max_blocks] int32 (a seeded permutation scatters the logical blocks over the physical
+    pool; unused entries are -1) and seq_lens [num_seqs] int32 (seeded, uniform in [min_len, max_len]).
+    """
+    u = hash_u01(seed, TENSOR_PAGED_Q, 9, np.arange(num_seqs, dtype=np.uint64))
+    seq_lens = (min_len + np.floor(u * (max_len - min_len + 1))).astype(np.int32)
+    seq_lens = np.minimum(seq_lens, max_len)
+    blocks_per_seq = (seq_lens + block_size - 1) // block_size
+    max_blocks = int((max_len + block_size - 1) // block_size)
+    total = int(blocks_per_seq.sum())
+    num_blocks = total + spare_blocks
+    # seeded permutation of the physical pool: order blocks by a hash
+    order = np.argsort(hash_u01(seed, TENSOR_PAGED_K, 9, np.arange(num_blocks, dtype=np.uint64)), kind="stable")
+    block_table = np.full((num_seqs, max_blocks), -1, dtype=np.int32)
+    pos = 0
+    for s in range(num_seqs):
+        n = int(blocks_per_seq[s])
+        block_table[s, :n] = order[pos:pos + n]
+        pos += n
+    Q = matrix_bf16(num_seqs * H, D, seed=seed, tensor_id=TENSOR_PAGED_Q, kind="normal").reshape(num_seqs, H, D)
+    Kc = matrix_bf16(num_blocks * H_kv * block_size, D, seed=seed, tensor_id=TENSOR_PAGED_K, kind="normal")
+    Vc = matrix_bf16(num_blocks * H_kv * block_size, D, seed=seed, tensor_id=TENSOR_PAGED_V, kind="normal")
+    shape = (num_blocks, H_kv, block_size, D)
+    return Q, Kc.reshape(shape), Vc.reshape(shape), block_table, seq_lens
+
+
+PAGED_CONFIGS = {
+    # name: (num_seqs, H, H_kv, D, block_size, min_len, max_len, seed); the paper lists no decode shapes
+    "paged_s64h32d128_len1k-8k": (64, 32, 32, 128, 16, 1024, 8192, 7),
+    "paged_s8h32d128_len32k": (8, 32, 32, 128, 16, 30000, 32768, 8),
+    "paged_s128h32kv8d128_len2k-4k": (128, 32, 8, 128, 16, 2048, 4096, 9),
+}
+
+
+def paged_bytes(seq_lens, H_kv: int, D: int) -> float:
+    """Algorithmic HBM bytes of a decode step: every visible key and value read once (BF16)."""
+    return float(np.asarray(seq_lens, dtype=np.int64).sum()) * H_kv * D * 2 * 2
+
+
 GEMM_CONFIGS = {
     # name: (M, N, K, value kind, seed)
     "gemm_512": (512, 512, 512, "uniform", 0),
