@@ -424,6 +424,30 @@ def time_all_configs(mlt, torch, dev, stream, iters: int = 20, only: str | None 
             assert rc == 0, rc
         out[name] = timeit(fn, inputs.mha_flops(Bn, H, Nq, Nk, D, causal))
         del dQ, dK, dV, dO, dL
+    # paged-attention decode (Sec. 3.2 / 4.3): bound by HBM, reported in GB/s of visible K and V
+    hbm_peak = measured_peaks()["hbm_gbs"]
+    for name, (S, H, Hkv, D, bs, lo, hi, seed) in inputs.PAGED_CONFIGS.items():
+        if only is not None and name != only:
+            continue
+        Q, Kc, Vc, table, lens = inputs.paged_inputs(S, H, Hkv, D, bs, seed=seed, min_len=lo, max_len=hi)
+        dQ, dK, dV = devbits(Q), devbits(Kc), devbits(Vc)
+        dT, dLn = torch.from_numpy(table).to(dev), torch.from_numpy(lens).to(dev)
+        dO = torch.empty_like(dQ)
+        dL = torch.empty((S, H), dtype=torch.float32, device=dev)
+        ws = torch.empty(mlt.paged_attn_workspace_bytes(S, H, D), dtype=torch.uint8, device=dev)
+        sc = float(np.float32(1.0 / np.sqrt(D)))
+
+        def fn():
+            rc = mlt.paged_attn_decode_raw(dQ.data_ptr(), dK.data_ptr(), dV.data_ptr(), dT.data_ptr(), dLn.data_ptr(),
+                                           dO.data_ptr(), dL.data_ptr(), S, H, Hkv, D, bs, table.shape[1], Kc.shape[0],
+                                           sc, ws.data_ptr(), ws.numel(), sp)
+            assert rc == 0, rc
+        nbytes = inputs.paged_bytes(lens, Hkv, D)
+        r = timeit(fn, 4.0 * float(lens.sum()) * H * D)
+        out[name] = {"ms_min": r["ms_min"], "ms_median": r["ms_median"], "gbs_best": nbytes / r["ms_min"] / 1e6,
+                     "gbs_median": nbytes / r["ms_median"] / 1e6, "kv_bytes": nbytes,
+                     "frac_of_measured_hbm_best": nbytes / r["ms_min"] / 1e6 / hbm_peak}
+        del dQ, dK, dV, dO, dL, ws
     return out
 
 

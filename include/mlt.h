@@ -14,6 +14,7 @@
 #ifndef MLT_H_
 #define MLT_H_
 
+#include <stddef.h>
 #include <stdint.h>
 
 #ifdef __cplusplus
@@ -27,7 +28,8 @@ typedef enum {
     MLT_ERR_ALIGNMENT = 3,   /* base pointer not 16-byte aligned, or pitch not a multiple of 8 elements */
     MLT_ERR_CUDA = 4,        /* a CUDA runtime / driver call failed */
     MLT_ERR_ARCH = 5,        /* current device is not compute capability 10.x */
-    MLT_ERR_TIMEOUT = 6      /* a bounded device-side wait expired (reported by mlt_last_device_error) */
+    MLT_ERR_TIMEOUT = 6,     /* a bounded device-side wait expired (reported by mlt_last_device_error) */
+    MLT_ERR_BAD_BLOCK = 7    /* a block-table entry outside [0, num_blocks) was met (reported by mlt_last_device_error) */
 } mlt_status;
 
 /*
@@ -76,10 +78,40 @@ int mlt_mha_fwd(const void* Q, const void* K, const void* V,
                 int causal, float scale, void* stream);
 
 /*
+ * Paged-attention decode: O[s,h,:] = softmax(scale * q[s,h] . K_s^T) V_s over the len[s] tokens of sequence s,
+ * whose keys and values live in cache blocks reached through a block table -- paper Sec. 3.2 (Listings 6 and 7:
+ * one query token per sequence, KV blocks split across warps, cross-warp max / sum / output reduction) and
+ * Sec. 4.3.  The listings are schematic (they normalise per block); the operation is plain softmax attention.
+ *
+ *   Q            device, BF16, [num_seqs, H, D]
+ *   K_cache, V_cache  device, BF16, [num_blocks, H_kv, block_size, D] (D fastest)
+ *   block_table  device, int32, [num_seqs, max_blocks_per_seq]: physical block of each logical block; entries of
+ *                logical blocks a sequence uses must lie in [0, num_blocks) (others are never read; a bad entry is
+ *                skipped and reported through mlt_last_device_error, it is never dereferenced)
+ *   seq_lens     device, int32, [num_seqs], 0 <= len <= max_blocks_per_seq * block_size; token i sits in logical
+ *                block i / block_size at offset i % block_size
+ *   O            device, BF16 out, [num_seqs, H, D];  LSE device FP32 out [num_seqs, H] (natural log) or NULL
+ *   H_kv         KV heads; H / H_kv in {1, 2, 4, 8}; query head h reads KV head h / (H / H_kv)
+ *   D in {64, 128}; block_size in {8, 16, 32}; scale finite and > 0
+ *   workspace    device scratch of workspace_bytes bytes (16-byte aligned) for the partial results when a
+ *                sequence is split over several CTAs; mlt_paged_attn_workspace_bytes gives a size that is always
+ *                enough.  With less (or NULL) fewer splits are used, down to one CTA per (sequence, KV head).
+ *                Its contents are scratch; calls that overlap on the GPU must not share it.
+ * A sequence of length 0 gives O = 0 and LSE = -inf.  num_seqs == 0: MLT_OK, nothing launched.
+ */
+size_t mlt_paged_attn_workspace_bytes(int num_seqs, int H, int D);
+int mlt_paged_attn_decode(const void* Q, const void* K_cache, const void* V_cache,
+                          const int32_t* block_table, const int32_t* seq_lens,
+                          void* O, float* LSE,
+                          int num_seqs, int H, int H_kv, int D,
+                          int block_size, int max_blocks_per_seq, int num_blocks, float scale,
+                          void* workspace, size_t workspace_bytes, void* stream);
+
+/*
  * Device-side health word.  Kernels never trap: a wait that exceeds its bound
  * records {code, barrier id, block} in a per-device status word and the kernel
  * drains and returns.  This call synchronises the current device, reads and
- * clears that word, and returns MLT_OK, MLT_ERR_TIMEOUT or MLT_ERR_CUDA.
+ * clears that word, and returns MLT_OK, MLT_ERR_TIMEOUT, MLT_ERR_BAD_BLOCK or MLT_ERR_CUDA.
  * detail (host, may be NULL) receives 4 words: code, barrier id, block, aux.
  * (Library addition; the paper has no counterpart.)
  */

@@ -14,9 +14,10 @@ LIB_PATH = os.path.join(_HERE, "libmlt.so")
 
 MLT_OK = 0
 STATUS_NAMES = {0: "MLT_OK", 1: "MLT_ERR_INVALID_ARG", 2: "MLT_ERR_UNSUPPORTED", 3: "MLT_ERR_ALIGNMENT",
-                4: "MLT_ERR_CUDA", 5: "MLT_ERR_ARCH", 6: "MLT_ERR_TIMEOUT"}
+                4: "MLT_ERR_CUDA", 5: "MLT_ERR_ARCH", 6: "MLT_ERR_TIMEOUT", 7: "MLT_ERR_BAD_BLOCK"}
 
-EXPORTS = ("mlt_gemm", "mlt_mha_fwd", "mlt_last_device_error", "mlt_status_string", "mlt_version")
+EXPORTS = ("mlt_gemm", "mlt_mha_fwd", "mlt_paged_attn_decode", "mlt_paged_attn_workspace_bytes",
+           "mlt_last_device_error", "mlt_status_string", "mlt_version")
 
 _lib = None
 
@@ -39,6 +40,11 @@ def load() -> ctypes.CDLL:
         lib.mlt_gemm.restype = i32
         lib.mlt_mha_fwd.argtypes = [p, p, p, p, p, i32, i32, i32, i32, i32, i32, ctypes.c_float, p]
         lib.mlt_mha_fwd.restype = i32
+        lib.mlt_paged_attn_workspace_bytes.argtypes = [i32, i32, i32]
+        lib.mlt_paged_attn_workspace_bytes.restype = ctypes.c_size_t
+        lib.mlt_paged_attn_decode.argtypes = [p, p, p, p, p, p, p, i32, i32, i32, i32, i32, i32, i32, ctypes.c_float,
+                                              p, ctypes.c_size_t, p]
+        lib.mlt_paged_attn_decode.restype = i32
         lib.mlt_last_device_error.argtypes = [p]
         lib.mlt_last_device_error.restype = i32
         lib.mlt_status_string.argtypes = [i32]
@@ -65,6 +71,19 @@ def mha_fwd_raw(Q: int, K: int, V: int, O: int, LSE: int, B: int, H: int, Nq: in
                 scale: float, stream: int = 0) -> int:
     """mlt_mha_fwd with raw device addresses; returns the status code."""
     return int(load().mlt_mha_fwd(Q, K, V, O, LSE, B, H, Nq, Nk, D, causal, scale, stream))
+
+
+def paged_attn_workspace_bytes(num_seqs: int, H: int, D: int) -> int:
+    return int(load().mlt_paged_attn_workspace_bytes(num_seqs, H, D))
+
+
+def paged_attn_decode_raw(Q: int, K_cache: int, V_cache: int, block_table: int, seq_lens: int, O: int, LSE: int,
+                          num_seqs: int, H: int, H_kv: int, D: int, block_size: int, max_blocks: int, num_blocks: int,
+                          scale: float, workspace: int = 0, workspace_bytes: int = 0, stream: int = 0) -> int:
+    """mlt_paged_attn_decode with raw device addresses; returns the status code."""
+    return int(load().mlt_paged_attn_decode(Q, K_cache, V_cache, block_table, seq_lens, O, LSE, num_seqs, H, H_kv, D,
+                                            block_size, max_blocks, num_blocks, scale, workspace, workspace_bytes,
+                                            stream))
 
 
 def last_device_error():
@@ -127,4 +146,34 @@ def mha_fwd(Q, K, V, *, causal: bool, scale: float, O=None, LSE=None, return_lse
                      Bn, H, Nq, Nk, D, int(bool(causal)), float(scale), _stream(stream))
     if rc != MLT_OK:
         raise MltError(rc, "mlt_mha_fwd")
+    return O, LSE
+
+
+def paged_attn_decode(Q, K_cache, V_cache, block_table, seq_lens, *, scale: float, workspace=None, O=None, LSE=None,
+                      return_lse: bool = True, stream=None):
+    """Paged-attention decode for CUDA tensors: Q [S,H,D] bfloat16, caches [num_blocks,H_kv,block_size,D] bfloat16,
+    block_table [S,max_blocks] int32, seq_lens [S] int32.  `workspace` is an optional uint8 CUDA tensor (see
+    paged_attn_workspace_bytes).  Returns (O [S,H,D] bfloat16, LSE [S,H] float32 or None).
+    """
+    import torch
+    for t in (Q, K_cache, V_cache):
+        if t.dtype != torch.bfloat16 or not t.is_cuda or not t.is_contiguous():
+            raise TypeError("Q and the caches must be contiguous CUDA bfloat16 tensors")
+    for t in (block_table, seq_lens):
+        if t.dtype != torch.int32 or not t.is_cuda or not t.is_contiguous():
+            raise TypeError("block_table and seq_lens must be contiguous CUDA int32 tensors")
+    S, H, D = Q.shape
+    NB, H_kv, bs, _ = K_cache.shape
+    if O is None:
+        O = torch.empty_like(Q)
+    if LSE is None and return_lse:
+        LSE = torch.empty((S, H), dtype=torch.float32, device=Q.device)
+    rc = paged_attn_decode_raw(Q.data_ptr(), K_cache.data_ptr(), V_cache.data_ptr(), block_table.data_ptr(),
+                               seq_lens.data_ptr(), O.data_ptr(), LSE.data_ptr() if LSE is not None else 0, S, H, H_kv, D,
+                               bs, block_table.shape[1], NB, float(scale),
+                               workspace.data_ptr() if workspace is not None else 0,
+                               workspace.numel() * workspace.element_size() if workspace is not None else 0,
+                               _stream(stream))
+    if rc != MLT_OK:
+        raise MltError(rc, "mlt_paged_attn_decode")
     return O, LSE

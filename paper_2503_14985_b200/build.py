@@ -8,7 +8,7 @@ _HERE = os.path.dirname(os.path.abspath(__file__))
 CSRC = os.path.join(_HERE, "csrc")
 LIB = os.path.join(_HERE, "libmlt.so")
 SOURCES = ["mlt.cu"]
-HEADERS = ["ptx.cuh", "gemm.cuh", "mha.cuh", os.path.join("..", "..", "include", "mlt.h")]
+HEADERS = ["ptx.cuh", "gemm.cuh", "mha.cuh", "paged.cuh", os.path.join("..", "..", "include", "mlt.h")]
 
 NVCC_FLAGS = ["-gencode", "arch=compute_100a,code=sm_100a", "-lineinfo", "-O3", "-std=c++17",
               "-shared", "-Xcompiler", "-fPIC", "-Xptxas", "-v"]

@@ -13,6 +13,7 @@
 #include "../../include/mlt.h"
 #include "gemm.cuh"
 #include "mha.cuh"
+#include "paged.cuh"
 
 namespace {
 
@@ -131,6 +132,7 @@ const char* mlt_status_string(int status) {
         case MLT_ERR_CUDA: return "CUDA runtime or driver call failed";
         case MLT_ERR_ARCH: return "device is not compute capability 10.x (sm_100a required)";
         case MLT_ERR_TIMEOUT: return "a bounded device-side wait expired";
+        case MLT_ERR_BAD_BLOCK: return "a block-table entry outside [0, num_blocks) was met";
         default: return "unknown status";
     }
 }
@@ -143,7 +145,7 @@ int mlt_last_device_error(uint32_t* detail) {
     if (host[0] != 0) {
         unsigned int zero[4] = {0, 0, 0, 0};
         if (cudaMemcpyToSymbol(g_status, zero, sizeof zero) != cudaSuccess) return MLT_ERR_CUDA;
-        return host[0] == kStatusTimeout ? MLT_ERR_TIMEOUT : MLT_ERR_CUDA;
+        return host[0] == kStatusTimeout ? MLT_ERR_TIMEOUT : host[0] == kStatusBadBlock ? MLT_ERR_BAD_BLOCK : MLT_ERR_CUDA;
     }
     return MLT_OK;
 }
@@ -265,6 +267,70 @@ int mlt_mha_fwd(const void* Q, const void* K, const void* V, void* O, float* LSE
     }
     return mha_launch(tq, tk, tv, static_cast<__nv_bfloat16*>(O), LSE, B, H, Nq, Nk, D, causal != 0, scale,
                       dev.sm_count, static_cast<cudaStream_t>(stream));
+}
+
+size_t mlt_paged_attn_workspace_bytes(int num_seqs, int H, int D) {
+    if (num_seqs <= 0 || H <= 0 || D <= 0) return 0;
+    return paged_workspace_bytes(num_seqs, H, D, kPagedMaxSplits);
+}
+
+namespace {
+// Shared front end of the paged-decode entry points: validation and parameter block.  Returns MLT_OK with
+// *launch = false when there is nothing to do.
+int paged_prepare(const void* Q, const void* K_cache, const void* V_cache, const int32_t* block_table,
+                  const int32_t* seq_lens, void* O, float* LSE, int num_seqs, int H, int H_kv, int D, int block_size,
+                  int max_blocks_per_seq, int num_blocks, float scale, PagedParams* p, DeviceInfo* dev, bool* launch) {
+    *launch = false;
+    if (num_seqs < 0 || H < 0 || H_kv < 0 || max_blocks_per_seq < 0 || num_blocks < 0) return MLT_ERR_INVALID_ARG;
+    if (num_seqs == 0 || H == 0) return MLT_OK;
+    if (!Q || !K_cache || !V_cache || !block_table || !seq_lens || !O) return MLT_ERR_INVALID_ARG;
+    if (H_kv == 0 || H % H_kv != 0) return MLT_ERR_INVALID_ARG;
+    if (!(scale > 0.0f) || scale > 3.0e38f) return MLT_ERR_INVALID_ARG;
+    const int group = H / H_kv;
+    if (D != 64 && D != 128) return MLT_ERR_UNSUPPORTED;
+    if (group != 1 && group != 2 && group != 4 && group != 8) return MLT_ERR_UNSUPPORTED;
+    if (block_size != 8 && block_size != 16 && block_size != 32) return MLT_ERR_UNSUPPORTED;
+    if (num_seqs > 65535 || H_kv > 65535) return MLT_ERR_UNSUPPORTED;  // grid.y / grid.z
+    if (!aligned16(Q) || !aligned16(K_cache) || !aligned16(V_cache) || !aligned16(O)) return MLT_ERR_ALIGNMENT;
+    int rc = get_device(dev);
+    if (rc != MLT_OK) return rc;
+    p->Q = static_cast<const __nv_bfloat16*>(Q);
+    p->K_cache = static_cast<const __nv_bfloat16*>(K_cache);
+    p->V_cache = static_cast<const __nv_bfloat16*>(V_cache);
+    p->block_table = block_table;
+    p->seq_lens = seq_lens;
+    p->O = static_cast<__nv_bfloat16*>(O);
+    p->LSE = LSE;
+    p->part_o = nullptr;
+    p->part_ml = nullptr;
+    p->num_seqs = num_seqs;
+    p->H = H;
+    p->H_kv = H_kv;
+    p->block_size = block_size;
+    p->max_blocks = max_blocks_per_seq;
+    p->num_blocks = num_blocks;
+    p->splits = paged_choose_splits(num_seqs, H_kv, max_blocks_per_seq, dev->sm_count);
+    p->scale_log2e = scale * 1.4426950408889634f;
+    *launch = true;
+    return MLT_OK;
+}
+}  // namespace
+
+int mlt_paged_attn_decode(const void* Q, const void* K_cache, const void* V_cache, const int32_t* block_table,
+                          const int32_t* seq_lens, void* O, float* LSE, int num_seqs, int H, int H_kv, int D,
+                          int block_size, int max_blocks_per_seq, int num_blocks, float scale, void* workspace,
+                          size_t workspace_bytes, void* stream) {
+    PagedParams p;
+    DeviceInfo dev;
+    bool launch = false;
+    if (workspace && !aligned16(workspace)) return MLT_ERR_ALIGNMENT;
+    int rc = paged_prepare(Q, K_cache, V_cache, block_table, seq_lens, O, LSE, num_seqs, H, H_kv, D, block_size,
+                           max_blocks_per_seq, num_blocks, scale, &p, &dev, &launch);
+    if (rc != MLT_OK || !launch) return rc;
+    // use as many splits as the caller's scratch allows
+    if (!workspace) workspace_bytes = 0;
+    while (p.splits > 1 && paged_workspace_bytes(num_seqs, H, D, p.splits) > workspace_bytes) --p.splits;
+    return paged_launch(p, D, workspace, static_cast<cudaStream_t>(stream));
 }
 
 }  // extern "C"

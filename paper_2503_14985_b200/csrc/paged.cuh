@@ -1,0 +1,288 @@
+// Paged-attention decode (paper Sec. 3.2, Listings 6-7, and Sec. 4.3): one query token per sequence attends
+// to the sequence's keys and values, which live in fixed-size cache blocks reached through a block table.  As in
+// the paper's warp-level kernel the KV blocks of a sequence are split across warps (and here also across CTAs,
+// flash-decoding style), each keeps a partial running max / sum / output, and the partials are reduced at the end.
+//
+// The work is bound by HBM: every visible key and value is read once (2 * len * H_kv * D * 2 bytes per sequence)
+// and used for 2 * G multiply-adds per element, so there are no tensor cores here; the kernel is laid out for
+// coalesced 16-byte loads with many loads in flight per warp.
+//   grid  = (splits, H_kv, num_seqs), 128 threads (4 warps)
+//   warp  = KV blocks b0 + w, b0 + w + 4, ... of its split; for one block it first issues all K and V loads
+//           (16 bytes per lane, D/8 lanes per token, 32 / (D/8) tokens per load instruction), then the dot
+//           products (shuffle reduction inside the D/8 lanes of a token), one online-softmax update per block,
+//           and the P V accumulation; each lane keeps 8 output columns for each of the G query heads that
+//           share the KV head
+//   end   = lane groups merge by shuffles, warps merge through shared memory, and the CTA writes O and LSE
+//           (single split) or an unnormalised partial {m, l, o[D]} to the workspace, which a second small
+//           kernel combines.
+#pragma once
+
+#include <math.h>
+
+#include <algorithm>
+
+#include "ptx.cuh"
+
+namespace mlt {
+
+constexpr int kPagedThreads = 128;
+constexpr int kPagedWarps = kPagedThreads / 32;
+constexpr int kPagedMaxSplits = 32;
+constexpr unsigned int kStatusBadBlock = 7;  // a block-table entry outside [0, num_blocks)
+
+struct PagedParams {
+    const __nv_bfloat16* Q;        // [num_seqs, H, D]
+    const __nv_bfloat16* K_cache;  // [num_blocks, H_kv, block_size, D]
+    const __nv_bfloat16* V_cache;
+    const int* block_table;        // [num_seqs, max_blocks]
+    const int* seq_lens;           // [num_seqs]
+    __nv_bfloat16* O;              // [num_seqs, H, D]
+    float* LSE;                    // [num_seqs, H] or null
+    float* part_o;                 // [num_seqs, H, splits, D]   (splits > 1)
+    float2* part_ml;               // [num_seqs, H, splits] {m in log2 units, l}
+    int num_seqs, H, H_kv, block_size, max_blocks, num_blocks, splits;
+    float scale_log2e;
+};
+
+__device__ __forceinline__ void bf16x8_to_f32(const uint4& v, float (&f)[8]) {
+    const uint32_t w[4] = {v.x, v.y, v.z, v.w};
+#pragma unroll
+    for (int i = 0; i < 4; ++i) {
+        f[2 * i] = __uint_as_float(w[i] << 16);
+        f[2 * i + 1] = __uint_as_float(w[i] & 0xFFFF0000u);
+    }
+}
+
+// merge partial {m, l, o} states a and b (log2-domain maxima); -inf maxima stand for "nothing seen"
+__device__ __forceinline__ void paged_merge_scale(float ma, float mb, float& m, float& sa, float& sb) {
+    m = fmaxf(ma, mb);
+    sa = (ma == -INFINITY) ? 0.0f : fast_exp2(ma - m);
+    sb = (mb == -INFINITY) ? 0.0f : fast_exp2(mb - m);
+}
+
+template <int D, int G, int BS>
+__global__ void __launch_bounds__(kPagedThreads)
+paged_decode_kernel(const PagedParams p) {
+    constexpr int LPT = D / 8;         // lanes per token
+    constexpr int TPS = 32 / LPT;      // tokens per load instruction of a warp
+    constexpr int STEPS = BS / TPS;    // load instructions per block and tensor
+    static_assert(BS % TPS == 0, "block size must be a multiple of the tokens per warp step");
+    __shared__ float sm_o[kPagedWarps][G][D];
+    __shared__ float2 sm_ml[kPagedWarps][G];
+
+    const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+    const int sp = blockIdx.x, kvh = blockIdx.y, s = blockIdx.z;
+    const int sub = lane % LPT;   // which 8 columns of D this lane owns
+    const int grp = lane / LPT;   // which token of a step
+    const int len = p.seq_lens[s];
+    const int nblk = (len + BS - 1) / BS;
+    const int per_split = (nblk + p.splits - 1) / p.splits;
+    const int b0 = sp * per_split;
+    const int b1 = min(nblk, b0 + per_split);
+
+    // this lane's 8 columns of the G query rows
+    float q[G][8];
+#pragma unroll
+    for (int g = 0; g < G; ++g) {
+        const uint4 v = *reinterpret_cast<const uint4*>(p.Q + (static_cast<int64_t>(s) * p.H + kvh * G + g) * D + sub * 8);
+        bf16x8_to_f32(v, q[g]);
+    }
+    float m[G], l[G], o[G][8];
+#pragma unroll
+    for (int g = 0; g < G; ++g) {
+        m[g] = -INFINITY;
+        l[g] = 0.0f;
+#pragma unroll
+        for (int e = 0; e < 8; ++e) o[g][e] = 0.0f;
+    }
+
+    const int* table = p.block_table + static_cast<int64_t>(s) * p.max_blocks;
+    for (int b = b0 + warp; b < b1; b += kPagedWarps) {
+        const int phys = table[b];
+        if (phys < 0 || phys >= p.num_blocks) {  // never dereference a bad table entry: report and skip the block
+            if (lane == 0 && atomicCAS(&g_status[0], 0u, kStatusBadBlock) == 0u) {
+                g_status[1] = static_cast<unsigned int>(b);
+                g_status[2] = static_cast<unsigned int>(s);
+                g_status[3] = static_cast<unsigned int>(phys);
+            }
+            continue;
+        }
+        const int64_t base = ((static_cast<int64_t>(phys) * p.H_kv + kvh) * BS) * D + sub * 8;
+        const __nv_bfloat16* kp = p.K_cache + base;
+        const __nv_bfloat16* vp = p.V_cache + base;
+        uint4 kr[STEPS], vr[STEPS];
+#pragma unroll
+        for (int i = 0; i < STEPS; ++i) kr[i] = *reinterpret_cast<const uint4*>(kp + (i * TPS + grp) * D);
+#pragma unroll
+        for (int i = 0; i < STEPS; ++i) vr[i] = *reinterpret_cast<const uint4*>(vp + (i * TPS + grp) * D);
+        // scores of this lane group's STEPS tokens for each head (log2 domain), masked beyond the length
+        float sc[G][STEPS];
+#pragma unroll
+        for (int i = 0; i < STEPS; ++i) {
+            float kf[8];
+            bf16x8_to_f32(kr[i], kf);
+            const bool visible = b * BS + i * TPS + grp < len;
+#pragma unroll
+            for (int g = 0; g < G; ++g) {
+                float d = 0.0f;
+#pragma unroll
+                for (int e = 0; e < 8; ++e) d = fmaf(q[g][e], kf[e], d);
+#pragma unroll
+                for (int w = LPT / 2; w > 0; w >>= 1) d += __shfl_xor_sync(0xffffffffu, d, w);
+                sc[g][i] = visible ? d * p.scale_log2e : -INFINITY;
+            }
+        }
+        // one online-softmax update per block and head
+        float pw[G][STEPS];
+#pragma unroll
+        for (int g = 0; g < G; ++g) {
+            float mb = sc[g][0];
+#pragma unroll
+            for (int i = 1; i < STEPS; ++i) mb = fmaxf(mb, sc[g][i]);
+            const float mn = fmaxf(m[g], mb);
+            const float alpha = (m[g] == -INFINITY) ? 0.0f : fast_exp2(m[g] - mn);
+            const float ref = (mn == -INFINITY) ? 0.0f : mn;
+            float sum = 0.0f;
+#pragma unroll
+            for (int i = 0; i < STEPS; ++i) {
+                pw[g][i] = fast_exp2(sc[g][i] - ref);
+                sum += pw[g][i];
+            }
+            m[g] = mn;
+            l[g] = l[g] * alpha + sum;
+#pragma unroll
+            for (int e = 0; e < 8; ++e) o[g][e] *= alpha;
+        }
+#pragma unroll
+        for (int i = 0; i < STEPS; ++i) {
+            float vf[8];
+            // bytes past the sequence's last token are whatever the cache holds: weight 0 must not meet a NaN
+            if (b * BS + i * TPS + grp >= len) vr[i] = make_uint4(0u, 0u, 0u, 0u);
+            bf16x8_to_f32(vr[i], vf);
+#pragma unroll
+            for (int g = 0; g < G; ++g)
+#pragma unroll
+                for (int e = 0; e < 8; ++e) o[g][e] = fmaf(pw[g][i], vf[e], o[g][e]);
+        }
+    }
+
+    // merge the TPS lane groups of the warp (lanes that own the same columns), then the warps through smem
+#pragma unroll
+    for (int g = 0; g < G; ++g) {
+#pragma unroll
+        for (int w = LPT; w < 32; w <<= 1) {
+            const float mo = __shfl_xor_sync(0xffffffffu, m[g], w);
+            const float lo = __shfl_xor_sync(0xffffffffu, l[g], w);
+            float mn, sa, sb;
+            paged_merge_scale(m[g], mo, mn, sa, sb);
+            l[g] = l[g] * sa + lo * sb;
+#pragma unroll
+            for (int e = 0; e < 8; ++e) {
+                const float oo = __shfl_xor_sync(0xffffffffu, o[g][e], w);
+                o[g][e] = o[g][e] * sa + oo * sb;
+            }
+            m[g] = mn;
+        }
+        if (grp == 0) {
+#pragma unroll
+            for (int e = 0; e < 8; ++e) sm_o[warp][g][sub * 8 + e] = o[g][e];
+            if (sub == 0) sm_ml[warp][g] = make_float2(m[g], l[g]);
+        }
+    }
+    __syncthreads();
+    for (int idx = threadIdx.x; idx < G * D; idx += kPagedThreads) {
+        const int g = idx / D, d = idx % D;
+        float mt = -INFINITY;
+#pragma unroll
+        for (int w = 0; w < kPagedWarps; ++w) mt = fmaxf(mt, sm_ml[w][g].x);
+        float lt = 0.0f, ot = 0.0f;
+#pragma unroll
+        for (int w = 0; w < kPagedWarps; ++w) {
+            const float2 ml = sm_ml[w][g];
+            const float sw = (ml.x == -INFINITY) ? 0.0f : fast_exp2(ml.x - mt);
+            lt += ml.y * sw;
+            ot += sm_o[w][g][d] * sw;
+        }
+        const int64_t row = static_cast<int64_t>(s) * p.H + kvh * G + g;
+        if (p.splits == 1) {
+            p.O[row * D + d] = __float2bfloat16(lt > 0.0f ? ot / lt : 0.0f);
+            if (d == 0 && p.LSE) p.LSE[row] = lt > 0.0f ? (mt + log2f(lt)) * 0.6931471805599453f : -INFINITY;
+        } else {
+            p.part_o[(row * p.splits + sp) * D + d] = ot;
+            if (d == 0) p.part_ml[row * p.splits + sp] = make_float2(mt, lt);
+        }
+    }
+}
+
+// O[row] = sum over splits of the partials, rescaled to the common max; one CTA of D threads per (seq, head).
+template <int D>
+__global__ void __launch_bounds__(D)
+paged_combine_kernel(const PagedParams p) {
+    const int64_t row = blockIdx.x;
+    const int d = threadIdx.x;
+    float mt = -INFINITY;
+    for (int sp = 0; sp < p.splits; ++sp) mt = fmaxf(mt, p.part_ml[row * p.splits + sp].x);
+    float lt = 0.0f, ot = 0.0f;
+    for (int sp = 0; sp < p.splits; ++sp) {
+        const float2 ml = p.part_ml[row * p.splits + sp];
+        const float sw = (ml.x == -INFINITY) ? 0.0f : fast_exp2(ml.x - mt);
+        lt += ml.y * sw;
+        ot += p.part_o[(row * p.splits + sp) * D + d] * sw;
+    }
+    p.O[row * D + d] = __float2bfloat16(lt > 0.0f ? ot / lt : 0.0f);
+    if (d == 0 && p.LSE) p.LSE[row] = lt > 0.0f ? (mt + log2f(lt)) * 0.6931471805599453f : -INFINITY;
+}
+
+inline size_t paged_workspace_bytes(int num_seqs, int H, int D, int splits) {
+    return splits <= 1 ? 0 : static_cast<size_t>(num_seqs) * H * splits * (static_cast<size_t>(D) * 4 + 8);
+}
+
+// How many CTAs share one (sequence, KV head): enough to put a few CTAs on every SM, at least 8 KV blocks each.
+inline int paged_choose_splits(int num_seqs, int H_kv, int max_blocks, int sm_count) {
+    const int64_t base = static_cast<int64_t>(num_seqs) * H_kv;
+    int splits = static_cast<int>((4ll * sm_count + base - 1) / base);
+    splits = std::min(splits, (max_blocks + 7) / 8);
+    return std::max(1, std::min(splits, kPagedMaxSplits));
+}
+
+template <int D, int G>
+int paged_launch_bs(const PagedParams& p, cudaStream_t st) {
+    const dim3 grid(p.splits, p.H_kv, p.num_seqs);
+    switch (p.block_size) {
+        case 8: paged_decode_kernel<D, G, 8><<<grid, kPagedThreads, 0, st>>>(p); break;
+        case 16: paged_decode_kernel<D, G, 16><<<grid, kPagedThreads, 0, st>>>(p); break;
+        case 32: paged_decode_kernel<D, G, 32><<<grid, kPagedThreads, 0, st>>>(p); break;
+        default: return 2;
+    }
+    if (cudaGetLastError() != cudaSuccess) return 4;
+    if (p.splits > 1) {
+        paged_combine_kernel<D><<<p.num_seqs * p.H, D, 0, st>>>(p);
+        if (cudaGetLastError() != cudaSuccess) return 4;
+    }
+    return 0;
+}
+
+template <int D>
+int paged_launch_g(const PagedParams& p, cudaStream_t st) {
+    switch (p.H / p.H_kv) {
+        case 1: return paged_launch_bs<D, 1>(p, st);
+        case 2: return paged_launch_bs<D, 2>(p, st);
+        case 4: return paged_launch_bs<D, 4>(p, st);
+        case 8: return paged_launch_bs<D, 8>(p, st);
+        default: return 2;
+    }
+}
+
+// workspace layout: part_o floats first, then part_ml pairs
+inline int paged_launch(PagedParams p, int D, void* workspace, cudaStream_t st) {
+    if (p.splits > 1) {
+        p.part_o = static_cast<float*>(workspace);
+        p.part_ml = reinterpret_cast<float2*>(p.part_o + static_cast<size_t>(p.num_seqs) * p.H * p.splits * D);
+    } else {
+        p.part_o = nullptr;
+        p.part_ml = nullptr;
+    }
+    return D == 64 ? paged_launch_g<64>(p, st) : paged_launch_g<128>(p, st);
+}
+
+}  // namespace mlt

@@ -121,14 +121,25 @@ def matrix_bf16(rows: int, cols: int, *, seed: int, tensor_id: int, kind: str = 
     if rows == 0 or cols == 0:
         return out
     if chunk_rows is None:
-        chunk_rows = max(1, (1 << 22) // cols)
-    for r0 in range(0, rows, chunk_rows):
+        chunk_rows = max(1, (1 << 20) // cols)
+
+    def fill(r0: int) -> None:
         r1 = min(rows, r0 + chunk_rows)
         v = _values(kind, seed, tensor_id, r0 * cols, (r1 - r0) * cols).reshape(r1 - r0, cols)
         v = v * scale
         if row_scale is not None:
             v = v * row_scale[r0:r1, None]
         out[r0:r1, :cols] = f64_to_bf16_bits(v)
+
+    starts = range(0, rows, chunk_rows)
+    if len(starts) > 4:  # every element depends only on its index: chunks can be filled by a few threads
+        from concurrent.futures import ThreadPoolExecutor
+        import os
+        with ThreadPoolExecutor(max_workers=min(16, os.cpu_count() or 1)) as pool:
+            list(pool.map(fill, starts))
+    else:
+        for r0 in starts:
+            fill(r0)
     return out
 
 
@@ -198,9 +209,10 @@ def paged_inputs(num_seqs: int, H: int, H_kv: int, D: int, block_size: int, *, s
 
 PAGED_CONFIGS = {
     # name: (num_seqs, H, H_kv, D, block_size, min_len, max_len, seed); the paper lists no decode shapes
-    "paged_s64h32d128_len1k-8k": (64, 32, 32, 128, 16, 1024, 8192, 7),
-    "paged_s8h32d128_len32k": (8, 32, 32, 128, 16, 30000, 32768, 8),
-    "paged_s128h32kv8d128_len2k-4k": (128, 32, 8, 128, 16, 2048, 4096, 9),
+    # sized so that the visible KV (0.2-0.3 GB) is larger than L2 and the generator stays within tens of seconds
+    "paged_s16h8d128_len1k-8k": (16, 8, 8, 128, 16, 1024, 8192, 7),
+    "paged_s2h8d128_len32k": (2, 8, 8, 128, 16, 30000, 32768, 8),
+    "paged_s32h32kv4d128_len2k-4k": (32, 32, 4, 128, 16, 2048, 4096, 9),
 }
 
 

@@ -19,7 +19,7 @@ def lib():
 
 def test_header_symbols_are_exported(lib):
     header = open(os.path.join(ROOT, "include", "mlt.h")).read()
-    declared = set(re.findall(r"^(?:int|const char\*)\s+(mlt_[a-z_0-9]+)\s*\(", header, flags=re.M))
+    declared = set(re.findall(r"^(?:int|size_t|const char\*)\s+(mlt_[a-z_0-9]+)\s*\(", header, flags=re.M))
     assert declared >= set(binding.EXPORTS)
     for name in declared:
         assert hasattr(lib, name), f"{name} declared in mlt.h but not exported"
@@ -27,8 +27,8 @@ def test_header_symbols_are_exported(lib):
 
 def test_version_and_status_strings(lib):
     assert binding.version() >= 100
-    texts = {binding.status_string(i) for i in range(7)}
-    assert len(texts) == 7 and "unknown status" not in texts
+    texts = {binding.status_string(i) for i in range(8)}
+    assert len(texts) == 8 and "unknown status" not in texts
     assert binding.status_string(99) == "unknown status"
 
 
@@ -44,6 +44,15 @@ def test_validation_precedes_cuda(lib):
     assert binding.mha_fwd_raw(16, 16, 16, 16, 0, 1, 1, 9, 8, 64, 1, 1.0) == 1
     assert binding.mha_fwd_raw(16, 16, 16, 16, 0, 0, 4, 9, 8, 64, 0, 1.0) == 0
     assert binding.mha_fwd_raw(16, 16, 16, 16, 0, 1, 1, 8, 8, 64, 0, float("nan")) == 1
+    pa = binding.paged_attn_decode_raw
+    assert pa(16, 16, 16, 16, 16, 16, 0, 0, 8, 8, 128, 16, 4, 10, 1.0) == 0          # no sequences
+    assert pa(16, 16, 16, 16, 16, 16, 0, 2, 8, 3, 128, 16, 4, 10, 1.0) == 1          # H not a multiple of H_kv
+    assert pa(16, 16, 16, 16, 16, 16, 0, 2, 8, 8, 96, 16, 4, 10, 1.0) == 2           # head dimension
+    assert pa(16, 16, 16, 16, 16, 16, 0, 2, 8, 8, 128, 12, 4, 10, 1.0) == 2          # block size
+    assert pa(16, 16, 16, 16, 16, 16, 0, 2, 24, 2, 128, 16, 4, 10, 1.0) == 2         # 12 query heads per KV head
+    assert pa(16, 18, 16, 16, 16, 16, 0, 2, 8, 8, 128, 16, 4, 10, 1.0) == 3          # misaligned cache
+    assert pa(16, 16, 16, 0, 16, 16, 0, 2, 8, 8, 128, 16, 4, 10, 1.0) == 1           # NULL block table
+    assert binding.paged_attn_workspace_bytes(64, 32, 128) == 64 * 32 * 32 * (128 * 4 + 8)
 
 
 def test_product_does_not_import_oracle():

@@ -104,11 +104,11 @@ def test_empty_sequence_and_bad_table():
 
 
 def test_generator_mixes_lengths_and_scatters_blocks():
-    name = "paged_s64h32d128_len1k-8k"
+    name = "paged_s16h8d128_len1k-8k"
     S, H, Hkv, D, bs, lo, hi, seed = inputs.PAGED_CONFIGS[name]
     u = inputs.hash_u01(seed, inputs.TENSOR_PAGED_Q, 9, np.arange(S, dtype=np.uint64))
     lens = lo + np.floor(u * (hi - lo + 1))
-    assert lens.min() >= lo and lens.max() <= hi and lens.std() > 1000
+    assert lens.min() >= lo and lens.max() <= hi and lens.std() > 1000 and S >= 8
     _, _, _, table, l2 = inputs.paged_inputs(4, 2, 2, 8, 4, seed=seed, min_len=10, max_len=40)
     used = table[table >= 0]
     assert len(np.unique(used)) == len(used)                       # every physical block used once

@@ -1,0 +1,148 @@
+"""GPU parity of mlt_paged_attn_decode (through the C ABI) against the FP64 oracle."""
+import math
+
+import numpy as np
+import pytest
+
+pytestmark = pytest.mark.gpu
+
+torch = pytest.importorskip("torch")
+
+import oracle  # noqa: E402
+import paper_2503_14985_b200 as mlt  # noqa: E402
+from paper_2503_14985_b200 import inputs  # noqa: E402
+
+from gpu_util import assert_device_healthy, to_dev  # noqa: E402
+from parity import check_mha  # noqa: E402
+
+SENTINEL = 0x7FC1
+
+
+def run_paged(Q, Kc, Vc, table, lens, scale, workspace_bytes=None, with_lse=True):
+    """Runs the entry point on BF16 bit arrays with guard bands; returns (O [S*H, D] f64, LSE [S*H] f64)."""
+    S, H, D = Q.shape
+    NB, Hkv, bs, _ = Kc.shape
+    guard = 256
+    Obuf = torch.from_numpy(np.full((S * H * D + 2 * guard,), SENTINEL, np.uint16).view(np.int16)).cuda()
+    Lbuf = torch.full((S * H + 2 * guard,), float("nan"), dtype=torch.float32, device="cuda")
+    O = Obuf[guard:guard + S * H * D]
+    L = Lbuf[guard:guard + S * H]
+    if workspace_bytes is None:
+        workspace_bytes = mlt.paged_attn_workspace_bytes(S, H, D)
+    ws = torch.full((workspace_bytes + 64,), 0xAB, dtype=torch.uint8, device="cuda") if workspace_bytes else None
+    dQ, dK, dV = to_dev(Q), to_dev(Kc), to_dev(Vc)
+    dT = torch.from_numpy(np.ascontiguousarray(table, dtype=np.int32)).cuda()
+    dL = torch.from_numpy(np.ascontiguousarray(lens, dtype=np.int32)).cuda()
+    rc = mlt.paged_attn_decode_raw(dQ.data_ptr(), dK.data_ptr(), dV.data_ptr(), dT.data_ptr(), dL.data_ptr(),
+                                   O.data_ptr(), L.data_ptr() if with_lse else 0, S, H, Hkv, D, bs, table.shape[1], NB,
+                                   float(np.float32(scale)), ws.data_ptr() if ws is not None else 0, workspace_bytes,
+                                   torch.cuda.current_stream().cuda_stream)
+    assert rc == 0, mlt.status_string(rc)
+    assert_device_healthy()
+    ob = Obuf.cpu().numpy().view(np.uint16)
+    assert (ob[:guard] == SENTINEL).all() and (ob[-guard:] == SENTINEL).all(), "O guard band was written"
+    lb = Lbuf.cpu().numpy()
+    assert np.isnan(lb[:guard]).all() and np.isnan(lb[-guard:]).all(), "LSE guard band was written"
+    if ws is not None:
+        assert (ws[workspace_bytes:].cpu().numpy() == 0xAB).all(), "workspace overrun"
+    body = ob[guard:-guard]
+    assert not (body == SENTINEL).any(), "unwritten O elements"
+    return inputs.bf16_bits_to_f64(body).reshape(S * H, D), (lb[guard:-guard].astype(np.float64) if with_lse else None)
+
+
+def poison_unused(Kc, Vc, table, lens, bs):
+    """NaN patterns in every cache position no sequence may read: tails of last blocks and unreferenced blocks."""
+    used = np.zeros(Kc.shape[0], bool)
+    Kp, Vp = Kc.copy(), Vc.copy()
+    for s in range(table.shape[0]):
+        n = (int(lens[s]) + bs - 1) // bs
+        used[table[s, :n]] = True
+        if n and lens[s] % bs:
+            Kp[table[s, n - 1], :, lens[s] % bs:] = 0x7FC0
+            Vp[table[s, n - 1], :, lens[s] % bs:] = 0x7FC0
+    Kp[~used] = 0x7FC0
+    Vp[~used] = 0x7FC0
+    return Kp, Vp
+
+
+CASES = [  # S, H, H_kv, D, block_size, min_len, max_len
+    (3, 4, 4, 128, 16, 1, 100), (2, 8, 8, 64, 16, 17, 300), (5, 8, 2, 128, 16, 50, 700), (4, 8, 1, 64, 8, 1, 90),
+    (2, 4, 2, 128, 32, 200, 1500), (1, 2, 2, 128, 16, 5000, 5000), (7, 16, 8, 64, 32, 1, 2000), (3, 2, 2, 64, 8, 1, 7),
+]
+
+
+@pytest.mark.parametrize("S,H,Hkv,D,bs,lo,hi", CASES)
+def test_parity_with_length_mix_and_scattered_blocks(S, H, Hkv, D, bs, lo, hi):
+    Q, Kc, Vc, table, lens = inputs.paged_inputs(S, H, Hkv, D, bs, seed=300 + S + H + hi, min_len=lo, max_len=hi)
+    Kc, Vc = poison_unused(Kc, Vc, table, lens, bs)
+    scale = np.float32(1 / math.sqrt(D))
+    o, lse = run_paged(Q, Kc, Vc, table, lens, scale)
+    o_ref, l_ref = oracle.paged_attn_decode(Q, Kc, Vc, table, lens, scale=scale)
+    rel, mx, dl = check_mha(o, lse, o_ref.reshape(-1, D), l_ref.reshape(-1), f"{(S, H, Hkv, D, bs, lo, hi)}")
+    print(f"rel_fro={rel:.3e} max_abs={mx:.3e} lse={dl:.3e}")
+
+
+@pytest.mark.parametrize("workspace_bytes", [0, 4096, None])
+def test_any_workspace_size_gives_the_same_answer(workspace_bytes):
+    S, H, Hkv, D, bs = 2, 4, 4, 128, 16
+    Q, Kc, Vc, table, lens = inputs.paged_inputs(S, H, Hkv, D, bs, seed=310, min_len=900, max_len=1200)
+    scale = np.float32(1 / math.sqrt(D))
+    o, lse = run_paged(Q, Kc, Vc, table, lens, scale, workspace_bytes=workspace_bytes)
+    o_ref, l_ref = oracle.paged_attn_decode(Q, Kc, Vc, table, lens, scale=scale)
+    check_mha(o, lse, o_ref.reshape(-1, D), l_ref.reshape(-1), f"workspace {workspace_bytes}")
+
+
+def test_empty_and_single_token_sequences():
+    S, H, D, bs = 4, 2, 64, 16
+    Q, Kc, Vc, table, lens = inputs.paged_inputs(S, H, H, D, bs, seed=311, min_len=40, max_len=40)
+    lens = np.array([0, 1, 16, 40], dtype=np.int32)
+    o, lse = run_paged(Q, Kc, Vc, table, lens, 0.125)
+    o = o.reshape(S, H, D); lse = lse.reshape(S, H)
+    assert (o[0] == 0).all() and np.isneginf(lse[0]).all()
+    assert np.array_equal(o[1], inputs.bf16_bits_to_f64(Vc[table[1, 0], :, 0]))     # one token: exactly its value
+    o_ref, l_ref = oracle.paged_attn_decode(Q, Kc, Vc, table, lens, scale=0.125)
+    check_mha(o[2:].reshape(-1, D), lse[2:].reshape(-1), o_ref[2:].reshape(-1, D), l_ref[2:].reshape(-1), "16 and 40")
+
+
+def test_bad_block_table_entry_is_reported_not_dereferenced():
+    S, H, D, bs = 1, 2, 64, 16
+    Q, Kc, Vc, table, lens = inputs.paged_inputs(S, H, H, D, bs, seed=312, min_len=64, max_len=64)
+    bad = table.copy(); bad[0, 2] = Kc.shape[0] + 1000
+    dQ, dK, dV = to_dev(Q), to_dev(Kc), to_dev(Vc)
+    dT = torch.from_numpy(bad).cuda(); dL = torch.from_numpy(lens).cuda()
+    O = torch.empty(S * H * D, dtype=torch.int16, device="cuda")
+    rc = mlt.paged_attn_decode_raw(dQ.data_ptr(), dK.data_ptr(), dV.data_ptr(), dT.data_ptr(), dL.data_ptr(), O.data_ptr(),
+                                   0, S, H, H, D, bs, table.shape[1], Kc.shape[0], 0.125)
+    assert rc == 0
+    status, detail = mlt.last_device_error()
+    assert status == 7 and detail[0] == 7 and detail[1] == 2 and detail[2] == 0
+    assert mlt.last_device_error()[0] == 0      # cleared
+
+
+def test_deterministic_across_runs():
+    S, H, Hkv, D, bs = 6, 8, 2, 128, 16
+    Q, Kc, Vc, table, lens = inputs.paged_inputs(S, H, Hkv, D, bs, seed=313, min_len=100, max_len=3000)
+    a = run_paged(Q, Kc, Vc, table, lens, 0.09)
+    b = run_paged(Q, Kc, Vc, table, lens, 0.09)
+    assert np.array_equal(a[0], b[0]) and np.array_equal(a[1], b[1])
+
+
+@pytest.mark.parametrize("name", list(inputs.PAGED_CONFIGS))
+def test_benchmark_configs(name):
+    S, H, Hkv, D, bs, lo, hi, seed = inputs.PAGED_CONFIGS[name]
+    Q, Kc, Vc, table, lens = inputs.paged_inputs(S, H, Hkv, D, bs, seed=seed, min_len=lo, max_len=hi)
+    scale = np.float32(1 / math.sqrt(D))
+    ws = torch.empty(mlt.paged_attn_workspace_bytes(S, H, D), dtype=torch.uint8, device="cuda")
+    dT = torch.from_numpy(table).cuda(); dL = torch.from_numpy(lens).cuda()
+    O, LSE = mlt.paged_attn_decode(to_dev(Q), to_dev(Kc), to_dev(Vc), dT, dL, scale=float(scale), workspace=ws)
+    assert_device_healthy()
+    assert torch.isfinite(O.float()).all() and torch.isfinite(LSE).all()
+    # the oracle on a sample of sequences (all heads): shortest, longest and a few others
+    order = np.argsort(lens)
+    pick = sorted({int(order[0]), int(order[-1]), int(order[len(order) // 2]), 0, S - 1})[:4]
+    sub = np.array(pick)
+    o_ref, l_ref = oracle.paged_attn_decode(Q[sub], Kc, Vc, table[sub], lens[sub], scale=scale)
+    got_o = inputs.bf16_bits_to_f64(O[torch.from_numpy(sub).cuda()].contiguous().view(torch.int16).cpu().numpy().view(np.uint16))
+    got_l = LSE[torch.from_numpy(sub).cuda()].cpu().numpy().astype(np.float64)
+    rel, mx, dl = check_mha(got_o.reshape(-1, D), got_l.reshape(-1), o_ref.reshape(-1, D), l_ref.reshape(-1), name)
+    print(f"{name}: rel_fro={rel:.3e} max_abs={mx:.3e} lse={dl:.3e}")
