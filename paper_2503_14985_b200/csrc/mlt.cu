@@ -330,6 +330,7 @@ int mlt_paged_attn_decode(const void* Q, const void* K_cache, const void* V_cach
     // use as many splits as the caller's scratch allows
     if (!workspace) workspace_bytes = 0;
     while (p.splits > 1 && paged_workspace_bytes(num_seqs, H, D, p.splits) > workspace_bytes) --p.splits;
+    p.blocks_per_split = (max_blocks_per_seq + p.splits - 1) / p.splits;
     return paged_launch(p, D, workspace, static_cast<cudaStream_t>(stream));
 }
 

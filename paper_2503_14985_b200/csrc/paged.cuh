@@ -40,7 +40,10 @@ struct PagedParams {
     float* LSE;                    // [num_seqs, H] or null
     float* part_o;                 // [num_seqs, H, splits, D]   (splits > 1)
     float2* part_ml;               // [num_seqs, H, splits] {m in log2 units, l}
-    int num_seqs, H, H_kv, block_size, max_blocks, num_blocks, splits;
+    int num_seqs, H, H_kv, block_size, max_blocks, num_blocks;
+    int splits;            // CTAs per (sequence, KV head) = grid.x
+    int blocks_per_split;  // KV blocks each of them covers: the same for every sequence, so CTAs do equal work and
+                           // the CTAs beyond a short sequence's end exit at once
     float scale_log2e;
 };
 
@@ -76,9 +79,9 @@ paged_decode_kernel(const PagedParams p) {
     const int grp = lane / LPT;   // which token of a step
     const int len = p.seq_lens[s];
     const int nblk = (len + BS - 1) / BS;
-    const int per_split = (nblk + p.splits - 1) / p.splits;
-    const int b0 = sp * per_split;
-    const int b1 = min(nblk, b0 + per_split);
+    const int b0 = sp * p.blocks_per_split;
+    const int b1 = min(nblk, b0 + p.blocks_per_split);
+    if (p.splits > 1 && b0 >= nblk && !(sp == 0)) return;  // nothing of this sequence here (split 0 reports an empty one)
 
     // this lane's 8 columns of the G query rows
     float q[G][8];
@@ -220,10 +223,12 @@ __global__ void __launch_bounds__(D)
 paged_combine_kernel(const PagedParams p) {
     const int64_t row = blockIdx.x;
     const int d = threadIdx.x;
+    const int nblk = (p.seq_lens[row / p.H] + p.block_size - 1) / p.block_size;
+    const int used = max(1, min(p.splits, (nblk + p.blocks_per_split - 1) / p.blocks_per_split));  // splits that wrote
     float mt = -INFINITY;
-    for (int sp = 0; sp < p.splits; ++sp) mt = fmaxf(mt, p.part_ml[row * p.splits + sp].x);
+    for (int sp = 0; sp < used; ++sp) mt = fmaxf(mt, p.part_ml[row * p.splits + sp].x);
     float lt = 0.0f, ot = 0.0f;
-    for (int sp = 0; sp < p.splits; ++sp) {
+    for (int sp = 0; sp < used; ++sp) {
         const float2 ml = p.part_ml[row * p.splits + sp];
         const float sw = (ml.x == -INFINITY) ? 0.0f : fast_exp2(ml.x - mt);
         lt += ml.y * sw;
@@ -237,11 +242,15 @@ inline size_t paged_workspace_bytes(int num_seqs, int H, int D, int splits) {
     return splits <= 1 ? 0 : static_cast<size_t>(num_seqs) * H * splits * (static_cast<size_t>(D) * 4 + 8);
 }
 
-// How many CTAs share one (sequence, KV head): enough to put a few CTAs on every SM, at least 8 KV blocks each.
+// How many CTAs share one (sequence, KV head).  Each covers the same number of KV blocks, so the CTAs beyond a
+// short sequence's end are empty: aim at 16 blocks (256 tokens) per CTA, which leaves enough busy CTAs per SM to
+// hide the HBM latency even when most sequences are shorter than the longest allowed; 8 blocks if that still
+// leaves SMs idle; no split when there are already many (sequence, KV head) pairs per SM.
 inline int paged_choose_splits(int num_seqs, int H_kv, int max_blocks, int sm_count) {
     const int64_t base = static_cast<int64_t>(num_seqs) * H_kv;
-    int splits = static_cast<int>((4ll * sm_count + base - 1) / base);
-    splits = std::min(splits, (max_blocks + 7) / 8);
+    if (base >= 16ll * sm_count) return 1;
+    int splits = (max_blocks + 15) / 16;
+    if (base * splits < 4ll * sm_count) splits = (max_blocks + 7) / 8;
     return std::max(1, std::min(splits, kPagedMaxSplits));
 }
 
