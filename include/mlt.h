@@ -29,7 +29,8 @@ typedef enum {
     MLT_ERR_CUDA = 4,        /* a CUDA runtime / driver call failed */
     MLT_ERR_ARCH = 5,        /* current device is not compute capability 10.x */
     MLT_ERR_TIMEOUT = 6,     /* a bounded device-side wait expired (reported by mlt_last_device_error) */
-    MLT_ERR_BAD_BLOCK = 7    /* a block-table entry outside [0, num_blocks) was met (reported by mlt_last_device_error) */
+    MLT_ERR_BAD_BLOCK = 7,   /* a block-table entry outside [0, num_blocks) was met (reported by mlt_last_device_error) */
+    MLT_ERR_SCRATCH_LIMIT = 8 /* mlt_paged_attn_decode_static: the call needs more than MLT_PAGED_STATIC_SCRATCH_BYTES */
 } mlt_status;
 
 /*
@@ -106,6 +107,34 @@ int mlt_paged_attn_decode(const void* Q, const void* K_cache, const void* V_cach
                           int num_seqs, int H, int H_kv, int D,
                           int block_size, int max_blocks_per_seq, int num_blocks, float scale,
                           void* workspace, size_t workspace_bytes, void* stream);
+
+/*
+ * mlt_paged_attn_decode for callers that cannot supply scratch memory.  (The paper has no counterpart: this is a
+ * library addition.)  Who needs it: an engine whose own pool already owns all device memory, a plug-in that
+ * receives tensors but no allocator, a decode loop in which cudaMalloc -- it synchronises the device -- is ruled
+ * out once the loop is running.  The partial results of split sequences go into an array of
+ * MLT_PAGED_STATIC_SCRATCH_BYTES bytes that is part of the library's device image (every GPU that loads the
+ * library carries it until the process exits).  The call allocates nothing, on host or device.
+ *
+ * Arguments, layouts, results and errors are those of mlt_paged_attn_decode, without the workspace pair.  The
+ * split over CTAs is the one mlt_paged_attn_decode makes with a full workspace, so the outputs are the same;
+ * it needs num_seqs * H * splits * (4 * D + 8) bytes with splits <= 32 (splits = ceil(max_blocks_per_seq / 16),
+ * or / 8 for few sequences), and a call that needs more than the array holds returns MLT_ERR_SCRATCH_LIMIT
+ * and launches nothing.
+ *
+ * The first call on each device looks up the array's device address (with that device current); make that first
+ * call before any stream capture begins.  All calls on a device share the one array and it keeps the last call's
+ * contents: nothing in it has to be cleared between calls, but two calls that overlap on the GPU (different
+ * streams, or one thread per stream) race on it -- serialise them, or use mlt_paged_attn_decode with separate
+ * workspaces.
+ */
+#define MLT_PAGED_STATIC_SCRATCH_BYTES (16 * 1024 * 1024)
+int mlt_paged_attn_decode_static(const void* Q, const void* K_cache, const void* V_cache,
+                                 const int32_t* block_table, const int32_t* seq_lens,
+                                 void* O, float* LSE,
+                                 int num_seqs, int H, int H_kv, int D,
+                                 int block_size, int max_blocks_per_seq, int num_blocks, float scale,
+                                 void* stream);
 
 /*
  * Device-side health word.  Kernels never trap: a wait that exceeds its bound

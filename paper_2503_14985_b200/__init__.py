@@ -5,4 +5,5 @@
 """
 from . import inputs  # noqa: F401
 from .binding import (MltError, gemm, gemm_raw, last_device_error, load, mha_fwd, mha_fwd_raw,  # noqa: F401
-                      paged_attn_decode, paged_attn_decode_raw, paged_attn_workspace_bytes, status_string, version)
+                      paged_attn_decode, paged_attn_decode_raw, paged_attn_decode_static_raw,
+                      paged_attn_workspace_bytes, status_string, version)

@@ -14,9 +14,12 @@ LIB_PATH = os.path.join(_HERE, "libmlt.so")
 
 MLT_OK = 0
 STATUS_NAMES = {0: "MLT_OK", 1: "MLT_ERR_INVALID_ARG", 2: "MLT_ERR_UNSUPPORTED", 3: "MLT_ERR_ALIGNMENT",
-                4: "MLT_ERR_CUDA", 5: "MLT_ERR_ARCH", 6: "MLT_ERR_TIMEOUT", 7: "MLT_ERR_BAD_BLOCK"}
+                4: "MLT_ERR_CUDA", 5: "MLT_ERR_ARCH", 6: "MLT_ERR_TIMEOUT", 7: "MLT_ERR_BAD_BLOCK",
+                8: "MLT_ERR_SCRATCH_LIMIT"}
+PAGED_STATIC_SCRATCH_BYTES = 16 * 1024 * 1024
 
-EXPORTS = ("mlt_gemm", "mlt_mha_fwd", "mlt_paged_attn_decode", "mlt_paged_attn_workspace_bytes",
+EXPORTS = ("mlt_gemm", "mlt_mha_fwd", "mlt_paged_attn_decode", "mlt_paged_attn_decode_static",
+           "mlt_paged_attn_workspace_bytes",
            "mlt_last_device_error", "mlt_status_string", "mlt_version")
 
 _lib = None
@@ -45,6 +48,9 @@ def load() -> ctypes.CDLL:
         lib.mlt_paged_attn_decode.argtypes = [p, p, p, p, p, p, p, i32, i32, i32, i32, i32, i32, i32, ctypes.c_float,
                                               p, ctypes.c_size_t, p]
         lib.mlt_paged_attn_decode.restype = i32
+        lib.mlt_paged_attn_decode_static.argtypes = [p, p, p, p, p, p, p, i32, i32, i32, i32, i32, i32, i32,
+                                                     ctypes.c_float, p]
+        lib.mlt_paged_attn_decode_static.restype = i32
         lib.mlt_last_device_error.argtypes = [p]
         lib.mlt_last_device_error.restype = i32
         lib.mlt_status_string.argtypes = [i32]
@@ -84,6 +90,14 @@ def paged_attn_decode_raw(Q: int, K_cache: int, V_cache: int, block_table: int, 
     return int(load().mlt_paged_attn_decode(Q, K_cache, V_cache, block_table, seq_lens, O, LSE, num_seqs, H, H_kv, D,
                                             block_size, max_blocks, num_blocks, scale, workspace, workspace_bytes,
                                             stream))
+
+
+def paged_attn_decode_static_raw(Q: int, K_cache: int, V_cache: int, block_table: int, seq_lens: int, O: int, LSE: int,
+                                 num_seqs: int, H: int, H_kv: int, D: int, block_size: int, max_blocks: int,
+                                 num_blocks: int, scale: float, stream: int = 0) -> int:
+    """mlt_paged_attn_decode_static (scratch inside the library, nothing allocated) with raw device addresses."""
+    return int(load().mlt_paged_attn_decode_static(Q, K_cache, V_cache, block_table, seq_lens, O, LSE, num_seqs, H,
+                                                   H_kv, D, block_size, max_blocks, num_blocks, scale, stream))
 
 
 def last_device_error():

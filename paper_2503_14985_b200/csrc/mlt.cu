@@ -133,6 +133,7 @@ const char* mlt_status_string(int status) {
         case MLT_ERR_ARCH: return "device is not compute capability 10.x (sm_100a required)";
         case MLT_ERR_TIMEOUT: return "a bounded device-side wait expired";
         case MLT_ERR_BAD_BLOCK: return "a block-table entry outside [0, num_blocks) was met";
+        case MLT_ERR_SCRATCH_LIMIT: return "the call needs more scratch than the built-in array of mlt_paged_attn_decode_static holds";
         default: return "unknown status";
     }
 }
@@ -335,3 +336,56 @@ int mlt_paged_attn_decode(const void* Q, const void* K_cache, const void* V_cach
 }
 
 }  // extern "C"
+
+// ---------------------------------------------------------------------------------------------------------
+// Paged-attention decode for callers that cannot provide scratch memory.
+//
+// Some callers have no device memory to give and no way to get any at the point of the call: a serving engine
+// whose own pool already owns the whole GPU, a plug-in that is handed tensors but no allocator, or code on a
+// latency-critical path where a cudaMalloc (which synchronises the device) is forbidden once the loop runs.  For
+// them the partial results of the split sequences go into a fixed array that is part of this library's device
+// image.  Every GPU that loads the library carries the array until the process exits, so it is kept modest.
+// ---------------------------------------------------------------------------------------------------------
+namespace {
+
+static __device__ __align__(256) unsigned char g_paged_static_scratch[MLT_PAGED_STATIC_SCRATCH_BYTES];
+
+// In host code `g_paged_static_scratch` is only a handle for the runtime, not a device address: the address each
+// device gave the array is looked up once per device (with that device current) and kept here.
+void* g_paged_static_scratch_addr[64] = {};
+
+int paged_static_scratch(void** out) {
+    int dev = 0;
+    if (cudaGetDevice(&dev) != cudaSuccess || dev < 0 || dev >= 64) return MLT_ERR_CUDA;
+    std::lock_guard<std::mutex> lock(g_mutex);
+    if (!g_paged_static_scratch_addr[dev]) {
+        void* addr = nullptr;
+        if (cudaGetSymbolAddress(&addr, g_paged_static_scratch) != cudaSuccess || !addr) return MLT_ERR_CUDA;
+        g_paged_static_scratch_addr[dev] = addr;
+    }
+    *out = g_paged_static_scratch_addr[dev];
+    return MLT_OK;
+}
+
+}  // namespace
+
+extern "C" int mlt_paged_attn_decode_static(const void* Q, const void* K_cache, const void* V_cache,
+                                            const int32_t* block_table, const int32_t* seq_lens, void* O, float* LSE,
+                                            int num_seqs, int H, int H_kv, int D, int block_size,
+                                            int max_blocks_per_seq, int num_blocks, float scale, void* stream) {
+    PagedParams p;
+    DeviceInfo dev;
+    bool launch = false;
+    int rc = paged_prepare(Q, K_cache, V_cache, block_table, seq_lens, O, LSE, num_seqs, H, H_kv, D, block_size,
+                           max_blocks_per_seq, num_blocks, scale, &p, &dev, &launch);
+    if (rc != MLT_OK || !launch) return rc;
+    // the same split as mlt_paged_attn_decode makes with a full workspace; it must fit the built-in array
+    if (paged_workspace_bytes(num_seqs, H, D, p.splits) > static_cast<size_t>(MLT_PAGED_STATIC_SCRATCH_BYTES))
+        return MLT_ERR_SCRATCH_LIMIT;
+    p.blocks_per_split = (max_blocks_per_seq + p.splits - 1) / p.splits;
+    void* scratch = nullptr;
+    rc = paged_static_scratch(&scratch);
+    if (rc != MLT_OK) return rc;
+    // nothing in the array has to start at zero: every partial the combine step reads was written by this call
+    return paged_launch(p, D, scratch, static_cast<cudaStream_t>(stream));
+}

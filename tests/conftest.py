@@ -24,3 +24,10 @@ def pytest_collection_modifyitems(config, items):
     for item in items:
         if "gpu" in item.keywords:
             item.add_marker(skip)
+
+
+@pytest.fixture(scope="session", autouse=True)
+def _built_libraries():
+    """Compile libmlt.so and the oracle if they are missing or stale, so any test file can run on its own."""
+    import __graft_entry__ as entry
+    entry.build()

@@ -27,8 +27,8 @@ def test_header_symbols_are_exported(lib):
 
 def test_version_and_status_strings(lib):
     assert binding.version() >= 100
-    texts = {binding.status_string(i) for i in range(8)}
-    assert len(texts) == 8 and "unknown status" not in texts
+    texts = {binding.status_string(i) for i in range(9)}
+    assert len(texts) == 9 and "unknown status" not in texts
     assert binding.status_string(99) == "unknown status"
 
 
