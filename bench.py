@@ -381,12 +381,17 @@ def time_all_configs(mlt, torch, dev, stream, iters: int = 20, only: str | None 
 
     flush = torch.empty(256 << 20, dtype=torch.int8, device=dev)
 
-    def timeit(fn, flop):
+    def timeit(fn, flop, read_flush=False):
         for _ in range(warm):
             fn()
         times = []
         for _ in range(iters):
-            flush.zero_()  # evict L2 between timed launches
+            # evict L2 between timed launches: by writing a 256 MB buffer, or (for the HBM-bound decode kernel,
+            # whose reads would otherwise have to push 126 MB of dirty lines out first) by reading it
+            if read_flush:
+                flush.view(torch.int32).sum()
+            else:
+                flush.zero_()
             a, b = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
             a.record(stream)
             fn()
@@ -443,7 +448,7 @@ def time_all_configs(mlt, torch, dev, stream, iters: int = 20, only: str | None 
                                            sc, ws.data_ptr(), ws.numel(), sp)
             assert rc == 0, rc
         nbytes = inputs.paged_bytes(lens, Hkv, D)
-        r = timeit(fn, 4.0 * float(lens.sum()) * H * D)
+        r = timeit(fn, 4.0 * float(lens.sum()) * H * D, read_flush=True)
         out[name] = {"ms_min": r["ms_min"], "ms_median": r["ms_median"], "gbs_best": nbytes / r["ms_min"] / 1e6,
                      "gbs_median": nbytes / r["ms_median"] / 1e6, "kv_bytes": nbytes,
                      "frac_of_measured_hbm_best": nbytes / r["ms_min"] / 1e6 / hbm_peak}

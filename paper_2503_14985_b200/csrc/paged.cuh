@@ -218,22 +218,45 @@ paged_decode_kernel(const PagedParams p) {
 }
 
 // O[row] = sum over splits of the partials, rescaled to the common max; one CTA of D threads per (seq, head).
+// The {m, l} pairs go through shared memory once, and the partial outputs are read with independent loads
+// (eight in flight per thread), so the kernel is a few microseconds of latency rather than a chain of them.
 template <int D>
 __global__ void __launch_bounds__(D)
 paged_combine_kernel(const PagedParams p) {
+    __shared__ float sm_w[kPagedMaxSplits];  // 2^(m_sp - m) per split
+    __shared__ float sm_stat[2];             // common max, total l
     const int64_t row = blockIdx.x;
     const int d = threadIdx.x;
     const int nblk = (p.seq_lens[row / p.H] + p.block_size - 1) / p.block_size;
     const int used = max(1, min(p.splits, (nblk + p.blocks_per_split - 1) / p.blocks_per_split));  // splits that wrote
-    float mt = -INFINITY;
-    for (int sp = 0; sp < used; ++sp) mt = fmaxf(mt, p.part_ml[row * p.splits + sp].x);
-    float lt = 0.0f, ot = 0.0f;
-    for (int sp = 0; sp < used; ++sp) {
-        const float2 ml = p.part_ml[row * p.splits + sp];
+    if (d < 32) {
+        const float2 ml = d < used ? p.part_ml[row * p.splits + d] : make_float2(-INFINITY, 0.0f);
+        float mt = ml.x;
+#pragma unroll
+        for (int w = 16; w > 0; w >>= 1) mt = fmaxf(mt, __shfl_xor_sync(0xffffffffu, mt, w));
         const float sw = (ml.x == -INFINITY) ? 0.0f : fast_exp2(ml.x - mt);
-        lt += ml.y * sw;
-        ot += p.part_o[(row * p.splits + sp) * D + d] * sw;
+        float lt = ml.y * sw;
+#pragma unroll
+        for (int w = 16; w > 0; w >>= 1) lt += __shfl_xor_sync(0xffffffffu, lt, w);
+        sm_w[d] = sw;
+        if (d == 0) {
+            sm_stat[0] = mt;
+            sm_stat[1] = lt;
+        }
     }
+    __syncthreads();
+    const float* po = p.part_o + row * p.splits * D + d;
+    float ot = 0.0f;
+    int sp = 0;
+    for (; sp + 8 <= used; sp += 8) {
+        float v[8];
+#pragma unroll
+        for (int i = 0; i < 8; ++i) v[i] = po[(sp + i) * D];
+#pragma unroll
+        for (int i = 0; i < 8; ++i) ot = fmaf(v[i], sm_w[sp + i], ot);
+    }
+    for (; sp < used; ++sp) ot = fmaf(po[sp * D], sm_w[sp], ot);
+    const float mt = sm_stat[0], lt = sm_stat[1];
     p.O[row * D + d] = __float2bfloat16(lt > 0.0f ? ot / lt : 0.0f);
     if (d == 0 && p.LSE) p.LSE[row] = lt > 0.0f ? (mt + log2f(lt)) * 0.6931471805599453f : -INFINITY;
 }
