@@ -429,8 +429,27 @@ def time_all_configs(mlt, torch, dev, stream, iters: int = 20, only: str | None 
             assert rc == 0, rc
         out[name] = timeit(fn, inputs.mha_flops(Bn, H, Nq, Nk, D, causal))
         del dQ, dK, dV, dO, dL
-    # paged-attention decode (Sec. 3.2 / 4.3): bound by HBM, reported in GB/s of visible K and V
     hbm_peak = measured_peaks()["hbm_gbs"]
+    # memory-bound GEMM shapes (Sec. 4.1, next-token prediction): split-K through mlt_gemm_ex, reported in GB/s of
+    # A, B and C each moved once
+    for name, (M, N, K, kind, seed) in inputs.GEMM_DECODE_CONFIGS.items():
+        if only is not None and name != only:
+            continue
+        A, B = inputs.gemm_inputs(M, N, K, seed=seed, kind=kind)
+        dA, dB = devbits(A), devbits(B)
+        dC = torch.empty((M, N), dtype=torch.int16, device=dev)
+        ws = torch.empty(max(16, mlt.gemm_workspace_bytes(M, N, K)), dtype=torch.uint8, device=dev)
+
+        def fn():
+            rc = mlt.gemm_ex_raw(dA.data_ptr(), dB.data_ptr(), dC.data_ptr(), M, N, K, K, N, N, ws.data_ptr(), ws.numel(), sp)
+            assert rc == 0, rc
+        nbytes = 2.0 * (M * K + K * N + M * N)
+        r = timeit(fn, inputs.gemm_flops(M, N, K), read_flush=True)
+        out[name] = {"ms_min": r["ms_min"], "ms_median": r["ms_median"], "gbs_best": nbytes / r["ms_min"] / 1e6,
+                     "gbs_median": nbytes / r["ms_median"] / 1e6, "tflops_best": r["tflops_best"],
+                     "frac_of_measured_hbm_best": nbytes / r["ms_min"] / 1e6 / hbm_peak}
+        del dA, dB, dC, ws
+    # paged-attention decode (Sec. 3.2 / 4.3): bound by HBM, reported in GB/s of visible K and V
     for name, (S, H, Hkv, D, bs, lo, hi, seed) in inputs.PAGED_CONFIGS.items():
         if only is not None and name != only:
             continue

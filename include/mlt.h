@@ -54,6 +54,24 @@ int mlt_gemm(const void* A, const void* B, void* C,
              void* stream);
 
 /*
+ * mlt_gemm with caller-provided scratch, for the memory-bound shapes of paper Sec. 4.1 (next-token prediction:
+ * few rows of A against large weight matrices, "large k" and "large n" cases).  Such a problem has too few output
+ * tiles to occupy the GPU, so K is cut into slices (split-K): every SM streams a part of B, FP32 partial tiles go
+ * to the workspace and a second small kernel sums them in a fixed order and rounds once to BF16.  Same operation,
+ * arguments, layouts and errors as mlt_gemm; the result can differ from mlt_gemm's in the last BF16 bit (the FP32
+ * partial sums are added in a different order).
+ *
+ *   workspace        device scratch, 16-byte aligned, or NULL (then this is mlt_gemm)
+ *   workspace_bytes  its size; mlt_gemm_workspace_bytes(M, N, K) is always enough (0 when no split would be
+ *                    used); with less, fewer slices are used.  Calls that overlap on the GPU must not share it.
+ */
+size_t mlt_gemm_workspace_bytes(int64_t M, int64_t N, int64_t K);
+int mlt_gemm_ex(const void* A, const void* B, void* C,
+                int64_t M, int64_t N, int64_t K,
+                int64_t lda, int64_t ldb, int64_t ldc,
+                void* workspace, size_t workspace_bytes, void* stream);
+
+/*
  * O = softmax(scale * Q K^T [+ causal mask]) V,  LSE = log-sum-exp of the
  * scaled, masked scores (natural log)  -- paper Sec. 2.5, Algorithm 1
  * (FlashAttention-2 forward: per Q block, loop over K/V blocks, S = Q K_j^T,

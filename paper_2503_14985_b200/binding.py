@@ -18,7 +18,7 @@ STATUS_NAMES = {0: "MLT_OK", 1: "MLT_ERR_INVALID_ARG", 2: "MLT_ERR_UNSUPPORTED",
                 8: "MLT_ERR_SCRATCH_LIMIT"}
 PAGED_STATIC_SCRATCH_BYTES = 16 * 1024 * 1024
 
-EXPORTS = ("mlt_gemm", "mlt_mha_fwd", "mlt_paged_attn_decode", "mlt_paged_attn_decode_static",
+EXPORTS = ("mlt_gemm", "mlt_gemm_ex", "mlt_gemm_workspace_bytes", "mlt_mha_fwd", "mlt_paged_attn_decode", "mlt_paged_attn_decode_static",
            "mlt_paged_attn_workspace_bytes",
            "mlt_last_device_error", "mlt_status_string", "mlt_version")
 
@@ -41,6 +41,10 @@ def load() -> ctypes.CDLL:
         i64, p, i32 = ctypes.c_int64, ctypes.c_void_p, ctypes.c_int
         lib.mlt_gemm.argtypes = [p, p, p, i64, i64, i64, i64, i64, i64, p]
         lib.mlt_gemm.restype = i32
+        lib.mlt_gemm_ex.argtypes = [p, p, p, i64, i64, i64, i64, i64, i64, p, ctypes.c_size_t, p]
+        lib.mlt_gemm_ex.restype = i32
+        lib.mlt_gemm_workspace_bytes.argtypes = [i64, i64, i64]
+        lib.mlt_gemm_workspace_bytes.restype = ctypes.c_size_t
         lib.mlt_mha_fwd.argtypes = [p, p, p, p, p, i32, i32, i32, i32, i32, i32, ctypes.c_float, p]
         lib.mlt_mha_fwd.restype = i32
         lib.mlt_paged_attn_workspace_bytes.argtypes = [i32, i32, i32]
@@ -71,6 +75,16 @@ def version() -> int:
 def gemm_raw(A: int, B: int, C: int, M: int, N: int, K: int, lda: int, ldb: int, ldc: int, stream: int = 0) -> int:
     """mlt_gemm with raw device addresses; returns the status code."""
     return int(load().mlt_gemm(A, B, C, M, N, K, lda, ldb, ldc, stream))
+
+
+def gemm_workspace_bytes(M: int, N: int, K: int) -> int:
+    return int(load().mlt_gemm_workspace_bytes(M, N, K))
+
+
+def gemm_ex_raw(A: int, B: int, C: int, M: int, N: int, K: int, lda: int, ldb: int, ldc: int, workspace: int = 0,
+                workspace_bytes: int = 0, stream: int = 0) -> int:
+    """mlt_gemm_ex (split-K with caller scratch for skinny problems) with raw device addresses."""
+    return int(load().mlt_gemm_ex(A, B, C, M, N, K, lda, ldb, ldc, workspace, workspace_bytes, stream))
 
 
 def mha_fwd_raw(Q: int, K: int, V: int, O: int, LSE: int, B: int, H: int, Nq: int, Nk: int, D: int, causal: int,

@@ -33,6 +33,11 @@ struct GemmParams {
     int M, N, K;
     int tiles_m, tiles_n;
     int group_m;  // M-tiles per raster group
+    // split-K (single-CTA kernel only): work item = (tile, K slice); a slice covers kb_per_split blocks of 64 and
+    // its FP32 partial tile goes to partial[slice][M][N], which gemm_splitk_reduce_kernel sums and rounds.
+    int split_k;       // 1: no split, the epilogue writes BF16 C
+    int kb_per_split;
+    float* partial;
 };
 
 // tile index -> (tile_m, tile_n): groups of `group_m` M-tiles, M fastest inside a group, so that
@@ -64,7 +69,7 @@ gemm_bf16_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_consta
 
     const int warp = threadIdx.x >> 5;
     const int lane = threadIdx.x & 31;
-    const int num_tiles = p.tiles_m * p.tiles_n;
+    const int num_items = p.tiles_m * p.tiles_n * p.split_k;
     const int num_kb = (p.K + kGemmBK - 1) / kGemmBK;
     constexpr uint32_t kTmemCols = 2 * BN;  // 512 for BN = 256, 256 for BN = 128
 
@@ -99,11 +104,12 @@ gemm_bf16_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_consta
             int stage = 0;
             uint32_t phase = 0;
             bool ok = true;
-            for (int tile = blockIdx.x; tile < num_tiles && ok; tile += gridDim.x) {
+            for (int item = blockIdx.x; item < num_items && ok; item += gridDim.x) {
                 int tm, tn;
-                gemm_tile_coords(p, tile, tm, tn);
+                gemm_tile_coords(p, item / p.split_k, tm, tn);
                 const int m0 = tm * kGemmBM, n0 = tn * BN;
-                for (int kb = 0; kb < num_kb; ++kb) {
+                const int kb0 = (item % p.split_k) * p.kb_per_split, kb1 = min(num_kb, kb0 + p.kb_per_split);
+                for (int kb = kb0; kb < kb1; ++kb) {
                     ok = mbar_wait(&empty[stage], phase ^ 1, abort_flag, 0x100 + stage);
                     if (!ok) break;
                     uint8_t* sa = smem + stage * L::kStageBytes;
@@ -131,19 +137,20 @@ gemm_bf16_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_consta
             int acc = 0;
             uint32_t acc_phase = 0;
             bool ok = true;
-            for (int tile = blockIdx.x; tile < num_tiles && ok; tile += gridDim.x) {
+            for (int item = blockIdx.x; item < num_items && ok; item += gridDim.x) {
                 ok = __all_sync(0xffffffffu, mbar_wait(&acc_empty[acc], acc_phase ^ 1, abort_flag, 0x300 + acc));
                 if (!ok) break;
                 tc_fence_after();
                 const uint32_t d_tmem = tmem_base + acc * BN;
-                for (int kb = 0; kb < num_kb; ++kb) {
+                const int kb0 = (item % p.split_k) * p.kb_per_split, kb1 = min(num_kb, kb0 + p.kb_per_split);
+                for (int kb = kb0; kb < kb1; ++kb) {
                     ok = __all_sync(0xffffffffu, mbar_wait(&full[stage], phase, abort_flag, 0x200 + stage));
                     if (!ok) break;
                     tc_fence_after();
                     const uint32_t a_lo = a_lo0 + stage * (L::kStageBytes >> 4);
                     const uint32_t b_lo = b_lo0 + stage * (L::kStageBytes >> 4);
                     if (leader) {
-                        umma_ss_lo_dyn(d_tmem, a_lo, b_lo, idesc, kb != 0);
+                        umma_ss_lo_dyn(d_tmem, a_lo, b_lo, idesc, kb != kb0);
 #pragma unroll
                         for (int k = 1; k < kGemmBK / 16; ++k)
                             umma_ss_lo<true>(d_tmem, a_lo + k * (32 >> 4), b_lo + k * (2048 >> 4), idesc);
@@ -163,9 +170,9 @@ gemm_bf16_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_consta
         int acc = 0;
         uint32_t acc_phase = 0;
         bool ok = true;
-        for (int tile = blockIdx.x; tile < num_tiles && ok; tile += gridDim.x) {
+        for (int item = blockIdx.x; item < num_items && ok; item += gridDim.x) {
             int tm, tn;
-            gemm_tile_coords(p, tile, tm, tn);
+            gemm_tile_coords(p, item / p.split_k, tm, tn);
             const int row = tm * kGemmBM + quarter * 32 + lane;
             const int n0 = tn * BN;
             ok = __all_sync(0xffffffffu, mbar_wait(&acc_full[acc], acc_phase, abort_flag, 0x400 + acc));
@@ -173,13 +180,26 @@ gemm_bf16_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_consta
             tc_fence_after();
             const uint32_t t_row = tmem_base + (static_cast<uint32_t>(quarter * 32) << 16) + acc * BN;
             __nv_bfloat16* crow = p.C + static_cast<int64_t>(row) * p.ldc;
+            float* prow = p.partial
+                              ? p.partial + (static_cast<int64_t>(item % p.split_k) * p.M + row) * p.N
+                              : nullptr;
 #pragma unroll 1
             for (int c = 0; c < BN / 32; ++c) {
                 uint32_t v[32];
                 tmem_ld_32x32b_x32(t_row + c * 32, v);
                 tmem_wait_ld();
                 const int col0 = n0 + c * 32;
-                if (row < p.M) {
+                if (row < p.M && prow) {  // split-K: the FP32 partial of this K slice
+#pragma unroll
+                    for (int q = 0; q < 8; ++q) {
+                        const int col = col0 + q * 4;
+                        if (col + 4 <= p.N && (p.N & 3) == 0) {
+                            *reinterpret_cast<uint4*>(prow + col) = make_uint4(v[q * 4], v[q * 4 + 1], v[q * 4 + 2], v[q * 4 + 3]);
+                        } else {
+                            for (int j = 0; j < 4 && col + j < p.N; ++j) prow[col + j] = __uint_as_float(v[q * 4 + j]);
+                        }
+                    }
+                } else if (row < p.M) {
 #pragma unroll
                     for (int q = 0; q < 4; ++q) {
                         const int col = col0 + q * 8;
@@ -406,6 +426,40 @@ gemm_bf16_pair_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_c
         __syncwarp();
         tc_fence_after();
         tmem_dealloc_pair(tmem_base, kTmemCols);
+    }
+}
+
+// Split-K second step: C[i][j] = RNE_bf16(sum over slices of partial[slice][i][j]); 8 columns per thread.
+__global__ void gemm_splitk_reduce_kernel(const float* partial, __nv_bfloat16* C, int64_t ldc, int M, int N, int split_k) {
+    const int64_t groups_per_row = (N + 7) / 8;
+    const int64_t total = static_cast<int64_t>(M) * groups_per_row;
+    for (int64_t i = blockIdx.x * static_cast<int64_t>(blockDim.x) + threadIdx.x; i < total;
+         i += static_cast<int64_t>(gridDim.x) * blockDim.x) {
+        const int row = static_cast<int>(i / groups_per_row);
+        const int col = static_cast<int>(i % groups_per_row) * 8;
+        float acc[8] = {0, 0, 0, 0, 0, 0, 0, 0};
+        const bool full = col + 8 <= N && (N & 3) == 0;
+        for (int s = 0; s < split_k; ++s) {
+            const float* src = partial + (static_cast<int64_t>(s) * M + row) * N + col;
+            if (full) {
+                const float4 a = *reinterpret_cast<const float4*>(src), b = *reinterpret_cast<const float4*>(src + 4);
+                acc[0] += a.x; acc[1] += a.y; acc[2] += a.z; acc[3] += a.w;
+                acc[4] += b.x; acc[5] += b.y; acc[6] += b.z; acc[7] += b.w;
+            } else {
+                for (int j = 0; j < 8 && col + j < N; ++j) acc[j] += src[j];
+            }
+        }
+        __nv_bfloat16* dst = C + static_cast<int64_t>(row) * ldc + col;
+        if (col + 8 <= N) {
+            uint4 out;
+            out.x = pack_bf16x2(acc[0], acc[1]);
+            out.y = pack_bf16x2(acc[2], acc[3]);
+            out.z = pack_bf16x2(acc[4], acc[5]);
+            out.w = pack_bf16x2(acc[6], acc[7]);
+            *reinterpret_cast<uint4*>(dst) = out;
+        } else {
+            for (int j = 0; col + j < N; ++j) dst[j] = __float2bfloat16(acc[j]);
+        }
     }
 }
 

@@ -151,8 +151,22 @@ int mlt_last_device_error(uint32_t* detail) {
     return MLT_OK;
 }
 
-int mlt_gemm(const void* A, const void* B, void* C, int64_t M, int64_t N, int64_t K, int64_t lda, int64_t ldb,
-             int64_t ldc, void* stream) {
+// K slices a skinny problem may be cut into: enough work items for two per SM, at least 4 blocks of 64 per slice
+static int gemm_max_split(int64_t M, int64_t N, int64_t K) {
+    const int64_t tiles = ((M + 127) / 128) * ((N + 127) / 128);
+    const int64_t num_kb = (K + kGemmBK - 1) / kGemmBK;
+    if (tiles >= 1024 || num_kb < 8) return 1;
+    return static_cast<int>(std::min<int64_t>(32, num_kb / 4));
+}
+
+size_t mlt_gemm_workspace_bytes(int64_t M, int64_t N, int64_t K) {
+    if (M <= 0 || N <= 0 || K <= 0) return 0;
+    const int split = gemm_max_split(M, N, K);
+    return split > 1 ? static_cast<size_t>(split) * M * N * sizeof(float) : 0;
+}
+
+static int gemm_run(const void* A, const void* B, void* C, int64_t M, int64_t N, int64_t K, int64_t lda, int64_t ldb,
+                    int64_t ldc, void* workspace, size_t workspace_bytes, void* stream) {
     // ---- validation (no CUDA call before this block has passed) ----
     if (M < 0 || N < 0 || K < 0) return MLT_ERR_INVALID_ARG;
     if (M == 0 || N == 0) return MLT_OK;
@@ -161,6 +175,7 @@ int mlt_gemm(const void* A, const void* B, void* C, int64_t M, int64_t N, int64_
     if (M > INT32_MAX - 256 || N > INT32_MAX - 256 || K > INT32_MAX - 256) return MLT_ERR_UNSUPPORTED;
     if (!aligned16(C) || (ldc % 8) != 0) return MLT_ERR_ALIGNMENT;
     if (K > 0 && (!aligned16(A) || !aligned16(B) || (lda % 8) != 0 || (ldb % 8) != 0)) return MLT_ERR_ALIGNMENT;
+    if (workspace && !aligned16(workspace)) return MLT_ERR_ALIGNMENT;
 
     DeviceInfo dev;
     int rc = get_device(&dev);
@@ -217,6 +232,22 @@ int mlt_gemm(const void* A, const void* B, void* C, int64_t M, int64_t N, int64_
     p.K = static_cast<int>(K);
     p.tiles_m = static_cast<int>(tiles_m);
     p.tiles_n = static_cast<int>(tiles_n);
+    p.split_k = 1;
+    p.kb_per_split = static_cast<int>((K + kGemmBK - 1) / kGemmBK);
+    p.partial = nullptr;
+    if (variant == 2 && workspace) {
+        // Few tiles (skinny or small problem): cut K into slices so that about two work items per SM exist; the
+        // weights are then streamed by all SMs at once.  FP32 partials go to the caller's scratch.
+        const int num_kb = p.kb_per_split;
+        int split = static_cast<int>(std::min<int64_t>(gemm_max_split(M, N, K),
+                                                        (2ll * dev.sm_count + tiles_m * tiles_n - 1) / (tiles_m * tiles_n)));
+        while (split > 1 && static_cast<size_t>(split) * M * N * sizeof(float) > workspace_bytes) --split;
+        if (split > 1) {
+            p.kb_per_split = (num_kb + split - 1) / split;
+            p.split_k = (num_kb + p.kb_per_split - 1) / p.kb_per_split;  // no empty slice
+            p.partial = static_cast<float*>(workspace);
+        }
+    }
     if (variant == 0) {
         // M-tiles per raster group: wide problems re-read B once per group, so fewer, taller groups pay
         p.group_m = debug_env_int("MLT_GEMM_GROUP_M", tiles_n >= 32 ? 16 : 8);
@@ -224,13 +255,29 @@ int mlt_gemm(const void* A, const void* B, void* C, int64_t M, int64_t N, int64_
         gemm_bf16_pair_kernel<6><<<2 * clusters, kGemmThreads, GemmPairSmem<6>::kTotal, st>>>(ta, tb, p);
     } else {
         p.group_m = 16;
-        const int grid = static_cast<int>(std::min<int64_t>(tiles_m * tiles_n, dev.sm_count));
+        const int grid = static_cast<int>(std::min<int64_t>(tiles_m * tiles_n * p.split_k, dev.sm_count));
         if (variant == 1)
             gemm_bf16_kernel<256, 4><<<grid, kGemmThreads, GemmSmem<256, 4>::kTotal, st>>>(ta, tb, p);
         else
             gemm_bf16_kernel<128, 6><<<grid, kGemmThreads, GemmSmem<128, 6>::kTotal, st>>>(ta, tb, p);
+        if (p.split_k > 1) {
+            if (cudaGetLastError() != cudaSuccess) return MLT_ERR_CUDA;
+            const int64_t groups = M * ((N + 7) / 8);
+            const int blocks = static_cast<int>(std::min<int64_t>((groups + 255) / 256, 8 * dev.sm_count));
+            gemm_splitk_reduce_kernel<<<blocks, 256, 0, st>>>(p.partial, p.C, ldc, p.M, p.N, p.split_k);
+        }
     }
     return cudaGetLastError() == cudaSuccess ? MLT_OK : MLT_ERR_CUDA;
+}
+
+int mlt_gemm(const void* A, const void* B, void* C, int64_t M, int64_t N, int64_t K, int64_t lda, int64_t ldb,
+             int64_t ldc, void* stream) {
+    return gemm_run(A, B, C, M, N, K, lda, ldb, ldc, nullptr, 0, stream);
+}
+
+int mlt_gemm_ex(const void* A, const void* B, void* C, int64_t M, int64_t N, int64_t K, int64_t lda, int64_t ldb,
+                int64_t ldc, void* workspace, size_t workspace_bytes, void* stream) {
+    return gemm_run(A, B, C, M, N, K, lda, ldb, ldc, workspace, workspace_bytes, stream);
 }
 
 int mlt_mha_fwd(const void* Q, const void* K, const void* V, void* O, float* LSE, int B, int H, int Nq, int Nk, int D,

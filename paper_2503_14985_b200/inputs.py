@@ -229,6 +229,15 @@ GEMM_CONFIGS = {
     "gemm_8192x4096x28672": (8192, 4096, 28672, "normal", 3),
 }
 
+# Memory-bound GEMM shapes (Sec. 4.1: next-token prediction; "large k" and "large n" cases; the paper lists none)
+GEMM_DECODE_CONFIGS = {
+    # name: (M, N, K, value kind, seed)
+    "gemm_decode_16x4096x4096": (16, 4096, 4096, "normal", 11),
+    "gemm_decode_16x28672x4096": (16, 28672, 4096, "normal", 12),
+    "gemm_decode_16x4096x28672": (16, 4096, 28672, "normal", 13),
+    "gemm_decode_64x8192x8192": (64, 8192, 8192, "normal", 14),
+}
+
 MHA_CONFIGS = {
     # name: (B, H, Nq, Nk, D, causal, seed, outlier_percent)
     "mha_b4h32n1024d64": (4, 32, 1024, 1024, 64, 0, 4, 0),

@@ -1,0 +1,83 @@
+"""GPU parity of mlt_gemm_ex (split-K with caller scratch, for the memory-bound shapes of Sec. 4.1) against the oracle."""
+import numpy as np
+import pytest
+
+pytestmark = pytest.mark.gpu
+
+torch = pytest.importorskip("torch")
+
+import oracle  # noqa: E402
+import paper_2503_14985_b200 as mlt  # noqa: E402
+from paper_2503_14985_b200 import inputs  # noqa: E402
+
+from gpu_util import assert_device_healthy, to_bits, to_dev  # noqa: E402
+from parity import check_gemm  # noqa: E402
+
+SENTINEL = 0x7FC1
+
+
+def run_ex(A, B, M, N, K, ldc, workspace_bytes):
+    Cbuf = torch.from_numpy(np.full((M + 2, ldc), SENTINEL, dtype=np.uint16).view(np.int16)).cuda().view(torch.bfloat16)
+    ws = torch.full((workspace_bytes + 64,), 0xAB, dtype=torch.uint8, device="cuda") if workspace_bytes else None
+    dA, dB = to_dev(A), to_dev(B)
+    rc = mlt.gemm_ex_raw(dA.data_ptr(), dB.data_ptr(), Cbuf.data_ptr(), M, N, K, A.shape[1], B.shape[1], ldc,
+                         ws.data_ptr() if ws is not None else 0, workspace_bytes, torch.cuda.current_stream().cuda_stream)
+    assert rc == 0, mlt.status_string(rc)
+    assert_device_healthy()
+    bits = to_bits(Cbuf)
+    assert (bits[M:] == SENTINEL).all() and (bits[:M, N:] == SENTINEL).all(), "wrote outside C"
+    assert not (bits[:M, :N] == SENTINEL).any(), "unwritten output elements"
+    if ws is not None:
+        assert (ws[workspace_bytes:].cpu().numpy() == 0xAB).all(), "workspace overrun"
+    return inputs.bf16_bits_to_f64(bits[:M, :N]).reshape(M, N)
+
+
+SHAPES = [(1, 4096, 4096), (16, 4096, 4096), (7, 1000, 2056), (64, 520, 8192), (130, 264, 4100), (16, 4096, 520),
+          (512, 512, 512), (33, 6, 1024)]
+
+
+@pytest.mark.parametrize("M,N,K", SHAPES)
+def test_parity_skinny_and_ragged(M, N, K):
+    lda, ldb, ldc = (K + 7) // 8 * 8, (N + 7) // 8 * 8 + 8, (N + 7) // 8 * 8
+    A, B = inputs.gemm_inputs(M, N, K, seed=500 + M + N, kind="uniform", lda=lda, ldb=ldb)
+    need = mlt.gemm_workspace_bytes(M, N, K)
+    C = run_ex(A, B, M, N, K, ldc, need)
+    check_gemm(C, oracle.gemm(A, B, M, N, K), f"{M}x{N}x{K}")
+
+
+@pytest.mark.parametrize("fraction", [0.0, 0.26, 1.0])
+def test_any_workspace_size_is_correct(fraction):
+    M, N, K = 16, 1024, 4096
+    A, B = inputs.gemm_inputs(M, N, K, seed=510)
+    need = mlt.gemm_workspace_bytes(M, N, K)
+    assert need == 16 * M * N * 4           # 64 blocks of 64 -> at most 16 slices of 4
+    C = run_ex(A, B, M, N, K, N, int(need * fraction) // 16 * 16)
+    check_gemm(C, oracle.gemm(A, B, M, N, K), f"fraction {fraction}")
+
+
+def test_bit_exact_on_small_integers_and_deterministic():
+    M, N, K = 24, 776, 2048
+    A, B = inputs.gemm_inputs(M, N, K, seed=7, kind="ternary")
+    need = mlt.gemm_workspace_bytes(M, N, K)
+    C1 = run_ex(A, B, M, N, K, N, need)
+    ref = oracle.gemm(A, B, M, N, K)
+    assert np.abs(ref).max() <= 256 and np.array_equal(C1, ref)      # exact partial sums, exact final sum
+    assert np.array_equal(C1, run_ex(A, B, M, N, K, N, need))
+
+
+@pytest.mark.parametrize("name", list(inputs.GEMM_DECODE_CONFIGS))
+def test_decode_configs(name):
+    M, N, K, kind, seed = inputs.GEMM_DECODE_CONFIGS[name]
+    A, B = inputs.gemm_inputs(M, N, K, seed=seed, kind=kind)
+    C = run_ex(A, B, M, N, K, N, mlt.gemm_workspace_bytes(M, N, K))
+    rows = np.unique(np.linspace(0, M - 1, 8).astype(np.int64))
+    rel, mx = check_gemm(C[rows], oracle.gemm(A, B, M, N, K, rows=rows), name)
+    print(f"{name}: rel_fro={rel:.3e} max_abs/rms={mx:.3e}")
+
+
+def test_argument_errors():
+    x = torch.zeros(4096, dtype=torch.bfloat16, device="cuda")
+    p = x.data_ptr()
+    assert mlt.gemm_ex_raw(p, p, p, 8, 8, 8, 8, 8, 8, p + 4, 1024) == 3       # misaligned workspace
+    assert mlt.gemm_workspace_bytes(8192, 8192, 8192) == 0                     # plenty of tiles: no split
+    assert mlt.gemm_workspace_bytes(16, 4096, 256) == 0                        # K too short to cut
