@@ -475,6 +475,61 @@ def time_all_configs(mlt, torch, dev, stream, iters: int = 20, only: str | None 
     return out
 
 
+def run_sweeps(mlt, torch, dev, stream, iters: int = 10):
+    """Paper-shaped sweeps (Sec. 4.1 / 4.2): compute-bound GEMM with m = 1k..16k on Llama-like (n, k), and the
+    attention forward with 32k tokens in total, sequence length 1k..32k, hidden size 2048 as 32 heads of 64 or 16
+    heads of 128.  Synthetic N(0,1) data generated on the device (timing only; parity is the test suite's job)."""
+    sp = stream.cuda_stream
+    flush = torch.empty(256 << 20, dtype=torch.int8, device=dev)
+    rows = []
+
+    def best_ms(fn):
+        for _ in range(2):
+            fn()
+        ts = []
+        for _ in range(iters):
+            flush.zero_()
+            a, b = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+            a.record(stream)
+            fn()
+            b.record(stream)
+            torch.cuda.synchronize()
+            ts.append(a.elapsed_time(b))
+        return float(np.min(ts))
+
+    for (N, K) in ((4096, 4096), (14336, 4096), (4096, 14336), (8192, 8192)):
+        Bm = (torch.randn(K, N, device=dev) / np.sqrt(K)).to(torch.bfloat16)
+        for M in (1024, 2048, 4096, 8192, 16384):
+            A = (torch.randn(M, K, device=dev) / np.sqrt(K)).to(torch.bfloat16)
+            C = torch.empty(M, N, dtype=torch.bfloat16, device=dev)
+
+            def fn():
+                rc = mlt.gemm_raw(A.data_ptr(), Bm.data_ptr(), C.data_ptr(), M, N, K, K, N, N, sp)
+                assert rc == 0, rc
+            ms = best_ms(fn)
+            rows.append({"op": "gemm", "M": M, "N": N, "K": K, "ms": ms, "tflops": 2.0 * M * N * K / ms / 1e9})
+            del A, C
+        del Bm
+    for D, H in ((64, 32), (128, 16)):
+        for N in (1024, 2048, 4096, 8192, 16384, 32768):
+            Bn = 32768 // N
+            q = torch.randn(Bn, H, N, D, device=dev).to(torch.bfloat16)
+            k = torch.randn(Bn, H, N, D, device=dev).to(torch.bfloat16)
+            v = torch.randn(Bn, H, N, D, device=dev).to(torch.bfloat16)
+            o = torch.empty_like(q)
+            lse = torch.empty(Bn, H, N, dtype=torch.float32, device=dev)
+            for causal in (0, 1):
+                def fn():
+                    rc = mlt.mha_fwd_raw(q.data_ptr(), k.data_ptr(), v.data_ptr(), o.data_ptr(), lse.data_ptr(), Bn, H, N, N,
+                                         D, causal, float(D ** -0.5), sp)
+                    assert rc == 0, rc
+                ms = best_ms(fn)
+                rows.append({"op": "mha_fwd", "B": Bn, "H": H, "N": N, "D": D, "causal": causal, "ms": ms,
+                             "tflops": inputs.mha_flops(Bn, H, N, N, D, causal) / ms / 1e9})
+            del q, k, v, o, lse
+    return rows
+
+
 def main(argv=None):
     ap = argparse.ArgumentParser(description=__doc__, formatter_class=argparse.RawDescriptionHelpFormatter)
     ap.add_argument("--gpus", type=int, default=1)
@@ -482,8 +537,15 @@ def main(argv=None):
     ap.add_argument("--warmup", type=int, default=5)
     ap.add_argument("--impl", choices=["mlt", "reference"], default="mlt")
     ap.add_argument("--all", action="store_true", help="also time every benchmark configuration on its own")
+    ap.add_argument("--sweep", action="store_true", help="paper-shaped GEMM and attention sweeps (one JSON line)")
     ap.add_argument("--only", default=None, help="time one named configuration alone (kernel launches only; for profiling)")
     args = ap.parse_args(argv)
+    if args.sweep:
+        import torch
+        import paper_2503_14985_b200 as mlt
+        torch.cuda.set_device(0)
+        print(json.dumps({"sweep": run_sweeps(mlt, torch, torch.device("cuda", 0), torch.cuda.current_stream())}))
+        return 0
     if args.only is not None:
         import torch
         import paper_2503_14985_b200 as mlt
