@@ -46,6 +46,10 @@ def _load():
         i64, p, i32 = ctypes.c_int64, ctypes.c_void_p, ctypes.c_int
         lib.oracle_gemm.argtypes = [p, p, p, i64, i64, i64, i64, i64, p, i64, i32]
         lib.oracle_gemm.restype = i32
+        lib.oracle_gemm_f16.argtypes = [p, p, p, p, i64, i64, i64, i64, i64, i64, p, i64, i32]
+        lib.oracle_gemm_f16.restype = i32
+        lib.oracle_f16_to_double.argtypes = [p, p, i64]
+        lib.oracle_f16_to_double.restype = i32
         lib.oracle_mha_fwd.argtypes = [p, p, p, p, p, p, i32, i32, i32, i32, i32, i32, ctypes.c_float, p, i64, i32]
         lib.oracle_mha_fwd.restype = i32
         lib.oracle_hardware_threads.restype = i32
@@ -90,6 +94,49 @@ def gemm(A: np.ndarray, B: np.ndarray, M: int, N: int, K: int, *, rows=None, nth
                              out.ctypes.data, M, N, K, lda, ldb, rp, R, nthreads)
     if rc != 0:
         raise ValueError("oracle_gemm: invalid argument")
+    return out
+
+
+def f16_to_double(bits: np.ndarray) -> np.ndarray:
+    """Values of binary16 bit patterns, by the oracle's own field-by-field conversion."""
+    bits = np.ascontiguousarray(_u16(bits)).ravel()
+    out = np.empty(bits.size, dtype=np.float64)
+    if bits.size and _load().oracle_f16_to_double(bits.ctypes.data, out.ctypes.data, bits.size) != 0:
+        raise ValueError("oracle_f16_to_double: invalid argument")
+    return out
+
+
+def gemm_f16(A: np.ndarray, B: np.ndarray, M: int, N: int, K: int, *, C_in=None, rows=None,
+             nthreads: int = 0) -> np.ndarray:
+    """C = [C_in +] A @ B in FP64 over FP16 inputs (Listing 2 data types; Sec. 2 accumulate form).
+
+    A: (M, lda) uint16 binary16 patterns, B: (K, ldb) uint16; C_in: None or (M, ldc) float32.
+    rows: optional 1-D list of output rows; returns (len(rows) or M, N) float64.
+    """
+    A = np.ascontiguousarray(_u16(A))
+    B = np.ascontiguousarray(_u16(B))
+    lda = A.shape[1] if A.ndim == 2 and A.shape[0] > 0 else max(K, 1)
+    ldb = B.shape[1] if B.ndim == 2 and B.shape[0] > 0 else max(N, 1)
+    if A.size and A.shape[0] < M or B.size and B.shape[0] < K:
+        raise ValueError("array smaller than the stated shape")
+    cp, ldc = None, max(N, 1)
+    if C_in is not None:
+        C_in = np.ascontiguousarray(C_in, dtype=np.float32)
+        if C_in.ndim != 2 or C_in.shape[0] < M or C_in.shape[1] < N:
+            raise ValueError("C_in smaller than the stated shape")
+        cp, ldc = (C_in.ctypes.data if C_in.size else None), max(C_in.shape[1], 1)
+    if rows is not None:
+        rows = np.ascontiguousarray(rows, dtype=np.int64)
+        R, rp = len(rows), rows.ctypes.data
+    else:
+        R, rp = M, None
+    out = np.empty((R, N), dtype=np.float64)
+    if R == 0 or N == 0:
+        return out
+    rc = _load().oracle_gemm_f16(A.ctypes.data if A.size else None, B.ctypes.data if B.size else None, cp,
+                                 out.ctypes.data, M, N, K, lda, ldb, ldc, rp, R, nthreads)
+    if rc != 0:
+        raise ValueError("oracle_gemm_f16: invalid argument")
     return out
 
 

@@ -48,6 +48,19 @@ inline double bf16_to_double(uint16_t bits) {
     return static_cast<double>(f);
 }
 
+// IEEE 754 binary16 -> double, from the bit fields: 1 sign, 5 exponent (bias 15), 10 fraction bits.
+//   e = 0      : (-1)^s * f * 2^-24            (zero and subnormals)
+//   e = 1..30  : (-1)^s * (1024 + f) * 2^(e-25)
+//   e = 31     : infinity (f = 0) or NaN
+inline double f16_to_double(uint16_t bits) {
+    const int s = bits >> 15, e = (bits >> 10) & 31, f = bits & 1023;
+    double v;
+    if (e == 0) v = std::ldexp(static_cast<double>(f), -24);
+    else if (e == 31) v = f ? std::numeric_limits<double>::quiet_NaN() : std::numeric_limits<double>::infinity();
+    else v = std::ldexp(static_cast<double>(1024 + f), e - 25);
+    return s ? -v : v;
+}
+
 template <class F>
 void parallel_for(int64_t n, int nthreads, F&& body) {
     if (nthreads <= 0) nthreads = static_cast<int>(std::thread::hardware_concurrency());
@@ -98,6 +111,41 @@ int oracle_gemm(const uint16_t* A, const uint16_t* B, double* C_out,
             const uint16_t* b = B + k * ldb;
             for (int64_t j = 0; j < N; ++j) c[j] += a * bf16_to_double(b[j]);
         }
+    });
+    return 0;
+}
+
+// out[i] = value of the binary16 pattern in[i]  (test access to the conversion the FP16 GEMM uses).
+int oracle_f16_to_double(const uint16_t* in, double* out, int64_t n) {
+    if (n < 0) return 1;
+    for (int64_t i = 0; i < n; ++i) out[i] = f16_to_double(in[i]);
+    return 0;
+}
+
+// C_out[r][j] = (C_in ? C_in[rows[r]][j] : 0) + sum_{k<K} A[rows[r]][k] * B[k][j]
+//
+// The GEMM in the data types of Listing 2 (FP16 operands) with the accumulate form of Sec. 2 (C += A * B).
+// A, B: binary16 bit patterns, layouts as in oracle_gemm.  C_in: NULL, or the prior C as FP32, M x N row-major with
+// pitch ldc.  The product is summed first (k ascending) and the prior C added last.  rows / C_out as in oracle_gemm.
+int oracle_gemm_f16(const uint16_t* A, const uint16_t* B, const float* C_in, double* C_out,
+                    int64_t M, int64_t N, int64_t K, int64_t lda, int64_t ldb, int64_t ldc,
+                    const int64_t* rows, int64_t nrows, int nthreads) {
+    if (M < 0 || N < 0 || K < 0 || lda < K || ldb < N || (C_in && ldc < N)) return 1;
+    const int64_t R = rows ? nrows : M;
+    if (rows)
+        for (int64_t r = 0; r < R; ++r)
+            if (rows[r] < 0 || rows[r] >= M) return 1;
+    parallel_for(R, nthreads, [&](int64_t r) {
+        const int64_t i = rows ? rows[r] : r;
+        double* c = C_out + r * N;
+        for (int64_t j = 0; j < N; ++j) c[j] = 0.0;
+        for (int64_t k = 0; k < K; ++k) {
+            const double a = f16_to_double(A[i * lda + k]);
+            const uint16_t* b = B + k * ldb;
+            for (int64_t j = 0; j < N; ++j) c[j] += a * f16_to_double(b[j]);
+        }
+        if (C_in)
+            for (int64_t j = 0; j < N; ++j) c[j] += static_cast<double>(C_in[i * ldc + j]);
     });
     return 0;
 }

@@ -108,8 +108,11 @@ def outlier_rows(seed: int, tensor_id: int, nrows: int, percent: int = 1) -> np.
 
 def matrix_bf16(rows: int, cols: int, *, seed: int, tensor_id: int, kind: str = "normal",
                 scale: float = 1.0, ld: int | None = None, pad_bits: int = 0x7FC0,
-                row_scale: np.ndarray | None = None, chunk_rows: int | None = None) -> np.ndarray:
+                row_scale: np.ndarray | None = None, chunk_rows: int | None = None,
+                to_bits=None) -> np.ndarray:
     """rows x cols BF16 bit patterns in a (rows, ld) uint16 array.
+
+    `to_bits` replaces the FP64 -> BF16 rounding by another 16-bit encoder (see matrix_f16).
 
     Padding columns (ld > cols) hold `pad_bits` (a NaN pattern by default) so
     that any read of padding poisons a result.
@@ -129,7 +132,7 @@ def matrix_bf16(rows: int, cols: int, *, seed: int, tensor_id: int, kind: str = 
         v = v * scale
         if row_scale is not None:
             v = v * row_scale[r0:r1, None]
-        out[r0:r1, :cols] = f64_to_bf16_bits(v)
+        out[r0:r1, :cols] = (to_bits or f64_to_bf16_bits)(v)
 
     starts = range(0, rows, chunk_rows)
     if len(starts) > 4:  # every element depends only on its index: chunks can be filled by a few threads
@@ -141,6 +144,19 @@ def matrix_bf16(rows: int, cols: int, *, seed: int, tensor_id: int, kind: str = 
         for r0 in starts:
             fill(r0)
     return out
+
+
+def f64_to_f16_bits(v: np.ndarray) -> np.ndarray:
+    """FP64 values rounded to nearest-even binary16, as uint16 bit patterns."""
+    with np.errstate(over="ignore"):  # beyond 65520 rounds to infinity, as the format says
+        return np.asarray(v, dtype=np.float64).astype(np.float16).view(np.uint16)
+
+
+def matrix_f16(rows: int, cols: int, *, seed: int, tensor_id: int, kind: str = "normal", scale: float = 1.0,
+               ld: int | None = None) -> np.ndarray:
+    """matrix_bf16's values (same generator, same indices) rounded to binary16 instead; padding holds a NaN."""
+    return matrix_bf16(rows, cols, seed=seed, tensor_id=tensor_id, kind=kind, scale=scale, ld=ld, pad_bits=0x7E00,
+                       to_bits=f64_to_f16_bits)
 
 
 # --------------------------------------------------------------------------
@@ -155,6 +171,26 @@ def gemm_inputs(M: int, N: int, K: int, *, seed: int, kind: str = "normal", scal
     A = matrix_bf16(M, K, seed=seed, tensor_id=TENSOR_A, kind=kind, scale=scale, ld=lda)
     B = matrix_bf16(K, N, seed=seed, tensor_id=TENSOR_B, kind=kind, scale=scale, ld=ldb)
     return A, B
+
+
+TENSOR_C = 6
+
+
+def gemm_f16_inputs(M: int, N: int, K: int, *, seed: int, kind: str = "normal", scale: float | None = None,
+                    lda: int | None = None, ldb: int | None = None, ldc: int | None = None):
+    """A, B as binary16 bit patterns (layouts of gemm_inputs) and a prior C (M x ldc float32, N(0,1) values,
+    NaN in padding columns) for the accumulate form."""
+    if scale is None:
+        scale = 1.0 / np.sqrt(max(K, 1)) if kind == "normal" else 1.0
+    A = matrix_f16(M, K, seed=seed, tensor_id=TENSOR_A, kind=kind, scale=scale, ld=lda)
+    B = matrix_f16(K, N, seed=seed, tensor_id=TENSOR_B, kind=kind, scale=scale, ld=ldb)
+    ldc = N if ldc is None else ldc
+    C = np.full((M, ldc), np.nan, dtype=np.float32)
+    step = max(1, (1 << 20) // max(N, 1))
+    for r0 in range(0, M if N else 0, step):
+        r1 = min(M, r0 + step)
+        C[r0:r1, :N] = _values("normal", seed, TENSOR_C, r0 * N, (r1 - r0) * N).reshape(r1 - r0, N).astype(np.float32)
+    return A, B, C
 
 
 def mha_inputs(B: int, H: int, Nq: int, Nk: int, D: int, *, seed: int, outlier_percent: int = 0,
