@@ -414,6 +414,21 @@ def time_all_configs(mlt, torch, dev, stream, iters: int = 20, only: str | None 
             assert rc == 0, rc
         out[name] = timeit(fn, inputs.gemm_flops(M, N, K))
         del dA, dB, dC
+    # the same shapes in the data types of Listing 2 (FP16 operands, FP32 result), plain and as C += A * B
+    for base, (M, N, K, kind, seed) in inputs.GEMM_CONFIGS.items():
+        for acc in (0, 1):
+            name = base.replace("gemm_", "gemm_f16_acc_" if acc else "gemm_f16_")
+            if (only is not None and name != only) or base == "gemm_512":
+                continue
+            A, B, _ = inputs.gemm_f16_inputs(M, N, K, seed=seed, kind=kind, prior_c=False)
+            dA, dB = devbits(A), devbits(B)
+            dC = torch.zeros((M, N), dtype=torch.float32, device=dev)
+
+            def fn():
+                rc = mlt.gemm_f16_raw(dA.data_ptr(), dB.data_ptr(), dC.data_ptr(), M, N, K, K, N, N, acc, sp)
+                assert rc == 0, rc
+            out[name] = timeit(fn, inputs.gemm_flops(M, N, K))
+            del dA, dB, dC
     for name, (Bn, H, Nq, Nk, D, causal, seed, outl) in inputs.MHA_CONFIGS.items():
         if only is not None and name != only:
             continue

@@ -54,6 +54,21 @@ int mlt_gemm(const void* A, const void* B, void* C,
              void* stream);
 
 /*
+ * The GEMM in the data types of the paper's Listing 2 (FP16 operands, FP32 accumulator and FP32 result), with
+ * the accumulate form of the problem statement of Sec. 2 (C += A * B) as an option.
+ *
+ *   A, B   device, FP16 (bit patterns), layouts and pitches as for mlt_gemm
+ *   C      device, FP32, M x N row-major, pitch ldc in ELEMENTS, a multiple of 4; 16-byte aligned
+ *   accumulate  0: C = A * B (prior contents ignored);  non-zero: C = C + A * B, the product summed in FP32 first
+ *               and added to the prior C once
+ * K == 0: C is zero-filled, or left as it is when accumulating.  Errors as for mlt_gemm.
+ */
+int mlt_gemm_f16(const void* A, const void* B, float* C,
+                 int64_t M, int64_t N, int64_t K,
+                 int64_t lda, int64_t ldb, int64_t ldc,
+                 int accumulate, void* stream);
+
+/*
  * mlt_gemm with caller-provided scratch, for the memory-bound shapes of paper Sec. 4.1 (next-token prediction:
  * few rows of A against large weight matrices, "large k" and "large n" cases).  Such a problem has too few output
  * tiles to occupy the GPU, so K is cut into slices (split-K): every SM streams a part of B, FP32 partial tiles go

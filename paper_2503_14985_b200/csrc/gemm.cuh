@@ -38,7 +38,64 @@ struct GemmParams {
     int split_k;       // 1: no split, the epilogue writes BF16 C
     int kb_per_split;
     float* partial;
+    // FP16-input / FP32-output variant (the dtypes of the paper's Listing 2) and its accumulate form C += A*B
+    float* Cf;         // non-null: FP32 output with pitch ldcf instead of BF16 C
+    int64_t ldcf;
+    int accumulate;    // with Cf: add to the prior contents of C (the "C += A*B" of Sec. 2)
+    uint32_t f16_inputs;  // 0: BF16 operands, 1: FP16 operands (same tiles and descriptors, other format field)
 };
+
+// Instruction descriptor with the operand format chosen at run time (BF16: format 1, FP16: format 0).
+__device__ __forceinline__ uint32_t gemm_idesc(uint32_t m, uint32_t n, uint32_t f16_inputs) {
+    const uint32_t bf16 = make_idesc_bf16(m, n, /*a_mn_major=*/false, /*b_mn_major=*/true);
+    return f16_inputs ? (bf16 & ~((7u << 7) | (7u << 10))) : bf16;
+}
+
+// One row segment of 32 accumulator columns (TMEM -> registers) to its destination: the split-K FP32 partial, the
+// FP32 C (optionally added to what is there), or BF16 C.  Ragged right edges fall back to element stores.
+__device__ __forceinline__ void gemm_store_chunk(const GemmParams& p, const uint32_t (&v)[32], int row, int col0, int slice) {
+    if (row >= p.M) return;
+    float* frow = p.partial ? p.partial + (static_cast<int64_t>(slice) * p.M + row) * p.N
+                            : (p.Cf ? p.Cf + static_cast<int64_t>(row) * p.ldcf : nullptr);
+    if (frow) {
+        const bool add = !p.partial && p.accumulate;
+        const bool vec_ok = p.partial ? (p.N & 3) == 0 : true;  // partial rows are N floats apart; C rows are aligned
+#pragma unroll
+        for (int q = 0; q < 8; ++q) {
+            const int col = col0 + q * 4;
+            if (col + 4 <= p.N && vec_ok) {
+                float4 o = make_float4(__uint_as_float(v[q * 4]), __uint_as_float(v[q * 4 + 1]), __uint_as_float(v[q * 4 + 2]),
+                                       __uint_as_float(v[q * 4 + 3]));
+                if (add) {
+                    const float4 c = *reinterpret_cast<const float4*>(frow + col);
+                    o.x += c.x; o.y += c.y; o.z += c.z; o.w += c.w;
+                }
+                *reinterpret_cast<float4*>(frow + col) = o;
+            } else {
+                for (int j = 0; j < 4 && col + j < p.N; ++j)
+                    frow[col + j] = __uint_as_float(v[q * 4 + j]) + (add ? frow[col + j] : 0.0f);
+            }
+        }
+        return;
+    }
+    __nv_bfloat16* crow = p.C + static_cast<int64_t>(row) * p.ldc;
+#pragma unroll
+    for (int q = 0; q < 4; ++q) {
+        const int col = col0 + q * 8;
+        uint4 out;
+        out.x = pack_bf16x2(__uint_as_float(v[q * 8 + 0]), __uint_as_float(v[q * 8 + 1]));
+        out.y = pack_bf16x2(__uint_as_float(v[q * 8 + 2]), __uint_as_float(v[q * 8 + 3]));
+        out.z = pack_bf16x2(__uint_as_float(v[q * 8 + 4]), __uint_as_float(v[q * 8 + 5]));
+        out.w = pack_bf16x2(__uint_as_float(v[q * 8 + 6]), __uint_as_float(v[q * 8 + 7]));
+        if (col + 8 <= p.N) {
+            *reinterpret_cast<uint4*>(crow + col) = out;
+        } else if (col < p.N) {
+            const uint32_t w[4] = {out.x, out.y, out.z, out.w};
+            for (int j = 0; col + j < p.N; ++j)
+                crow[col + j] = __ushort_as_bfloat16(static_cast<unsigned short>(w[j >> 1] >> ((j & 1) * 16)));
+        }
+    }
+}
 
 // tile index -> (tile_m, tile_n): groups of `group_m` M-tiles, M fastest inside a group, so that
 // the CTAs running at the same time share few A and B panels (L2 reuse).
@@ -129,7 +186,7 @@ gemm_bf16_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_consta
         // one elected lane executes the tcgen05 instructions.
         {
             const bool leader = elect_one();
-            constexpr uint32_t idesc = make_idesc_bf16(kGemmBM, BN, /*a_mn_major=*/false, /*b_mn_major=*/true);
+            const uint32_t idesc = gemm_idesc(kGemmBM, BN, p.f16_inputs);
             const uint32_t a_lo0 = sdesc_lo(smem_u32(smem), 16);
             const uint32_t b_lo0 = sdesc_lo(smem_u32(smem + L::kABytes), kGemmBK * 128);
             int stage = 0;
@@ -179,44 +236,12 @@ gemm_bf16_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_consta
             if (!ok) break;
             tc_fence_after();
             const uint32_t t_row = tmem_base + (static_cast<uint32_t>(quarter * 32) << 16) + acc * BN;
-            __nv_bfloat16* crow = p.C + static_cast<int64_t>(row) * p.ldc;
-            float* prow = p.partial
-                              ? p.partial + (static_cast<int64_t>(item % p.split_k) * p.M + row) * p.N
-                              : nullptr;
 #pragma unroll 1
             for (int c = 0; c < BN / 32; ++c) {
                 uint32_t v[32];
                 tmem_ld_32x32b_x32(t_row + c * 32, v);
                 tmem_wait_ld();
-                const int col0 = n0 + c * 32;
-                if (row < p.M && prow) {  // split-K: the FP32 partial of this K slice
-#pragma unroll
-                    for (int q = 0; q < 8; ++q) {
-                        const int col = col0 + q * 4;
-                        if (col + 4 <= p.N && (p.N & 3) == 0) {
-                            *reinterpret_cast<uint4*>(prow + col) = make_uint4(v[q * 4], v[q * 4 + 1], v[q * 4 + 2], v[q * 4 + 3]);
-                        } else {
-                            for (int j = 0; j < 4 && col + j < p.N; ++j) prow[col + j] = __uint_as_float(v[q * 4 + j]);
-                        }
-                    }
-                } else if (row < p.M) {
-#pragma unroll
-                    for (int q = 0; q < 4; ++q) {
-                        const int col = col0 + q * 8;
-                        uint4 out;
-                        out.x = pack_bf16x2(__uint_as_float(v[q * 8 + 0]), __uint_as_float(v[q * 8 + 1]));
-                        out.y = pack_bf16x2(__uint_as_float(v[q * 8 + 2]), __uint_as_float(v[q * 8 + 3]));
-                        out.z = pack_bf16x2(__uint_as_float(v[q * 8 + 4]), __uint_as_float(v[q * 8 + 5]));
-                        out.w = pack_bf16x2(__uint_as_float(v[q * 8 + 6]), __uint_as_float(v[q * 8 + 7]));
-                        if (col + 8 <= p.N) {
-                            *reinterpret_cast<uint4*>(crow + col) = out;
-                        } else if (col < p.N) {
-                            const uint32_t w[4] = {out.x, out.y, out.z, out.w};
-                            for (int j = 0; col + j < p.N; ++j)
-                                crow[col + j] = __ushort_as_bfloat16(static_cast<unsigned short>(w[j >> 1] >> ((j & 1) * 16)));
-                        }
-                    }
-                }
+                gemm_store_chunk(p, v, row, n0 + c * 32, item % p.split_k);
             }
             tc_fence_before();
             __syncwarp();
@@ -338,7 +363,7 @@ gemm_bf16_pair_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_c
         if (leader) {
             // whole warp, uniform control flow; one elected lane executes the tcgen05 instructions
             const bool issuer = elect_one();
-            constexpr uint32_t idesc = make_idesc_bf16(kPairBM, kPairBN, /*a_mn_major=*/false, /*b_mn_major=*/true);
+            const uint32_t idesc = gemm_idesc(kPairBM, kPairBN, p.f16_inputs);
             const uint32_t a_lo0 = sdesc_lo(smem_u32(smem), 16);
             const uint32_t b_lo0 = sdesc_lo(smem_u32(smem + L::kABytes), kGemmBK * 128);
             int stage = 0;
@@ -386,31 +411,12 @@ gemm_bf16_pair_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_c
             if (!ok) break;
             tc_fence_after();
             const uint32_t t_row = tmem_base + (static_cast<uint32_t>(quarter * 32) << 16) + acc * kPairBN;
-            __nv_bfloat16* crow = p.C + static_cast<int64_t>(row) * p.ldc;
 #pragma unroll 1
             for (int c = 0; c < kPairBN / 32; ++c) {
                 uint32_t v[32];
                 tmem_ld_32x32b_x32(t_row + c * 32, v);
                 tmem_wait_ld();
-                const int col0 = n0 + c * 32;
-                if (row < p.M) {
-#pragma unroll
-                    for (int q = 0; q < 4; ++q) {
-                        const int col = col0 + q * 8;
-                        uint4 out;
-                        out.x = pack_bf16x2(__uint_as_float(v[q * 8 + 0]), __uint_as_float(v[q * 8 + 1]));
-                        out.y = pack_bf16x2(__uint_as_float(v[q * 8 + 2]), __uint_as_float(v[q * 8 + 3]));
-                        out.z = pack_bf16x2(__uint_as_float(v[q * 8 + 4]), __uint_as_float(v[q * 8 + 5]));
-                        out.w = pack_bf16x2(__uint_as_float(v[q * 8 + 6]), __uint_as_float(v[q * 8 + 7]));
-                        if (col + 8 <= p.N) {
-                            *reinterpret_cast<uint4*>(crow + col) = out;
-                        } else if (col < p.N) {
-                            const uint32_t w[4] = {out.x, out.y, out.z, out.w};
-                            for (int j = 0; col + j < p.N; ++j)
-                                crow[col + j] = __ushort_as_bfloat16(static_cast<unsigned short>(w[j >> 1] >> ((j & 1) * 16)));
-                        }
-                    }
-                }
+                gemm_store_chunk(p, v, row, n0 + c * 32, 0);
             }
             tc_fence_before();
             __syncwarp();
@@ -461,6 +467,13 @@ __global__ void gemm_splitk_reduce_kernel(const float* partial, __nv_bfloat16* C
             for (int j = 0; col + j < N; ++j) dst[j] = __float2bfloat16(acc[j]);
         }
     }
+}
+
+__global__ void gemm_zero_fill_f32_kernel(float* C, int64_t ldc, int M, int N) {
+    const int64_t total = static_cast<int64_t>(M) * N;
+    for (int64_t i = blockIdx.x * static_cast<int64_t>(blockDim.x) + threadIdx.x; i < total;
+         i += static_cast<int64_t>(gridDim.x) * blockDim.x)
+        C[(i / N) * ldc + (i % N)] = 0.0f;
 }
 
 // C[i][0..N) = 0 for K == 0 (BLAS convention for an empty sum).

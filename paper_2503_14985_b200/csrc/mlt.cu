@@ -77,7 +77,7 @@ int get_device(DeviceInfo* out) {
 
 // BF16 tensor map with 128-byte swizzle.  dims / strides innermost first; strides[0] is implicit.
 int encode_bf16(CUtensorMap* map, const void* base, int rank, const uint64_t* dims, const uint64_t* strides_bytes,
-                const uint32_t* box) {
+                const uint32_t* box, bool f16 = false) {
     EncodeTiledFn enc;
     int rc = get_encoder(&enc);
     if (rc != MLT_OK) return rc;
@@ -95,7 +95,7 @@ int encode_bf16(CUtensorMap* map, const void* base, int rank, const uint64_t* di
             gstride[i - 1] = strides_bytes[i - 1];
         }
     }
-    CUresult r = enc(map, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, static_cast<cuuint32_t>(rank), const_cast<void*>(base),
+    CUresult r = enc(map, f16 ? CU_TENSOR_MAP_DATA_TYPE_FLOAT16 : CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, static_cast<cuuint32_t>(rank), const_cast<void*>(base),
                      gdim, gstride, gbox, estr, CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B,
                      CU_TENSOR_MAP_L2_PROMOTION_L2_256B, CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
     return r == CUDA_SUCCESS ? MLT_OK : MLT_ERR_CUDA;
@@ -165,15 +165,17 @@ size_t mlt_gemm_workspace_bytes(int64_t M, int64_t N, int64_t K) {
     return split > 1 ? static_cast<size_t>(split) * M * N * sizeof(float) : 0;
 }
 
+// C is BF16 (f32_out false) or FP32 (f32_out true, optionally accumulating); A and B are BF16 or FP16.
 static int gemm_run(const void* A, const void* B, void* C, int64_t M, int64_t N, int64_t K, int64_t lda, int64_t ldb,
-                    int64_t ldc, void* workspace, size_t workspace_bytes, void* stream) {
+                    int64_t ldc, void* workspace, size_t workspace_bytes, void* stream, bool f16_in = false,
+                    bool f32_out = false, bool accumulate = false) {
     // ---- validation (no CUDA call before this block has passed) ----
     if (M < 0 || N < 0 || K < 0) return MLT_ERR_INVALID_ARG;
     if (M == 0 || N == 0) return MLT_OK;
     if (!C || ldc < N) return MLT_ERR_INVALID_ARG;
     if (K > 0 && (!A || !B || lda < K || ldb < N)) return MLT_ERR_INVALID_ARG;
     if (M > INT32_MAX - 256 || N > INT32_MAX - 256 || K > INT32_MAX - 256) return MLT_ERR_UNSUPPORTED;
-    if (!aligned16(C) || (ldc % 8) != 0) return MLT_ERR_ALIGNMENT;
+    if (!aligned16(C) || (ldc % (f32_out ? 4 : 8)) != 0) return MLT_ERR_ALIGNMENT;
     if (K > 0 && (!aligned16(A) || !aligned16(B) || (lda % 8) != 0 || (ldb % 8) != 0)) return MLT_ERR_ALIGNMENT;
     if (workspace && !aligned16(workspace)) return MLT_ERR_ALIGNMENT;
 
@@ -183,10 +185,15 @@ static int gemm_run(const void* A, const void* B, void* C, int64_t M, int64_t N,
     cudaStream_t st = static_cast<cudaStream_t>(stream);
 
     if (K == 0) {
+        if (f32_out && accumulate) return MLT_OK;  // C += empty sum
         const int64_t total = M * N;
         const int blocks = static_cast<int>(std::min<int64_t>((total + 255) / 256, 4 * dev.sm_count));
-        gemm_zero_fill_kernel<<<blocks, 256, 0, st>>>(static_cast<__nv_bfloat16*>(C), ldc, static_cast<int>(M),
-                                                      static_cast<int>(N));
+        if (f32_out)
+            gemm_zero_fill_f32_kernel<<<blocks, 256, 0, st>>>(static_cast<float*>(C), ldc, static_cast<int>(M),
+                                                              static_cast<int>(N));
+        else
+            gemm_zero_fill_kernel<<<blocks, 256, 0, st>>>(static_cast<__nv_bfloat16*>(C), ldc, static_cast<int>(M),
+                                                          static_cast<int>(N));
         return cudaGetLastError() == cudaSuccess ? MLT_OK : MLT_ERR_CUDA;
     }
 
@@ -213,14 +220,14 @@ static int gemm_run(const void* A, const void* B, void* C, int64_t M, int64_t N,
         const uint64_t dims[2] = {static_cast<uint64_t>(K), static_cast<uint64_t>(M)};
         const uint64_t strides[1] = {static_cast<uint64_t>(lda) * 2};
         const uint32_t box[2] = {kGemmBK, 128};
-        rc = encode_bf16(&ta, A, 2, dims, strides, box);
+        rc = encode_bf16(&ta, A, 2, dims, strides, box, f16_in);
         if (rc != MLT_OK) return rc;
     }
     {
         const uint64_t dims[2] = {static_cast<uint64_t>(N), static_cast<uint64_t>(K)};
         const uint64_t strides[1] = {static_cast<uint64_t>(ldb) * 2};
         const uint32_t box[2] = {64, kGemmBK};
-        rc = encode_bf16(&tb, B, 2, dims, strides, box);
+        rc = encode_bf16(&tb, B, 2, dims, strides, box, f16_in);
         if (rc != MLT_OK) return rc;
     }
 
@@ -235,7 +242,11 @@ static int gemm_run(const void* A, const void* B, void* C, int64_t M, int64_t N,
     p.split_k = 1;
     p.kb_per_split = static_cast<int>((K + kGemmBK - 1) / kGemmBK);
     p.partial = nullptr;
-    if (variant == 2 && workspace) {
+    p.Cf = f32_out ? static_cast<float*>(C) : nullptr;
+    p.ldcf = ldc;
+    p.accumulate = accumulate ? 1 : 0;
+    p.f16_inputs = f16_in ? 1u : 0u;
+    if (variant == 2 && workspace && !f32_out) {
         // Few tiles (skinny or small problem): cut K into slices so that about two work items per SM exist; the
         // weights are then streamed by all SMs at once.  FP32 partials go to the caller's scratch.
         const int num_kb = p.kb_per_split;
@@ -273,6 +284,12 @@ static int gemm_run(const void* A, const void* B, void* C, int64_t M, int64_t N,
 int mlt_gemm(const void* A, const void* B, void* C, int64_t M, int64_t N, int64_t K, int64_t lda, int64_t ldb,
              int64_t ldc, void* stream) {
     return gemm_run(A, B, C, M, N, K, lda, ldb, ldc, nullptr, 0, stream);
+}
+
+int mlt_gemm_f16(const void* A, const void* B, float* C, int64_t M, int64_t N, int64_t K, int64_t lda, int64_t ldb,
+                 int64_t ldc, int accumulate, void* stream) {
+    return gemm_run(A, B, C, M, N, K, lda, ldb, ldc, nullptr, 0, stream, /*f16_in=*/true, /*f32_out=*/true,
+                    accumulate != 0);
 }
 
 int mlt_gemm_ex(const void* A, const void* B, void* C, int64_t M, int64_t N, int64_t K, int64_t lda, int64_t ldb,

@@ -177,13 +177,15 @@ TENSOR_C = 6
 
 
 def gemm_f16_inputs(M: int, N: int, K: int, *, seed: int, kind: str = "normal", scale: float | None = None,
-                    lda: int | None = None, ldb: int | None = None, ldc: int | None = None):
+                    lda: int | None = None, ldb: int | None = None, ldc: int | None = None, prior_c: bool = True):
     """A, B as binary16 bit patterns (layouts of gemm_inputs) and a prior C (M x ldc float32, N(0,1) values,
-    NaN in padding columns) for the accumulate form."""
+    NaN in padding columns; None if not `prior_c`) for the accumulate form."""
     if scale is None:
         scale = 1.0 / np.sqrt(max(K, 1)) if kind == "normal" else 1.0
     A = matrix_f16(M, K, seed=seed, tensor_id=TENSOR_A, kind=kind, scale=scale, ld=lda)
     B = matrix_f16(K, N, seed=seed, tensor_id=TENSOR_B, kind=kind, scale=scale, ld=ldb)
+    if not prior_c:
+        return A, B, None
     ldc = N if ldc is None else ldc
     C = np.full((M, ldc), np.nan, dtype=np.float32)
     step = max(1, (1 << 20) // max(N, 1))
