@@ -45,20 +45,23 @@ struct MhaSmem {
     static constexpr int kChunkBytes = kMhaBlock * 128;
     static constexpr int kStages = (D == 128) ? 4 : 8;
     static constexpr int kBarrierBytes = 512;
-    static constexpr int kTotal = 2 * kTileBytes + kStages * kTileBytes + kBarrierBytes + 1024;
+    static constexpr int kItemSlots = 64;       // work items decoded ahead of time (16 bytes each)
+    static constexpr int kStageBytes = 8 * 4096;  // output staging: 4 KB per softmax warp
+    static constexpr int kTotal =
+        2 * kTileBytes + kStages * kTileBytes + kBarrierBytes + kItemSlots * 16 + kStageBytes + 1024;
 };
 
 struct MhaParams {
-    __nv_bfloat16* O;
     float* LSE;  // may be null
     int BH, Nq, Nk;
     int causal;
     float scale;
     int num_pairs;   // 256-row query groups per head
-    int head_group;  // heads that share a span of consecutive block indices
+    int head_group;  // heads that share a span of consecutive item indices
+    int num_items;   // num_pairs * BH
 };
 
-// block index -> (pair, bh).  Heads are taken in groups; inside a group the query
+// item index -> (pair, bh).  Heads are taken in groups; inside a group the query
 // position is the slow index and runs from the last rows to the first, so under a
 // causal mask the longest items are dispatched first, and the CTAs resident at any
 // time read the K/V of few heads (L2 reuse).
@@ -94,7 +97,8 @@ __device__ __forceinline__ float2 exp2_poly2(float2 x) {
 template <int D>
 __global__ void __launch_bounds__(kMhaThreads, 1)
 mha_fwd_kernel(const __grid_constant__ CUtensorMap tmap_q, const __grid_constant__ CUtensorMap tmap_k,
-               const __grid_constant__ CUtensorMap tmap_v, const MhaParams p) {
+               const __grid_constant__ CUtensorMap tmap_v, const __grid_constant__ CUtensorMap tmap_o,
+               const MhaParams p) {
     using L = MhaSmem<D>;
     constexpr int kStages = L::kStages;
     constexpr int kChunks = D / 64;
@@ -102,43 +106,98 @@ mha_fwd_kernel(const __grid_constant__ CUtensorMap tmap_q, const __grid_constant
     uint8_t* smem = reinterpret_cast<uint8_t*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~uintptr_t(1023));
     uint8_t* smem_q = smem;                        // [2][tile]
     uint8_t* smem_kv = smem + 2 * L::kTileBytes;   // [kStages][tile]
-    uint64_t* bars = reinterpret_cast<uint64_t*>(smem_kv + kStages * L::kTileBytes);
+    uint8_t* smem_stage = smem_kv + kStages * L::kTileBytes;  // [8 warps][4 KB], 1024-byte aligned (TMA swizzle atoms)
+    uint64_t* bars = reinterpret_cast<uint64_t*>(smem_stage + L::kStageBytes);
     uint64_t* q_full = bars;                  // [1]
     uint64_t* kv_full = bars + 1;             // [kStages]
     uint64_t* kv_empty = kv_full + kStages;   // [kStages]
     uint64_t* s_full = kv_empty + kStages;    // [2]  UMMA -> softmax: S_t(j) complete
     uint64_t* p_full = s_full + 2;            // [2]  softmax -> UMMA: P_t(j) in TMEM, O_t rescaled
     uint64_t* o_full = p_full + 2;            // [2]  UMMA -> epilogue: O_t complete
-    uint32_t* tmem_base_slot = reinterpret_cast<uint32_t*>(o_full + 2);
+    uint64_t* q_empty = o_full + 2;           // [1]  UMMA -> loader: the item's last Q K^T has read the Q tiles
+    uint32_t* tmem_base_slot = reinterpret_cast<uint32_t*>(q_empty + 1);
     volatile uint32_t* abort_flag = tmem_base_slot + 1;
 
     const int warp = threadIdx.x >> 5;
     const int lane = threadIdx.x & 31;
 
-    int pair, bh;
-    mha_item(p, blockIdx.x, pair, bh);
-    const int q_base = pair * 2 * kMhaBlock;
+    // Work items of this CTA: item list position r * gridDim.x + (c or gridDim.x - 1 - c), the direction alternating
+    // from round to round, so that with the list sorted by length the CTAs' sums stay within about one item.
+    const int G = static_cast<int>(gridDim.x);
+    const int rounds = (p.num_items + G - 1) / G;
     const int shift = p.Nk - p.Nq;  // bottom-right alignment of the causal mask
-    // number of K/V blocks each tile needs
-    int J[2];
+    struct Item {
+        int q_base, bh, J[2], Jmax;
+    };
+    auto decode_item = [&](int r, Item& it) -> bool {
+        const int idx = r * G + ((r & 1) ? G - 1 - static_cast<int>(blockIdx.x) : static_cast<int>(blockIdx.x));
+        if (r >= rounds || idx >= p.num_items) return false;
+        int pair;
+        mha_item(p, idx, pair, it.bh);
+        it.q_base = pair * 2 * kMhaBlock;
 #pragma unroll
-    for (int t = 0; t < 2; ++t) {
-        const int q0 = q_base + t * kMhaBlock;
-        if (q0 >= p.Nq) {
-            J[t] = 0;
-        } else {
-            int last_key = p.Nk - 1;
-            if (p.causal) last_key = min(last_key, min(q0 + kMhaBlock, p.Nq) - 1 + shift);
-            J[t] = last_key / kMhaBlock + 1;
+        for (int t = 0; t < 2; ++t) {  // number of K/V blocks each tile needs
+            const int q0 = it.q_base + t * kMhaBlock;
+            if (q0 >= p.Nq) {
+                it.J[t] = 0;
+            } else {
+                int last_key = p.Nk - 1;
+                if (p.causal) last_key = min(last_key, min(q0 + kMhaBlock, p.Nq) - 1 + shift);
+                it.J[t] = last_key / kMhaBlock + 1;
+            }
         }
+        it.Jmax = max(it.J[0], it.J[1]);
+        return true;
+    };
+    // The first kItemSlots items of this CTA are decoded once, one per thread, into shared memory before the
+    // CTA-wide sync: the issuing and loading warps share their scheduler partitions with the softmax warps and
+    // get few issue slots, so the divisions of the decode would cost them thousands of clocks per item.
+    int4* item_table = reinterpret_cast<int4*>(reinterpret_cast<uint8_t*>(bars) + L::kBarrierBytes);
+    if (threadIdx.x < L::kItemSlots) {
+        Item it;
+        const bool have = decode_item(threadIdx.x, it);
+        item_table[threadIdx.x] = have ? make_int4(it.q_base, it.bh, it.J[0], it.J[1]) : make_int4(0, 0, 0, 0);
     }
-    const int Jmax = max(J[0], J[1]);
+    auto item_at = [&](int r, Item& it) -> bool {  // valid after the CTA-wide sync
+        if (r >= L::kItemSlots) return decode_item(r, it);
+        const int4 e = item_table[r];
+        it.q_base = e.x;
+        it.bh = e.y;
+        it.J[0] = e.z;
+        it.J[1] = e.w;
+        it.Jmax = max(e.z, e.w);
+        return it.Jmax > 0;
+    };
 
-    // The loader lane initialises the barriers and issues the first loads (Q and the first K/V tiles: the ring
-    // is empty, nothing to wait for) before the CTA-wide sync, so they overlap the tensor-memory allocation.
-    int pre_tiles = 0;  // ring tiles already requested (K_0, V_0, K_1, ...)
+    // loader state: ring position and the number of Q loads so far
+    int ld_stage = 0;
+    uint32_t ld_phase = 0;
+    auto load_q = [&](const Item& it) {
+        mbar_arrive_expect_tx(q_full, 2 * L::kTileBytes);
+#pragma unroll
+        for (int t = 0; t < 2; ++t)
+#pragma unroll
+            for (int c = 0; c < kChunks; ++c)
+                tma_load_3d(smem_q + t * L::kTileBytes + c * L::kChunkBytes, &tmap_q, q_full, c * 64,
+                            it.q_base + t * kMhaBlock, it.bh);
+    };
+    auto load_kv = [&](const Item& it, int i) {  // ring tile i of the item: K_0, V_0, K_1, V_1, ...
+        uint8_t* dst = smem_kv + ld_stage * L::kTileBytes;
+        mbar_arrive_expect_tx(&kv_full[ld_stage], L::kTileBytes);
+#pragma unroll
+        for (int c = 0; c < kChunks; ++c)
+            tma_load_3d(dst + c * L::kChunkBytes, (i & 1) == 0 ? &tmap_k : &tmap_v, &kv_full[ld_stage], c * 64,
+                        (i >> 1) * kMhaBlock, it.bh);
+        if (++ld_stage == kStages) { ld_stage = 0; ld_phase ^= 1; }
+    };
+
+    // The loader lane initialises the barriers and issues the first loads (Q and the first K/V tiles of the first
+    // item: the ring is empty, nothing to wait for) before the CTA-wide sync, so they overlap the tensor-memory
+    // allocation.
+    int pre_tiles = 0;  // ring tiles of the first item already requested
     if (warp == 9 && lane == 0) {
         mbar_init(q_full, 1);
+        mbar_init(q_empty, 1);
         for (int s = 0; s < kStages; ++s) {
             mbar_init(&kv_full[s], 1);
             mbar_init(&kv_empty[s], 1);
@@ -153,24 +212,15 @@ mha_fwd_kernel(const __grid_constant__ CUtensorMap tmap_q, const __grid_constant
         prefetch_tensormap(&tmap_q);
         prefetch_tensormap(&tmap_k);
         prefetch_tensormap(&tmap_v);
-        // K_0 first: with Q it is all the first product needs
-        pre_tiles = min(2 * Jmax, kStages);
-        for (int i = 0; i < pre_tiles; ++i) {
-            if (i == 1) {
-                mbar_arrive_expect_tx(q_full, 2 * L::kTileBytes);
-#pragma unroll
-                for (int t = 0; t < 2; ++t)
-#pragma unroll
-                    for (int c = 0; c < kChunks; ++c)
-                        tma_load_3d(smem_q + t * L::kTileBytes + c * L::kChunkBytes, &tmap_q, q_full, c * 64,
-                                    q_base + t * kMhaBlock, bh);
+        prefetch_tensormap(&tmap_o);
+        Item it;
+        if (decode_item(0, it)) {
+            // K_0 first: with Q it is all the first product needs
+            pre_tiles = min(2 * it.Jmax, kStages);
+            for (int i = 0; i < pre_tiles; ++i) {
+                if (i == 1) load_q(it);
+                load_kv(it, i);
             }
-            uint8_t* dst = smem_kv + i * L::kTileBytes;
-            mbar_arrive_expect_tx(&kv_full[i], L::kTileBytes);
-#pragma unroll
-            for (int c = 0; c < kChunks; ++c)
-                tma_load_3d(dst + c * L::kChunkBytes, (i & 1) == 0 ? &tmap_k : &tmap_v, &kv_full[i], c * 64,
-                            (i >> 1) * kMhaBlock, bh);
         }
     }
     if (warp == 8) {
@@ -190,19 +240,20 @@ mha_fwd_kernel(const __grid_constant__ CUtensorMap tmap_q, const __grid_constant
         // ------------------------------- loader -------------------------------
         setmaxnreg_dec<40>();
         if (lane == 0) {
-            int stage = pre_tiles == kStages ? 0 : pre_tiles;
-            uint32_t phase = pre_tiles == kStages ? 1 : 0;
             bool ok = true;
-            for (int i = pre_tiles; i < 2 * Jmax && ok; ++i) {
-                ok = mbar_wait(&kv_empty[stage], phase ^ 1, abort_flag, 0x100 + stage);
-                if (!ok) break;
-                uint8_t* dst = smem_kv + stage * L::kTileBytes;
-                mbar_arrive_expect_tx(&kv_full[stage], L::kTileBytes);
-#pragma unroll
-                for (int c = 0; c < kChunks; ++c)
-                    tma_load_3d(dst + c * L::kChunkBytes, (i & 1) == 0 ? &tmap_k : &tmap_v, &kv_full[stage], c * 64,
-                                (i >> 1) * kMhaBlock, bh);
-                if (++stage == kStages) { stage = 0; phase ^= 1; }
+            Item it;
+            for (int r = 0; ok && item_at(r, it); ++r) {
+                for (int i = (r == 0 ? pre_tiles : 0); i < 2 * it.Jmax && ok; ++i) {
+                    if (i == 1 && r > 0) {
+                        // Q of the next item: the tiles are free once the previous item's last Q K^T has completed
+                        ok = mbar_wait(q_empty, (r - 1) & 1, abort_flag, 0x110);
+                        if (!ok) break;
+                        load_q(it);
+                    }
+                    ok = mbar_wait(&kv_empty[ld_stage], ld_phase ^ 1, abort_flag, 0x100 + ld_stage);
+                    if (!ok) break;
+                    load_kv(it, i);
+                }
             }
         }
     } else if (warp == 8) {
@@ -253,47 +304,57 @@ mha_fwd_kernel(const __grid_constant__ CUtensorMap tmap_q, const __grid_constant
             };
             int stage = 0;
             uint32_t phase = 0;
+            uint32_t n_p[2] = {0, 0};  // P tiles consumed so far, per query tile (parity of p_full)
             bool ok = true;
-            if (Jmax > 0) {
-                ok = wait_all(q_full, 0, 0x200);
-                if (ok) ok = wait_all(&kv_full[stage], phase, 0x210 + stage);
-                if (ok) {
-                    tc_fence_after();
-                    for (int t = 0; t < 2; ++t)
-                        if (J[t] > 0) issue_qk(t, stage);
-                    if (leader) umma_commit(&kv_empty[stage]);
-                    if (++stage == kStages) { stage = 0; phase ^= 1; }
-                }
-            }
-            for (int j = 0; j < Jmax && ok; ++j) {
-                const int vslot = stage;
-                ok = wait_all(&kv_full[vslot], phase, 0x220 + vslot);
-                if (!ok) break;
-                if (++stage == kStages) { stage = 0; phase ^= 1; }
-                const int kslot = stage;  // K_{j+1}, if there is one
-                bool k_ready = false;
-                for (int t = 0; t < 2 && ok; ++t) {
-                    if (j >= J[t]) continue;
-                    ok = wait_all(&p_full[t], j & 1, 0x230 + t);
-                    if (!ok) break;
-                    tc_fence_after();
-                    issue_pv(t, vslot, j == 0);
-                    if (j == J[t] - 1 && leader) umma_commit(&o_full[t]);
-                    if (j + 1 < J[t]) {
-                        if (!k_ready) {
-                            ok = wait_all(&kv_full[kslot], phase, 0x240 + kslot);
-                            if (!ok) break;
-                            tc_fence_after();
-                            k_ready = true;
-                        }
-                        issue_qk(t, kslot);
+            Item it;
+            for (int r = 0; ok && item_at(r, it); ++r) {
+                const int Jmax = it.Jmax;
+                ok = wait_all(q_full, r & 1, 0x200);
+                // Step j issues P_t(j) V_j and then Q_t K_{j+1}^T for both tiles; step -1 issues only the first
+                // Q K^T products, through the same instructions as every other step (code that runs once per item
+                // would be fetched cold each time).  S_t(0) may overwrite P_t of the previous item: the tensor
+                // pipe runs the products in issue order.
+#pragma unroll 1
+                for (int j = -1; j < Jmax && ok; ++j) {
+                    int vslot = 0;
+                    if (j >= 0) {
+                        vslot = stage;
+                        ok = wait_all(&kv_full[vslot], phase, 0x220 + vslot);
+                        if (!ok) break;
+                        if (++stage == kStages) { stage = 0; phase ^= 1; }
                     }
-                }
-                if (!ok) break;
-                if (leader) umma_commit(&kv_empty[vslot]);
-                if (j + 1 < Jmax) {
-                    if (leader) umma_commit(&kv_empty[kslot]);
-                    if (++stage == kStages) { stage = 0; phase ^= 1; }
+                    const int kslot = stage;  // K_{j+1}, if there is one
+                    bool k_ready = false;
+                    for (int t = 0; t < 2 && ok; ++t) {
+                        if (j >= 0 && j < it.J[t]) {
+                            // P_t(0) of an item also tells that the softmax warps have read the previous item's O_t
+                            ok = wait_all(&p_full[t], n_p[t] & 1, 0x230 + t);
+                            if (!ok) break;
+                            ++n_p[t];
+                            tc_fence_after();
+                            issue_pv(t, vslot, j == 0);
+                            if (j == it.J[t] - 1 && leader) umma_commit(&o_full[t]);
+                        }
+                        if (j + 1 < it.J[t]) {
+                            if (!k_ready) {
+                                ok = wait_all(&kv_full[kslot], phase, 0x240 + kslot);
+                                if (!ok) break;
+                                tc_fence_after();
+                                k_ready = true;
+                            }
+                            issue_qk(t, kslot);
+                        }
+                    }
+                    if (!ok) break;
+                    if (leader) {
+                        if (j >= 0) umma_commit(&kv_empty[vslot]);
+                        if (j + 1 < Jmax) umma_commit(&kv_empty[kslot]);
+                        if (j + 2 == Jmax) umma_commit(q_empty);  // the item's last Q K^T products are issued
+                    }
+                    __syncwarp();
+                    if (j + 1 < Jmax) {
+                        if (++stage == kStages) { stage = 0; phase ^= 1; }
+                    }
                 }
             }
         }
@@ -303,20 +364,25 @@ mha_fwd_kernel(const __grid_constant__ CUtensorMap tmap_q, const __grid_constant
         const int t = warp >> 2;
         const int quarter = warp & 3;
         const int row_in_tile = quarter * 32 + lane;
-        const int qi = q_base + t * kMhaBlock + row_in_tile;  // query index inside the head
         const uint32_t lane_addr = tmem_base + (static_cast<uint32_t>(quarter * 32) << 16);
         const uint32_t s_addr = lane_addr + kColS + t * kMhaBlock;
         const uint32_t o_addr = lane_addr + kColO + t * D;
         const float c = p.scale * kLog2e;
-        const int Jt = J[t];
-        const int limit = p.causal ? min(p.Nk - 1, qi + shift) : p.Nk - 1;  // last visible key of this row
-        float m_run = -INFINITY;  // reference max (raw score units); may lag the true max by < 2^8 in exp2 units
-        float l_run = 0.0f;
+        uint32_t n_s = 0, n_o = 0;  // S tiles and O tiles taken so far (parities of s_full / o_full)
         bool ok = true;
+        Item it;
+        for (int r = 0; ok && item_at(r, it); ++r) {
+        const int Jt = it.J[t];
+        if (Jt == 0) continue;  // this tile lies beyond the last query row
+        const int qi = it.q_base + t * kMhaBlock + row_in_tile;  // query index inside the head
+        const int limit = p.causal ? min(p.Nk - 1, qi + shift) : p.Nk - 1;  // last visible key of this row
+        float m_run = -INFINITY;  // reference max (raw score units), taken from the row's first block
+        float l_run = 0.0f;
 
         for (int j = 0; j < Jt; ++j) {
-            ok = __all_sync(0xffffffffu, mbar_wait(&s_full[t], j & 1, abort_flag, 0x300 + t));
+            ok = __all_sync(0xffffffffu, mbar_wait(&s_full[t], n_s & 1, abort_flag, 0x300 + t));
             if (!ok) break;
+            ++n_s;
             tc_fence_after();
             uint32_t s[4][32];  // this thread's row of S: 4 chunks of 32 keys
 #pragma unroll
@@ -375,11 +441,10 @@ mha_fwd_kernel(const __grid_constant__ CUtensorMap tmap_q, const __grid_constant
                     if (w & 1) tmem_st_32x32b_x16(s_addr + (w >> 1) * 16, pk);
                 }
             };
-            if (j == 0) {
-                m_run = row_max();  // no reference yet
-                exp_pass((m_run == -INFINITY) ? 0.0f : -m_run * c);
-            } else {
-                exp_pass((m_run == -INFINITY) ? 0.0f : -m_run * c);
+            // The first block of a row takes its max first and then runs the same pass as every other block.
+            if (j == 0) m_run = row_max();
+            exp_pass((m_run == -INFINITY) ? 0.0f : -m_run * c);
+            if (j > 0) {
                 const float blk = (acc0.x + acc0.y) + (acc1.x + acc1.y);
                 const bool moved = !(blk < kRescaleLimit);  // also catches inf and NaN
                 if (__any_sync(0xffffffffu, moved)) {
@@ -411,46 +476,51 @@ mha_fwd_kernel(const __grid_constant__ CUtensorMap tmap_q, const __grid_constant
             if (lane == 0) mbar_arrive(&p_full[t]);
         }
 
-        if (ok && Jt > 0) {
-            ok = __all_sync(0xffffffffu, mbar_wait(&o_full[t], 0, abort_flag, 0x400 + t));
-            if (ok) {
-                tc_fence_after();
-                const float inv_l = 1.0f / l_run;
-                const bool valid = qi < p.Nq;
-                // O / l -> BF16 into the tile's Q region (no product reads it any more), 16-byte chunks XOR-swizzled
-                // by row; then each warp writes its own 32 rows out row-major, 512 contiguous bytes per instruction.
-                constexpr int kRowChunks = D / 8;  // 16-byte chunks per row
-                uint8_t* stage_o = smem_q + t * L::kTileBytes;
-                {
-                    uint32_t o[D / 32][32];  // the whole row at once: one TMEM round trip instead of eight
-#pragma unroll
-                    for (int q = 0; q < D / 32; ++q) tmem_ld_32x32b_x32(o_addr + q * 32, o[q]);
-                    tmem_wait_ld();
-#pragma unroll
-                    for (int k = 0; k < D / 8; ++k) {  // 16-byte chunks of the BF16 row
-                        const uint32_t* w = &o[k >> 2][(k & 3) * 8];
-                        uint4 out;
-                        out.x = pack_bf16x2(__uint_as_float(w[0]) * inv_l, __uint_as_float(w[1]) * inv_l);
-                        out.y = pack_bf16x2(__uint_as_float(w[2]) * inv_l, __uint_as_float(w[3]) * inv_l);
-                        out.z = pack_bf16x2(__uint_as_float(w[4]) * inv_l, __uint_as_float(w[5]) * inv_l);
-                        out.w = pack_bf16x2(__uint_as_float(w[6]) * inv_l, __uint_as_float(w[7]) * inv_l);
-                        const int chunk = k ^ (row_in_tile & (kRowChunks - 1));
-                        *reinterpret_cast<uint4*>(stage_o + row_in_tile * (D * 2) + chunk * 16) = out;
-                    }
-                }
+        if (!ok) break;
+        ok = __all_sync(0xffffffffu, mbar_wait(&o_full[t], n_o & 1, abort_flag, 0x400 + t));
+        if (!ok) break;
+        ++n_o;
+        tc_fence_after();
+        {
+            // Once the loads from tensor memory have completed the next item's first P V may overwrite O_t: the
+            // softmax of that item, and with it P_t(0), comes after this point in program order.
+            const float inv_l = __fdividef(1.0f, l_run);
+            const bool valid = qi < p.Nq;
+            // 64 columns at a time: BF16 into this warp's 4 KB staging area (32 rows x 128 B in the 128-byte
+            // swizzle of the tensor map: 16-byte chunk k of row r sits at chunk k ^ (r & 7)), then one TMA store
+            // of the 32 x 64 box; rows beyond Nq are clipped by the tensor map.
+            uint8_t* stage_o = smem_stage + warp * 4096;
+            const int row0 = it.q_base + t * kMhaBlock + quarter * 32;  // first query row of this warp
+#pragma unroll 1
+            for (int h = 0; h < D / 64; ++h) {  // a short loop, not unrolled: this code runs once per item
+                uint32_t o[2][32];
+                tmem_ld_32x32b_x32(o_addr + h * 64, o[0]);
+                tmem_ld_32x32b_x32(o_addr + h * 64 + 32, o[1]);
+                if (lane == 0) tma_store_wait_read<0>();  // the staging area's previous store has been read out
                 __syncwarp();
-                constexpr int kRowsPerStore = 32 / kRowChunks;
-                __nv_bfloat16* obase = p.O + (static_cast<int64_t>(bh) * p.Nq + q_base + t * kMhaBlock) * D;
+                tmem_wait_ld();
 #pragma unroll
-                for (int r0 = 0; r0 < 32; r0 += kRowsPerStore) {
-                    const int rr = quarter * 32 + r0 + lane / kRowChunks;
-                    const int cc = lane % kRowChunks;
-                    const uint4 v = *reinterpret_cast<const uint4*>(stage_o + rr * (D * 2) + ((cc ^ (rr & (kRowChunks - 1))) * 16));
-                    if (q_base + t * kMhaBlock + rr < p.Nq) *reinterpret_cast<uint4*>(obase + rr * D + cc * 8) = v;
+                for (int k = 0; k < 8; ++k) {  // 16-byte chunks of the BF16 half row
+                    const uint32_t* w = &o[k >> 2][(k & 3) * 8];
+                    uint4 out;
+                    out.x = pack_bf16x2(__uint_as_float(w[0]) * inv_l, __uint_as_float(w[1]) * inv_l);
+                    out.y = pack_bf16x2(__uint_as_float(w[2]) * inv_l, __uint_as_float(w[3]) * inv_l);
+                    out.z = pack_bf16x2(__uint_as_float(w[4]) * inv_l, __uint_as_float(w[5]) * inv_l);
+                    out.w = pack_bf16x2(__uint_as_float(w[6]) * inv_l, __uint_as_float(w[7]) * inv_l);
+                    *reinterpret_cast<uint4*>(stage_o + lane * 128 + ((k ^ (lane & 7)) * 16)) = out;
                 }
-                if (valid && p.LSE) p.LSE[static_cast<int64_t>(bh) * p.Nq + qi] = m_run * p.scale + logf(l_run);
+                fence_proxy_async_smem();
+                __syncwarp();
+                if (lane == 0 && row0 < p.Nq) {
+                    tma_store_3d(&tmap_o, stage_o, h * 64, row0, it.bh);
+                    tma_store_commit();
+                }
             }
+            if (valid && p.LSE)
+                p.LSE[static_cast<int64_t>(it.bh) * p.Nq + qi] = m_run * p.scale + __log2f(l_run) * 0.6931471805599453f;
         }
+        }  // items
+        if (lane == 0) tma_store_wait_all<0>();  // shared memory must outlive the stores that read it
     }
 
     // common exit: every role reaches this, also after an aborted wait
@@ -473,11 +543,10 @@ inline int mha_configure() {
     return 0;
 }
 
-inline int mha_launch(const CUtensorMap& tq, const CUtensorMap& tk, const CUtensorMap& tv, __nv_bfloat16* O, float* LSE,
-                      int B, int H, int Nq, int Nk, int D, bool causal, float scale, int sm_count, cudaStream_t st) {
-    (void)sm_count;
+inline int mha_launch(const CUtensorMap& tq, const CUtensorMap& tk, const CUtensorMap& tv, const CUtensorMap& to, float* LSE,
+                      int B, int H, int Nq, int Nk, int D, bool causal, float scale, int sm_count, cudaStream_t st,
+                      int head_group_override = 0, int grid_override = 0) {
     MhaParams p;
-    p.O = O;
     p.LSE = LSE;
     p.BH = B * H;
     p.Nq = Nq;
@@ -485,14 +554,20 @@ inline int mha_launch(const CUtensorMap& tq, const CUtensorMap& tk, const CUtens
     p.causal = causal ? 1 : 0;
     p.scale = scale;
     p.num_pairs = (Nq + 2 * kMhaBlock - 1) / (2 * kMhaBlock);
-    p.head_group = 8;
+    // Item list order.  Causal: all heads' last query rows first (longest items first over the whole problem), so
+    // that the static hand-out balances; otherwise all items cost the same and heads go in groups of 8, so that
+    // the CTAs running at any time read the K/V of few heads (L2 reuse).
+    p.head_group = causal ? p.BH : 8;
+    if (head_group_override > 0) p.head_group = head_group_override;
     const int64_t items = static_cast<int64_t>(p.num_pairs) * p.BH;
-    if (items > INT32_MAX) return 2;
-    const int grid = static_cast<int>(items);
+    if (items > INT32_MAX - 1024) return 2;
+    p.num_items = static_cast<int>(items);
+    int grid = static_cast<int>(std::min<int64_t>(items, sm_count));
+    if (grid_override > 0) grid = static_cast<int>(std::min<int64_t>(items, grid_override));
     if (D == 64)
-        mha_fwd_kernel<64><<<grid, kMhaThreads, MhaSmem<64>::kTotal, st>>>(tq, tk, tv, p);
+        mha_fwd_kernel<64><<<grid, kMhaThreads, MhaSmem<64>::kTotal, st>>>(tq, tk, tv, to, p);
     else
-        mha_fwd_kernel<128><<<grid, kMhaThreads, MhaSmem<128>::kTotal, st>>>(tq, tk, tv, p);
+        mha_fwd_kernel<128><<<grid, kMhaThreads, MhaSmem<128>::kTotal, st>>>(tq, tk, tv, to, p);
     return cudaGetLastError() == cudaSuccess ? 0 : 4;
 }
 

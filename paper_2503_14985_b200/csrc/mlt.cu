@@ -313,13 +313,16 @@ int mlt_mha_fwd(const void* Q, const void* K, const void* V, void* O, float* LSE
     int rc = get_device(&dev);
     if (rc != MLT_OK) return rc;
 
-    CUtensorMap tq, tk, tv;
+    CUtensorMap tq, tk, tv, to;
     const uint64_t bh = static_cast<uint64_t>(B) * H;
     const uint32_t box[3] = {64, kMhaBlock, 1};
     {
         const uint64_t dims[3] = {static_cast<uint64_t>(D), static_cast<uint64_t>(Nq), bh};
         const uint64_t strides[2] = {static_cast<uint64_t>(D) * 2, static_cast<uint64_t>(Nq) * D * 2};
         rc = encode_bf16(&tq, Q, 3, dims, strides, box);
+        if (rc != MLT_OK) return rc;
+        const uint32_t obox[3] = {64, 32, 1};  // the output is stored per warp: 32 rows x 64 columns
+        rc = encode_bf16(&to, O, 3, dims, strides, obox);
         if (rc != MLT_OK) return rc;
     }
     {
@@ -330,8 +333,9 @@ int mlt_mha_fwd(const void* Q, const void* K, const void* V, void* O, float* LSE
         rc = encode_bf16(&tv, V, 3, dims, strides, box);
         if (rc != MLT_OK) return rc;
     }
-    return mha_launch(tq, tk, tv, static_cast<__nv_bfloat16*>(O), LSE, B, H, Nq, Nk, D, causal != 0, scale,
-                      dev.sm_count, static_cast<cudaStream_t>(stream));
+    return mha_launch(tq, tk, tv, to, LSE, B, H, Nq, Nk, D, causal != 0, scale,
+                      dev.sm_count, static_cast<cudaStream_t>(stream), debug_env_int("MLT_MHA_HEAD_GROUP", 0),
+                      debug_env_int("MLT_MHA_GRID", 0));
 }
 
 size_t mlt_paged_attn_workspace_bytes(int num_seqs, int H, int D) {

@@ -50,7 +50,9 @@ def scale_for(D):
 CASES = [(1, 1, 128, 128, 64, 0), (1, 1, 128, 128, 128, 1), (1, 2, 1, 1, 64, 0), (2, 3, 200, 333, 128, 0),
          (1, 1, 77, 200, 64, 1), (1, 1, 129, 129, 128, 1), (1, 4, 1024, 1024, 64, 1), (1, 2, 256, 256, 128, 0),
          (1, 3, 300, 300, 64, 0), (2, 2, 257, 640, 128, 1), (1, 1, 512, 384 + 1, 64, 0), (1, 9, 384, 384, 64, 1),
-         (1, 1, 1, 700, 128, 1)]
+         (1, 1, 1, 700, 128, 1),
+         # more work items than SMs: a CTA runs several items one after another (ragged last pairs among them)
+         (3, 70, 300, 300, 64, 1), (2, 80, 300, 420, 128, 1), (5, 40, 520, 260, 128, 0), (2, 90, 257, 257, 64, 0)]
 
 
 @pytest.mark.parametrize("B,H,Nq,Nk,D,causal", CASES)
