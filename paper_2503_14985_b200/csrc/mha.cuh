@@ -115,7 +115,9 @@ mha_fwd_kernel(const __grid_constant__ CUtensorMap tmap_q, const __grid_constant
     uint64_t* p_full = s_full + 2;            // [2]  softmax -> UMMA: P_t(j) in TMEM, O_t rescaled
     uint64_t* o_full = p_full + 2;            // [2]  UMMA -> epilogue: O_t complete
     uint64_t* q_empty = o_full + 2;           // [1]  UMMA -> loader: the item's last Q K^T has read the Q tiles
-    uint32_t* tmem_base_slot = reinterpret_cast<uint32_t*>(q_empty + 1);
+    uint64_t* s_free = q_empty + 1;           // [2]  softmax -> UMMA (D = 64): S_t(j) is in registers
+    uint64_t* p_free = s_free + 2;            // [2]  UMMA -> softmax (D = 64): P_t(j) V has completed
+    uint32_t* tmem_base_slot = reinterpret_cast<uint32_t*>(p_free + 2);
     volatile uint32_t* abort_flag = tmem_base_slot + 1;
 
     const int warp = threadIdx.x >> 5;
@@ -181,13 +183,26 @@ mha_fwd_kernel(const __grid_constant__ CUtensorMap tmap_q, const __grid_constant
                 tma_load_3d(smem_q + t * L::kTileBytes + c * L::kChunkBytes, &tmap_q, q_full, c * 64,
                             it.q_base + t * kMhaBlock, it.bh);
     };
-    auto load_kv = [&](const Item& it, int i) {  // ring tile i of the item: K_0, V_0, K_1, V_1, ...
+    // ring tile i of the item: K_0, V_0, K_1, V_1, ... (D = 128), or in the order the early Q K^T consumes them:
+    // K_0, K_1, V_0, K_2, V_1, ..., K_{J-1}, V_{J-2}, V_{J-1} (D = 64)
+    auto load_kv = [&](const Item& it, int i) {
+        bool is_k = (i & 1) == 0;
+        int blk = i >> 1;
+        if (D == 64 && i > 0) {
+            if (i == 2 * it.Jmax - 1) {
+                is_k = false;
+                blk = it.Jmax - 1;
+            } else {
+                is_k = (i & 1) == 1;
+                blk = is_k ? (i + 1) >> 1 : (i >> 1) - 1;
+            }
+        }
         uint8_t* dst = smem_kv + ld_stage * L::kTileBytes;
         mbar_arrive_expect_tx(&kv_full[ld_stage], L::kTileBytes);
 #pragma unroll
         for (int c = 0; c < kChunks; ++c)
-            tma_load_3d(dst + c * L::kChunkBytes, (i & 1) == 0 ? &tmap_k : &tmap_v, &kv_full[ld_stage], c * 64,
-                        (i >> 1) * kMhaBlock, it.bh);
+            tma_load_3d(dst + c * L::kChunkBytes, is_k ? &tmap_k : &tmap_v, &kv_full[ld_stage], c * 64,
+                        blk * kMhaBlock, it.bh);
         if (++ld_stage == kStages) { ld_stage = 0; ld_phase ^= 1; }
     };
 
@@ -206,6 +221,8 @@ mha_fwd_kernel(const __grid_constant__ CUtensorMap tmap_q, const __grid_constant
             mbar_init(&s_full[t], 1);
             mbar_init(&p_full[t], 4);  // one arrive per softmax warp
             mbar_init(&o_full[t], 1);
+            mbar_init(&s_free[t], 4);
+            mbar_init(&p_free[t], 1);
         }
         *abort_flag = 0;
         fence_mbar_init();
@@ -233,6 +250,12 @@ mha_fwd_kernel(const __grid_constant__ CUtensorMap tmap_q, const __grid_constant
     const uint32_t tmem_base = *tmem_base_slot;
     constexpr uint32_t kColS = 0;      // S_t at kColS + t*128
     constexpr uint32_t kColO = 256;    // O_t at kColO + t*D
+    // D = 128 fills the 512 columns, so P_t (BF16) overwrites the first 64 columns of S_t and the next Q K^T of a
+    // tile has to follow its P V.  D = 64 leaves 128 columns: P_t gets its own, and Q_t K_{j+1}^T is issued as soon
+    // as the softmax warps hold S_t(j) in registers, so S_t(j+1) is ready when they come back for it.
+    constexpr bool kEarlyQK = (D == 64);
+    constexpr uint32_t kColP = kEarlyQK ? 384 : kColS;  // P_t at kColP + t*(kEarlyQK ? 64 : 128)
+    constexpr uint32_t kStrideP = kEarlyQK ? 64 : kMhaBlock;
 
     if (warp >= 10) {
         setmaxnreg_dec<40>();  // only hand their registers over
@@ -289,7 +312,7 @@ mha_fwd_kernel(const __grid_constant__ CUtensorMap tmap_q, const __grid_constant
             // O_t (+)= P_t V over the 8 k-steps (16 keys each) of the tile in ring slot `slot`
             auto issue_pv = [&](int t, int slot, bool first) {
                 const uint32_t d = tmem_base + kColO + t * D;
-                const uint32_t a0 = tmem_base + kColS + t * kMhaBlock;
+                const uint32_t a0 = tmem_base + kColP + t * kStrideP;
                 const uint32_t b0 = (kv_lo0 & 0xFFFFu) + slot * (L::kTileBytes >> 4) + v_lbo;
                 if (leader) {
                     umma_ts_lo(d, a0, b0, idesc_pv, first ? 0u : 1u);
@@ -307,6 +330,64 @@ mha_fwd_kernel(const __grid_constant__ CUtensorMap tmap_q, const __grid_constant
             uint32_t n_p[2] = {0, 0};  // P tiles consumed so far, per query tile (parity of p_full)
             bool ok = true;
             Item it;
+            uint32_t n_qk[2] = {0, 0};  // Q K^T products issued so far, per query tile (parity of s_free)
+            if constexpr (kEarlyQK) {
+                for (int r = 0; ok && item_at(r, it); ++r) {
+                    const int Jmax = it.Jmax;
+                    ok = wait_all(q_full, r & 1, 0x200);
+                    // Step j: Q_t K_{j+1}^T for both tiles as soon as S_t(j) has been read, then P_t(j) V_j.
+                    // Step -1 issues the first Q K^T products only (same instructions, no cold copy).
+#pragma unroll 1
+                    for (int j = -1; j < Jmax && ok; ++j) {
+                        if (j + 1 < Jmax) {
+                            const int kslot = stage;
+                            ok = wait_all(&kv_full[kslot], phase, 0x240 + kslot);
+                            if (!ok) break;
+                            if (++stage == kStages) { stage = 0; phase ^= 1; }
+                            tc_fence_after();
+                            for (int t = 0; t < 2 && ok; ++t) {
+                                if (j + 1 >= it.J[t]) continue;
+                                if (n_qk[t] > 0) {  // S_t is free once the softmax warps hold its previous contents
+                                    ok = wait_all(&s_free[t], (n_qk[t] - 1) & 1, 0x250 + t);
+                                    if (!ok) break;
+                                    tc_fence_after();
+                                }
+                                ++n_qk[t];
+                                issue_qk(t, kslot);
+                            }
+                            if (!ok) break;
+                            if (leader) {
+                                umma_commit(&kv_empty[kslot]);
+                                if (j + 2 == Jmax) umma_commit(q_empty);  // the item's last Q K^T products are issued
+                            }
+                            __syncwarp();
+                        }
+                        if (j >= 0) {
+                            const int vslot = stage;
+                            ok = wait_all(&kv_full[vslot], phase, 0x220 + vslot);
+                            if (!ok) break;
+                            if (++stage == kStages) { stage = 0; phase ^= 1; }
+                            for (int t = 0; t < 2 && ok; ++t) {
+                                if (j >= it.J[t]) continue;
+                                // P_t(0) of an item also tells that the softmax warps have read the previous O_t
+                                ok = wait_all(&p_full[t], n_p[t] & 1, 0x230 + t);
+                                if (!ok) break;
+                                ++n_p[t];
+                                tc_fence_after();
+                                issue_pv(t, vslot, j == 0);
+                                if (leader) {
+                                    umma_commit(&p_free[t]);
+                                    if (j == it.J[t] - 1) umma_commit(&o_full[t]);
+                                }
+                                __syncwarp();
+                            }
+                            if (!ok) break;
+                            if (leader) umma_commit(&kv_empty[vslot]);
+                            __syncwarp();
+                        }
+                    }
+                }
+            } else {
             for (int r = 0; ok && item_at(r, it); ++r) {
                 const int Jmax = it.Jmax;
                 ok = wait_all(q_full, r & 1, 0x200);
@@ -357,6 +438,7 @@ mha_fwd_kernel(const __grid_constant__ CUtensorMap tmap_q, const __grid_constant
                     }
                 }
             }
+            }  // !kEarlyQK
         }
     } else {
         // ------------------- softmax, O rescale and epilogue of tile t -------------------
@@ -367,6 +449,7 @@ mha_fwd_kernel(const __grid_constant__ CUtensorMap tmap_q, const __grid_constant
         const uint32_t lane_addr = tmem_base + (static_cast<uint32_t>(quarter * 32) << 16);
         const uint32_t s_addr = lane_addr + kColS + t * kMhaBlock;
         const uint32_t o_addr = lane_addr + kColO + t * D;
+        const uint32_t p_addr = lane_addr + kColP + t * kStrideP;
         const float c = p.scale * kLog2e;
         uint32_t n_s = 0, n_o = 0;  // S tiles and O tiles taken so far (parities of s_full / o_full)
         bool ok = true;
@@ -388,6 +471,11 @@ mha_fwd_kernel(const __grid_constant__ CUtensorMap tmap_q, const __grid_constant
 #pragma unroll
             for (int q = 0; q < 4; ++q) tmem_ld_32x32b_x32(s_addr + q * 32, s[q]);
             tmem_wait_ld();
+            if constexpr (kEarlyQK) {  // S_t is in registers: the next Q K^T of this tile may overwrite it
+                tc_fence_before();
+                __syncwarp();
+                if (lane == 0) mbar_arrive(&s_free[t]);
+            }
             const int j0 = j * kMhaBlock;
             if (j0 + kMhaBlock - 1 > limit) {  // diagonal or tail block: mask keys beyond the row's last visible one
 #pragma unroll
@@ -438,7 +526,12 @@ mha_fwd_kernel(const __grid_constant__ CUtensorMap tmap_q, const __grid_constant
                         pk[(w & 1) * 8 + i] = pack_bf16x2(x0.x, x0.y);
                         pk[(w & 1) * 8 + i + 1] = pack_bf16x2(x1.x, x1.y);
                     }
-                    if (w & 1) tmem_st_32x32b_x16(s_addr + (w >> 1) * 16, pk);
+                    if (kEarlyQK && w == 1 && n_s > 1) {
+                        // P_t has its own columns: the previous P_t V (P number n_s - 1) must have read them
+                        if (!__all_sync(0xffffffffu, mbar_wait(&p_free[t], n_s & 1, abort_flag, 0x310 + t))) ok = false;
+                        tc_fence_after();
+                    }
+                    if (w & 1) tmem_st_32x32b_x16(p_addr + (w >> 1) * 16, pk);
                 }
             };
             // The first block of a row takes its max first and then runs the same pass as every other block.
@@ -469,6 +562,7 @@ mha_fwd_kernel(const __grid_constant__ CUtensorMap tmap_q, const __grid_constant
                     exp_pass((m_run == -INFINITY) ? 0.0f : -m_run * c);
                 }
             }
+            if (!ok) break;
             l_run += (acc0.x + acc0.y) + (acc1.x + acc1.y);
             tmem_wait_st();
             tc_fence_before();
