@@ -18,13 +18,16 @@ constexpr int kGemmBM = 128;
 constexpr int kGemmBK = 64;
 constexpr int kGemmThreads = 192;
 
+// FP32 output goes through shared memory and TMA: two 4 KB boxes (32 rows x 32 FP32 columns) per epilogue warp
+constexpr int kGemmStagingBytes = 4 * 2 * 4096;
+
 template <int BN, int kStages>
 struct GemmSmem {
     static constexpr int kABytes = kGemmBM * kGemmBK * 2;  // 16 KB
     static constexpr int kBBytes = kGemmBK * BN * 2;       // 64 rows x BN, as BN/64 boxes of 64 x 64
     static constexpr int kStageBytes = kABytes + kBBytes;
     static constexpr int kBarrierBytes = 256;
-    static constexpr int kTotal = kStages * kStageBytes + kBarrierBytes + 1024;  // + alignment slack
+    static constexpr int kTotal = kStages * kStageBytes + kGemmStagingBytes + kBarrierBytes + 1024;  // + alignment slack
 };
 
 struct GemmParams {
@@ -43,6 +46,7 @@ struct GemmParams {
     int64_t ldcf;
     int accumulate;    // with Cf: add to the prior contents of C (the "C += A*B" of Sec. 2)
     uint32_t f16_inputs;  // 0: BF16 operands, 1: FP16 operands (same tiles and descriptors, other format field)
+    int c_tma;  // FP32 C is written through the tensor map tmap_c (TMA store / add-reduction), not by the threads
 };
 
 // Instruction descriptor with the operand format chosen at run time (BF16: format 1, FP16: format 0).
@@ -97,6 +101,42 @@ __device__ __forceinline__ void gemm_store_chunk(const GemmParams& p, const uint
     }
 }
 
+// The same segment for a whole warp when C is FP32 and reached through a tensor map (p.c_tma): the warp's 32 rows
+// x 32 columns go into a 4 KB staging box (128-byte rows, 16-byte chunk k of row r at chunk k ^ (r & 7): the
+// 128-byte swizzle of the map) and one lane issues a TMA store, or a TMA add-reduction for C += A * B, which adds
+// at the destination and reads nothing back.  Edges are clipped by the tensor map.  `stg` alternates between
+// two boxes; at most one newer store may still be reading the other box when this one is refilled.
+__device__ __forceinline__ void gemm_store_chunk_tma(const GemmParams& p, const CUtensorMap* tmap_c, uint8_t* stg,
+                                                     const uint32_t (&v)[32], int lane, int row0, int col0) {
+    if (lane == 0) tma_store_wait_read<1>();
+    __syncwarp();
+#pragma unroll
+    for (int k = 0; k < 8; ++k)
+        *reinterpret_cast<uint4*>(stg + lane * 128 + ((k ^ (lane & 7)) * 16)) =
+            make_uint4(v[k * 4], v[k * 4 + 1], v[k * 4 + 2], v[k * 4 + 3]);
+    fence_proxy_async_smem();
+    __syncwarp();
+    if (lane == 0) {
+        if (row0 < p.M && col0 < p.N) {
+            if (p.accumulate)
+                tma_reduce_add_2d(tmap_c, stg, col0, row0);
+            else
+                tma_store_2d(tmap_c, stg, col0, row0);
+        }
+        tma_store_commit();  // also when nothing was stored: the group count is what the wait above relies on
+    }
+    // The store works in 16-byte units, so the tensor map covers only the columns below N rounded down to a
+    // multiple of 4; the up to three columns beyond are written by the thread that owns the row.
+    const int n4 = p.N & ~3;
+    if (n4 != p.N && col0 <= n4 && n4 < col0 + 32 && row0 + lane < p.M) {
+        float* crow = p.Cf + static_cast<int64_t>(row0 + lane) * p.ldcf;
+        for (int col = n4; col < p.N; ++col) {
+            const float x = __uint_as_float(v[col - col0]);
+            crow[col] = p.accumulate ? crow[col] + x : x;
+        }
+    }
+}
+
 // tile index -> (tile_m, tile_n): groups of `group_m` M-tiles, M fastest inside a group, so that
 // the CTAs running at the same time share few A and B panels (L2 reuse).
 __device__ __forceinline__ void gemm_tile_coords(const GemmParams& p, int tile, int& tm, int& tn) {
@@ -112,11 +152,12 @@ __device__ __forceinline__ void gemm_tile_coords(const GemmParams& p, int tile, 
 template <int BN, int kStages>
 __global__ void __launch_bounds__(kGemmThreads, 1)
 gemm_bf16_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_constant__ CUtensorMap tmap_b,
-                 const GemmParams p) {
+                 const __grid_constant__ CUtensorMap tmap_c, const GemmParams p) {
     using L = GemmSmem<BN, kStages>;
     extern __shared__ uint8_t smem_raw[];
     uint8_t* smem = reinterpret_cast<uint8_t*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~uintptr_t(1023));
-    uint64_t* bars = reinterpret_cast<uint64_t*>(smem + kStages * L::kStageBytes);
+    uint8_t* smem_staging = smem + kStages * L::kStageBytes;  // 1024-byte aligned (swizzle atoms of the TMA store)
+    uint64_t* bars = reinterpret_cast<uint64_t*>(smem_staging + kGemmStagingBytes);
     uint64_t* full = bars;                     // [kStages]  TMA -> MMA
     uint64_t* empty = bars + kStages;          // [kStages]  MMA -> TMA
     uint64_t* acc_full = bars + 2 * kStages;   // [2]        MMA -> epilogue
@@ -241,13 +282,18 @@ gemm_bf16_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_consta
                 uint32_t v[32];
                 tmem_ld_32x32b_x32(t_row + c * 32, v);
                 tmem_wait_ld();
-                gemm_store_chunk(p, v, row, n0 + c * 32, item % p.split_k);
+                if (p.c_tma)
+                    gemm_store_chunk_tma(p, &tmap_c, smem_staging + quarter * 8192 + (c & 1) * 4096, v, lane,
+                                         tm * kGemmBM + quarter * 32, n0 + c * 32);
+                else
+                    gemm_store_chunk(p, v, row, n0 + c * 32, item % p.split_k);
             }
             tc_fence_before();
             __syncwarp();
             if (lane == 0) mbar_arrive(&acc_empty[acc]);
             if (++acc == 2) { acc = 0; acc_phase ^= 1; }
         }
+        if (lane == 0) tma_store_wait_all<0>();  // shared memory must outlive the stores that read it
     }
 
     // common exit: every role reaches this, also after an aborted wait
@@ -280,17 +326,18 @@ struct GemmPairSmem {
     static constexpr int kABytes = 128 * kGemmBK * 2;  // this CTA's 128 rows of A
     static constexpr int kBBytes = kGemmBK * 128 * 2;  // this CTA's 128 columns of B: 2 boxes of 64 x 64
     static constexpr int kStageBytes = kABytes + kBBytes;
-    static constexpr int kTotal = kStages * kStageBytes + 256 + 1024;
+    static constexpr int kTotal = kStages * kStageBytes + kGemmStagingBytes + 256 + 1024;
 };
 
 template <int kStages>
 __global__ void __cluster_dims__(2, 1, 1) __launch_bounds__(kGemmThreads, 1)
 gemm_bf16_pair_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_constant__ CUtensorMap tmap_b,
-                      const GemmParams p) {
+                      const __grid_constant__ CUtensorMap tmap_c, const GemmParams p) {
     using L = GemmPairSmem<kStages>;
     extern __shared__ uint8_t smem_raw[];
     uint8_t* smem = reinterpret_cast<uint8_t*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~uintptr_t(1023));
-    uint64_t* bars = reinterpret_cast<uint64_t*>(smem + kStages * L::kStageBytes);
+    uint8_t* smem_staging = smem + kStages * L::kStageBytes;  // 1024-byte aligned (swizzle atoms of the TMA store)
+    uint64_t* bars = reinterpret_cast<uint64_t*>(smem_staging + kGemmStagingBytes);
     uint64_t* full = bars;
     uint64_t* empty = bars + kStages;
     uint64_t* acc_full = bars + 2 * kStages;
@@ -416,13 +463,18 @@ gemm_bf16_pair_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_c
                 uint32_t v[32];
                 tmem_ld_32x32b_x32(t_row + c * 32, v);
                 tmem_wait_ld();
-                gemm_store_chunk(p, v, row, n0 + c * 32, 0);
+                if (p.c_tma)
+                    gemm_store_chunk_tma(p, &tmap_c, smem_staging + quarter * 8192 + (c & 1) * 4096, v, lane,
+                                         tm * kPairBM + static_cast<int>(rank) * 128 + quarter * 32, n0 + c * 32);
+                else
+                    gemm_store_chunk(p, v, row, n0 + c * 32, 0);
             }
             tc_fence_before();
             __syncwarp();
             if (lane == 0) mbar_arrive_cluster(map_to_cta(smem_u32(&acc_empty[acc]), 0));
             if (++acc == 2) { acc = 0; acc_phase ^= 1; }
         }
+        if (lane == 0) tma_store_wait_all<0>();  // shared memory must outlive the stores that read it
     }
 
     // common exit: no CTA of the pair leaves while its peer may still touch its memory

@@ -3,29 +3,41 @@
 // tensor cores, online softmax with running row max m and row sum l, O += P V_j on
 // the tensor cores, final O / l and LSE = m + ln l.
 //
-// A CTA owns 256 query rows of one (batch, head): two 128-row tiles that take turns
-// on the tensor pipe, so the exponentials of one tile overlap the products of the other.
+// A work item is 256 query rows of one (batch, head): two 128-row tiles that take turns on the tensor pipe, so
+// the exponentials of one tile overlap the products of the other.  CTAs are persistent (one per SM): each runs
+// the items at positions r * gridDim.x +/- blockIdx.x of a list sorted by length (direction alternating per
+// round, which balances the CTAs' sums without a global counter); the loader prefetches the next item's K/V
+// tiles, and its Q tiles once the current item's last Q K^T has completed.
 //   warps 0-3   softmax / O-rescale / epilogue of tile 0 (one thread per query row)
 //   warps 4-7   the same for tile 1
 //   warp  8     UMMA issuer (the whole warp runs the loop, one elected lane issues) and owner of the
-//               tensor-memory allocation; it serves the tiles in a fixed order (P V of tile 0, next
-//               Q K^T of tile 0, the same for tile 1), which keeps the two softmax warpgroups half a
-//               period apart
-//   warp  9     TMA loader (one lane): both Q tiles once, then K_0, V_0, K_1, V_1, ... through a ring;
-//               it also initialises the barriers and issues the first loads before the CTA-wide sync
+//               tensor-memory allocation; it serves the tiles in a fixed order, which keeps the two softmax
+//               warpgroups half a period apart (one issuer per tile was tried: the tiles fall into step and
+//               D = 128 loses 18 %)
+//   warp  9     TMA loader (one lane): Q tiles, then K/V tiles through a ring; it also initialises the
+//               barriers and issues the first loads before the CTA-wide sync
 //   warps 10-11 idle (they complete the third warpgroup for the register hand-over)
-// Tensor memory (512 columns): S_0 | S_1 (128 FP32 columns each; the BF16 P of a tile
-// overwrites the first 64 columns of its S and is consumed from there as the A operand
-// of P V), then O_0 | O_1 (D FP32 columns each).
+// Tensor memory (512 columns): S_0 | S_1 (128 FP32 columns each), O_0 | O_1 (D FP32 columns each).  D = 128:
+// the BF16 P of a tile overwrites the first 64 columns of its S and is consumed from there as the A operand of
+// P V.  D = 64: P_0 | P_1 have their own columns, and the next Q K^T of a tile is issued as soon as the softmax
+// warps hold S in registers.
+// Epilogue: O / l as BF16 into a 4 KB staging area per warp (128-byte swizzle), one TMA store per 32 x 64 box.
 //
 // Measured on B200 (what shaped this kernel):
 //  * a UMMA of 128x128x16 takes 64 clocks, also with A from tensor memory; issuing one costs the issuing
 //    thread about 46 clocks from a single divergent lane and about 20 from warp-uniform code with an elected
-//    lane; a warp that shares its scheduler partition with a busy warp is served much more rarely;
+//    lane; a warp that shares its scheduler partition with busy warps is served rarely: a barrier wait costs
+//    the issuer about 280 clocks even when the barrier completed long before, and a step of both tiles (four
+//    waits, 32 products) takes about as long as the whole period -- the issuer is co-limiting;
+//  * code that runs once per item (a separate copy of the first Q K^T, an unrolled epilogue, the item decode
+//    with its divisions) is fetched cold every time and costs thousands of clocks on those starved warps: the
+//    first products go through the loop body, the epilogue is a short loop, the decode is done once per CTA
+//    into shared memory;
 //  * per tile and K/V block the chain is: S ready -> TMEM load (125) -> softmax (about 1700: 1024 MUFU clocks
 //    plus the packed FP32 work a single warp per partition cannot fully overlap) -> P V and next Q K^T
 //    (about 1085) -> S ready; with two tiles half a period apart the period is about 3230 clocks, i.e. the
-//    tensor pipe is busy about two thirds of the time.
+//    tensor pipe is busy about two thirds of the time;
+//  * the SM clock under this kernel is 1.72-1.77 GHz (power management), not the 1.965 GHz maximum.
 #pragma once
 
 #include <math.h>

@@ -77,7 +77,7 @@ int get_device(DeviceInfo* out) {
 
 // BF16 tensor map with 128-byte swizzle.  dims / strides innermost first; strides[0] is implicit.
 int encode_bf16(CUtensorMap* map, const void* base, int rank, const uint64_t* dims, const uint64_t* strides_bytes,
-                const uint32_t* box, bool f16 = false) {
+                const uint32_t* box, int dtype = 0 /* 0 BF16, 1 FP16, 2 FP32 */) {
     EncodeTiledFn enc;
     int rc = get_encoder(&enc);
     if (rc != MLT_OK) return rc;
@@ -95,7 +95,10 @@ int encode_bf16(CUtensorMap* map, const void* base, int rank, const uint64_t* di
             gstride[i - 1] = strides_bytes[i - 1];
         }
     }
-    CUresult r = enc(map, f16 ? CU_TENSOR_MAP_DATA_TYPE_FLOAT16 : CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, static_cast<cuuint32_t>(rank), const_cast<void*>(base),
+    const CUtensorMapDataType dt = dtype == 2   ? CU_TENSOR_MAP_DATA_TYPE_FLOAT32
+                                   : dtype == 1 ? CU_TENSOR_MAP_DATA_TYPE_FLOAT16
+                                                : CU_TENSOR_MAP_DATA_TYPE_BFLOAT16;
+    CUresult r = enc(map, dt, static_cast<cuuint32_t>(rank), const_cast<void*>(base),
                      gdim, gstride, gbox, estr, CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B,
                      CU_TENSOR_MAP_L2_PROMOTION_L2_256B, CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
     return r == CUDA_SUCCESS ? MLT_OK : MLT_ERR_CUDA;
@@ -220,14 +223,25 @@ static int gemm_run(const void* A, const void* B, void* C, int64_t M, int64_t N,
         const uint64_t dims[2] = {static_cast<uint64_t>(K), static_cast<uint64_t>(M)};
         const uint64_t strides[1] = {static_cast<uint64_t>(lda) * 2};
         const uint32_t box[2] = {kGemmBK, 128};
-        rc = encode_bf16(&ta, A, 2, dims, strides, box, f16_in);
+        rc = encode_bf16(&ta, A, 2, dims, strides, box, f16_in ? 1 : 0);
         if (rc != MLT_OK) return rc;
     }
     {
         const uint64_t dims[2] = {static_cast<uint64_t>(N), static_cast<uint64_t>(K)};
         const uint64_t strides[1] = {static_cast<uint64_t>(ldb) * 2};
         const uint32_t box[2] = {64, kGemmBK};
-        rc = encode_bf16(&tb, B, 2, dims, strides, box, f16_in);
+        rc = encode_bf16(&tb, B, 2, dims, strides, box, f16_in ? 1 : 0);
+        if (rc != MLT_OK) return rc;
+    }
+
+    CUtensorMap tc = tb;  // only read by the kernels when C is FP32
+    const bool c_tma = f32_out && N >= 4;
+    if (c_tma) {
+        // the TMA store works in 16-byte units: the map ends at N rounded down to a multiple of 4 columns
+        const uint64_t dims[2] = {static_cast<uint64_t>(N) & ~3ull, static_cast<uint64_t>(M)};
+        const uint64_t strides[1] = {static_cast<uint64_t>(ldc) * 4};
+        const uint32_t box[2] = {32, 32};  // 128-byte rows: one epilogue warp's 32 rows x 32 columns
+        rc = encode_bf16(&tc, C, 2, dims, strides, box, 2);
         if (rc != MLT_OK) return rc;
     }
 
@@ -246,6 +260,7 @@ static int gemm_run(const void* A, const void* B, void* C, int64_t M, int64_t N,
     p.ldcf = ldc;
     p.accumulate = accumulate ? 1 : 0;
     p.f16_inputs = f16_in ? 1u : 0u;
+    p.c_tma = c_tma ? 1 : 0;
     if (variant == 2 && workspace && !f32_out) {
         // Few tiles (skinny or small problem): cut K into slices so that about two work items per SM exist; the
         // weights are then streamed by all SMs at once.  FP32 partials go to the caller's scratch.
@@ -263,14 +278,14 @@ static int gemm_run(const void* A, const void* B, void* C, int64_t M, int64_t N,
         // M-tiles per raster group: wide problems re-read B once per group, so fewer, taller groups pay
         p.group_m = debug_env_int("MLT_GEMM_GROUP_M", tiles_n >= 32 ? 16 : 8);
         const int clusters = static_cast<int>(std::min<int64_t>(tiles_m * tiles_n, dev.sm_count / 2));
-        gemm_bf16_pair_kernel<6><<<2 * clusters, kGemmThreads, GemmPairSmem<6>::kTotal, st>>>(ta, tb, p);
+        gemm_bf16_pair_kernel<6><<<2 * clusters, kGemmThreads, GemmPairSmem<6>::kTotal, st>>>(ta, tb, tc, p);
     } else {
         p.group_m = 16;
         const int grid = static_cast<int>(std::min<int64_t>(tiles_m * tiles_n * p.split_k, dev.sm_count));
         if (variant == 1)
-            gemm_bf16_kernel<256, 4><<<grid, kGemmThreads, GemmSmem<256, 4>::kTotal, st>>>(ta, tb, p);
+            gemm_bf16_kernel<256, 4><<<grid, kGemmThreads, GemmSmem<256, 4>::kTotal, st>>>(ta, tb, tc, p);
         else
-            gemm_bf16_kernel<128, 6><<<grid, kGemmThreads, GemmSmem<128, 6>::kTotal, st>>>(ta, tb, p);
+            gemm_bf16_kernel<128, 6><<<grid, kGemmThreads, GemmSmem<128, 6>::kTotal, st>>>(ta, tb, tc, p);
         if (p.split_k > 1) {
             if (cudaGetLastError() != cudaSuccess) return MLT_ERR_CUDA;
             const int64_t groups = M * ((N + 7) / 8);
