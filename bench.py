@@ -101,6 +101,10 @@ class ClockSampler:
             self._nv = pynvml
             self._h = pynvml.nvmlDeviceGetHandleByIndex(index)
             self.max_mhz = int(pynvml.nvmlDeviceGetMaxClockInfo(self._h, pynvml.NVML_CLOCK_SM))
+            # first calls into NVML can take tens of milliseconds: make them before the timed region starts
+            pynvml.nvmlDeviceGetClockInfo(self._h, pynvml.NVML_CLOCK_SM)
+            pynvml.nvmlDeviceGetCurrentClocksEventReasons(self._h)
+            pynvml.nvmlDeviceGetPowerUsage(self._h)
         except Exception:
             self._nv = None
 

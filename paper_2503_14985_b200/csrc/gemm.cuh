@@ -27,7 +27,9 @@ struct GemmSmem {
     static constexpr int kBBytes = kGemmBK * BN * 2;       // 64 rows x BN, as BN/64 boxes of 64 x 64
     static constexpr int kStageBytes = kABytes + kBBytes;
     static constexpr int kBarrierBytes = 256;
-    static constexpr int kTotal = kStages * kStageBytes + kGemmStagingBytes + kBarrierBytes + 1024;  // + alignment slack
+    // stages | barriers (padded to 1 KB) | staging for FP32 output (only requested by launches that write FP32 C)
+    static constexpr int kNoStaging = kStages * kStageBytes + 1024 + 1024;  // + alignment slack
+    static constexpr int kTotal = kNoStaging + kGemmStagingBytes;
 };
 
 struct GemmParams {
@@ -46,7 +48,6 @@ struct GemmParams {
     int64_t ldcf;
     int accumulate;    // with Cf: add to the prior contents of C (the "C += A*B" of Sec. 2)
     uint32_t f16_inputs;  // 0: BF16 operands, 1: FP16 operands (same tiles and descriptors, other format field)
-    int c_tma;  // FP32 C is written through the tensor map tmap_c (TMA store / add-reduction), not by the threads
 };
 
 // Instruction descriptor with the operand format chosen at run time (BF16: format 1, FP16: format 0).
@@ -95,8 +96,10 @@ __device__ __forceinline__ void gemm_store_chunk(const GemmParams& p, const uint
             *reinterpret_cast<uint4*>(crow + col) = out;
         } else if (col < p.N) {
             const uint32_t w[4] = {out.x, out.y, out.z, out.w};
-            for (int j = 0; col + j < p.N; ++j)
-                crow[col + j] = __ushort_as_bfloat16(static_cast<unsigned short>(w[j >> 1] >> ((j & 1) * 16)));
+#pragma unroll
+            for (int j = 0; j < 8; ++j)  // constant indices keep w in registers
+                if (col + j < p.N)
+                    crow[col + j] = __ushort_as_bfloat16(static_cast<unsigned short>(w[j >> 1] >> ((j & 1) * 16)));
         }
     }
 }
@@ -130,9 +133,10 @@ __device__ __forceinline__ void gemm_store_chunk_tma(const GemmParams& p, const 
     const int n4 = p.N & ~3;
     if (n4 != p.N && col0 <= n4 && n4 < col0 + 32 && row0 + lane < p.M) {
         float* crow = p.Cf + static_cast<int64_t>(row0 + lane) * p.ldcf;
-        for (int col = n4; col < p.N; ++col) {
-            const float x = __uint_as_float(v[col - col0]);
-            crow[col] = p.accumulate ? crow[col] + x : x;
+#pragma unroll
+        for (int j = 0; j < 32; ++j) {  // constant indices keep v in registers
+            const int col = col0 + j;
+            if (col >= n4 && col < p.N) crow[col] = p.accumulate ? crow[col] + __uint_as_float(v[j]) : __uint_as_float(v[j]);
         }
     }
 }
@@ -149,15 +153,16 @@ __device__ __forceinline__ void gemm_tile_coords(const GemmParams& p, int tile, 
     tn = r / rows;
 }
 
-template <int BN, int kStages>
+template <int BN, int kStages, bool kCTma>
 __global__ void __launch_bounds__(kGemmThreads, 1)
 gemm_bf16_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_constant__ CUtensorMap tmap_b,
                  const __grid_constant__ CUtensorMap tmap_c, const GemmParams p) {
     using L = GemmSmem<BN, kStages>;
     extern __shared__ uint8_t smem_raw[];
     uint8_t* smem = reinterpret_cast<uint8_t*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~uintptr_t(1023));
-    uint8_t* smem_staging = smem + kStages * L::kStageBytes;  // 1024-byte aligned (swizzle atoms of the TMA store)
-    uint64_t* bars = reinterpret_cast<uint64_t*>(smem_staging + kGemmStagingBytes);
+    uint64_t* bars = reinterpret_cast<uint64_t*>(smem + kStages * L::kStageBytes);
+    // 1024-byte aligned (swizzle atoms of the TMA store); present only when the launch asked for it (p.c_tma)
+    uint8_t* smem_staging = smem + kStages * L::kStageBytes + 1024;
     uint64_t* full = bars;                     // [kStages]  TMA -> MMA
     uint64_t* empty = bars + kStages;          // [kStages]  MMA -> TMA
     uint64_t* acc_full = bars + 2 * kStages;   // [2]        MMA -> epilogue
@@ -282,7 +287,7 @@ gemm_bf16_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_consta
                 uint32_t v[32];
                 tmem_ld_32x32b_x32(t_row + c * 32, v);
                 tmem_wait_ld();
-                if (p.c_tma)
+                if constexpr (kCTma)
                     gemm_store_chunk_tma(p, &tmap_c, smem_staging + quarter * 8192 + (c & 1) * 4096, v, lane,
                                          tm * kGemmBM + quarter * 32, n0 + c * 32);
                 else
@@ -293,7 +298,7 @@ gemm_bf16_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_consta
             if (lane == 0) mbar_arrive(&acc_empty[acc]);
             if (++acc == 2) { acc = 0; acc_phase ^= 1; }
         }
-        if (lane == 0) tma_store_wait_all<0>();  // shared memory must outlive the stores that read it
+        if (kCTma && lane == 0) tma_store_wait_all<0>();  // shared memory must outlive the stores that read it
     }
 
     // common exit: every role reaches this, also after an aborted wait
@@ -326,18 +331,20 @@ struct GemmPairSmem {
     static constexpr int kABytes = 128 * kGemmBK * 2;  // this CTA's 128 rows of A
     static constexpr int kBBytes = kGemmBK * 128 * 2;  // this CTA's 128 columns of B: 2 boxes of 64 x 64
     static constexpr int kStageBytes = kABytes + kBBytes;
-    static constexpr int kTotal = kStages * kStageBytes + kGemmStagingBytes + 256 + 1024;
+    static constexpr int kNoStaging = kStages * kStageBytes + 1024 + 1024;
+    static constexpr int kTotal = kNoStaging + kGemmStagingBytes;
 };
 
-template <int kStages>
+template <int kStages, bool kCTma>
 __global__ void __cluster_dims__(2, 1, 1) __launch_bounds__(kGemmThreads, 1)
 gemm_bf16_pair_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_constant__ CUtensorMap tmap_b,
                       const __grid_constant__ CUtensorMap tmap_c, const GemmParams p) {
     using L = GemmPairSmem<kStages>;
     extern __shared__ uint8_t smem_raw[];
     uint8_t* smem = reinterpret_cast<uint8_t*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~uintptr_t(1023));
-    uint8_t* smem_staging = smem + kStages * L::kStageBytes;  // 1024-byte aligned (swizzle atoms of the TMA store)
-    uint64_t* bars = reinterpret_cast<uint64_t*>(smem_staging + kGemmStagingBytes);
+    uint64_t* bars = reinterpret_cast<uint64_t*>(smem + kStages * L::kStageBytes);
+    // 1024-byte aligned (swizzle atoms of the TMA store); present only when the launch asked for it (p.c_tma)
+    uint8_t* smem_staging = smem + kStages * L::kStageBytes + 1024;
     uint64_t* full = bars;
     uint64_t* empty = bars + kStages;
     uint64_t* acc_full = bars + 2 * kStages;
@@ -463,7 +470,7 @@ gemm_bf16_pair_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_c
                 uint32_t v[32];
                 tmem_ld_32x32b_x32(t_row + c * 32, v);
                 tmem_wait_ld();
-                if (p.c_tma)
+                if constexpr (kCTma)
                     gemm_store_chunk_tma(p, &tmap_c, smem_staging + quarter * 8192 + (c & 1) * 4096, v, lane,
                                          tm * kPairBM + static_cast<int>(rank) * 128 + quarter * 32, n0 + c * 32);
                 else
@@ -474,7 +481,7 @@ gemm_bf16_pair_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_c
             if (lane == 0) mbar_arrive_cluster(map_to_cta(smem_u32(&acc_empty[acc]), 0));
             if (++acc == 2) { acc = 0; acc_phase ^= 1; }
         }
-        if (lane == 0) tma_store_wait_all<0>();  // shared memory must outlive the stores that read it
+        if (kCTma && lane == 0) tma_store_wait_all<0>();  // shared memory must outlive the stores that read it
     }
 
     // common exit: no CTA of the pair leaves while its peer may still touch its memory

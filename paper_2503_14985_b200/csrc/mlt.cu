@@ -64,9 +64,12 @@ int get_device(DeviceInfo* out) {
             cudaDeviceGetAttribute(&d.sm_count, cudaDevAttrMultiProcessorCount, dev) != cudaSuccess)
             return MLT_ERR_CUDA;
         if (d.cc_major != 10) return MLT_ERR_ARCH;
-        if (set_smem(gemm_bf16_kernel<256, 4>, GemmSmem<256, 4>::kTotal) != MLT_OK ||
-            set_smem(gemm_bf16_kernel<128, 6>, GemmSmem<128, 6>::kTotal) != MLT_OK ||
-            set_smem(gemm_bf16_pair_kernel<6>, GemmPairSmem<6>::kTotal) != MLT_OK)
+        if (set_smem(gemm_bf16_kernel<256, 4, false>, GemmSmem<256, 4>::kNoStaging) != MLT_OK ||
+            set_smem(gemm_bf16_kernel<128, 6, false>, GemmSmem<128, 6>::kNoStaging) != MLT_OK ||
+            set_smem(gemm_bf16_pair_kernel<6, false>, GemmPairSmem<6>::kNoStaging) != MLT_OK ||
+            set_smem(gemm_bf16_kernel<256, 4, true>, GemmSmem<256, 4>::kTotal) != MLT_OK ||
+            set_smem(gemm_bf16_kernel<128, 6, true>, GemmSmem<128, 6>::kTotal) != MLT_OK ||
+            set_smem(gemm_bf16_pair_kernel<6, true>, GemmPairSmem<6>::kTotal) != MLT_OK)
             return MLT_ERR_CUDA;
         if (mha_configure() != MLT_OK) return MLT_ERR_CUDA;
         d.configured = true;
@@ -200,17 +203,30 @@ static int gemm_run(const void* A, const void* B, void* C, int64_t M, int64_t N,
         return cudaGetLastError() == cudaSuccess ? MLT_OK : MLT_ERR_CUDA;
     }
 
-    // Tile shape by problem size: CTA pairs on 256 x 256 tiles when there is at least one tile per pair of SMs,
-    // else 128 x 256 tiles, else (most SMs would idle) 128 x 128 tiles.
+    // Tile shape by problem size.  0: CTA pairs on 256 x 256 tiles, 1: 128 x 256 tiles, 2: 128 x 128 tiles.
+    // Problems with at least 512 rows are compute-bound: the variant with the least (waves x work per tile /
+    // efficiency) wins, with the measured relative efficiencies 1 : 0.8 : 0.62 of the three kernels (the smaller
+    // tiles are bound by the shared-memory operand path).  Shorter problems stream B once and are bound by memory:
+    // pairs when there is at least one tile per pair of SMs, else 128 x 256 tiles, else (most SMs would idle)
+    // 128 x 128 tiles, which can also be cut along K.
     const int64_t pair_tiles = ((M + kPairBM - 1) / kPairBM) * ((N + kPairBN - 1) / kPairBN);
     const int64_t tiles_m128 = (M + kGemmBM - 1) / kGemmBM;
-    int variant;  // 0: pair 256x256, 1: 128x256, 2: 128x128
-    if (pair_tiles >= dev.sm_count / 2 && forced_variant() != 1 && forced_variant() != 2)
+    const int64_t tiles1 = tiles_m128 * ((N + 255) / 256);
+    const int64_t tiles2 = tiles_m128 * ((N + 127) / 128);
+    int variant;
+    if (M >= 512) {
+        const int64_t pairs = dev.sm_count / 2;
+        const double c0 = static_cast<double>((pair_tiles + pairs - 1) / pairs);
+        const double c1 = static_cast<double>((tiles1 + dev.sm_count - 1) / dev.sm_count) / 0.8;
+        const double c2 = static_cast<double>((tiles2 + dev.sm_count - 1) / dev.sm_count) * 0.5 / 0.62;
+        variant = (c0 <= c1 && c0 <= c2) ? 0 : (c1 <= c2 ? 1 : 2);
+    } else if (pair_tiles >= dev.sm_count / 2) {
         variant = 0;
-    else if (tiles_m128 * ((N + 255) / 256) >= dev.sm_count && forced_variant() != 2)
+    } else if (tiles1 >= dev.sm_count) {
         variant = 1;
-    else
+    } else {
         variant = 2;
+    }
     if (forced_variant() >= 0 && forced_variant() <= 2) variant = forced_variant();
     const int bm = variant == 0 ? kPairBM : kGemmBM;
     const int bn = variant == 2 ? 128 : 256;
@@ -260,7 +276,6 @@ static int gemm_run(const void* A, const void* B, void* C, int64_t M, int64_t N,
     p.ldcf = ldc;
     p.accumulate = accumulate ? 1 : 0;
     p.f16_inputs = f16_in ? 1u : 0u;
-    p.c_tma = c_tma ? 1 : 0;
     if (variant == 2 && workspace && !f32_out) {
         // Few tiles (skinny or small problem): cut K into slices so that about two work items per SM exist; the
         // weights are then streamed by all SMs at once.  FP32 partials go to the caller's scratch.
@@ -278,14 +293,21 @@ static int gemm_run(const void* A, const void* B, void* C, int64_t M, int64_t N,
         // M-tiles per raster group: wide problems re-read B once per group, so fewer, taller groups pay
         p.group_m = debug_env_int("MLT_GEMM_GROUP_M", tiles_n >= 32 ? 16 : 8);
         const int clusters = static_cast<int>(std::min<int64_t>(tiles_m * tiles_n, dev.sm_count / 2));
-        gemm_bf16_pair_kernel<6><<<2 * clusters, kGemmThreads, GemmPairSmem<6>::kTotal, st>>>(ta, tb, tc, p);
+        if (c_tma)
+            gemm_bf16_pair_kernel<6, true><<<2 * clusters, kGemmThreads, GemmPairSmem<6>::kTotal, st>>>(ta, tb, tc, p);
+        else
+            gemm_bf16_pair_kernel<6, false><<<2 * clusters, kGemmThreads, GemmPairSmem<6>::kNoStaging, st>>>(ta, tb, tc, p);
     } else {
         p.group_m = 16;
         const int grid = static_cast<int>(std::min<int64_t>(tiles_m * tiles_n * p.split_k, dev.sm_count));
-        if (variant == 1)
-            gemm_bf16_kernel<256, 4><<<grid, kGemmThreads, GemmSmem<256, 4>::kTotal, st>>>(ta, tb, tc, p);
+        if (variant == 1 && c_tma)
+            gemm_bf16_kernel<256, 4, true><<<grid, kGemmThreads, GemmSmem<256, 4>::kTotal, st>>>(ta, tb, tc, p);
+        else if (variant == 1)
+            gemm_bf16_kernel<256, 4, false><<<grid, kGemmThreads, GemmSmem<256, 4>::kNoStaging, st>>>(ta, tb, tc, p);
+        else if (c_tma)
+            gemm_bf16_kernel<128, 6, true><<<grid, kGemmThreads, GemmSmem<128, 6>::kTotal, st>>>(ta, tb, tc, p);
         else
-            gemm_bf16_kernel<128, 6><<<grid, kGemmThreads, GemmSmem<128, 6>::kTotal, st>>>(ta, tb, tc, p);
+            gemm_bf16_kernel<128, 6, false><<<grid, kGemmThreads, GemmSmem<128, 6>::kNoStaging, st>>>(ta, tb, tc, p);
         if (p.split_k > 1) {
             if (cudaGetLastError() != cudaSuccess) return MLT_ERR_CUDA;
             const int64_t groups = M * ((N + 7) / 8);
