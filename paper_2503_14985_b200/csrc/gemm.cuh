@@ -47,6 +47,9 @@ struct GemmParams {
     float* Cf;         // non-null: FP32 output with pitch ldcf instead of BF16 C
     int64_t ldcf;
     int accumulate;    // with Cf: add to the prior contents of C (the "C += A*B" of Sec. 2)
+    // CTA-pair kernel: work items 0 .. full_items-1 are whole 256 x 256 tiles; the tiles after them (a last wave that
+    // would occupy at most half of the SM pairs) are cut into two 256 x 128 halves, one item each
+    int full_items, num_items;
     uint32_t f16_inputs;  // 0: BF16 operands, 1: FP16 operands (same tiles and descriptors, other format field)
 };
 
@@ -138,6 +141,20 @@ __device__ __forceinline__ void gemm_store_chunk_tma(const GemmParams& p, const 
             const int col = col0 + j;
             if (col >= n4 && col < p.N) crow[col] = p.accumulate ? crow[col] + __uint_as_float(v[j]) : __uint_as_float(v[j]);
         }
+    }
+}
+
+// CTA-pair kernel: work item -> (tile, first column inside the tile, width)
+__device__ __forceinline__ void gemm_pair_item(const GemmParams& p, int item, int& tile, int& n_off, int& bn) {
+    if (item < p.full_items) {
+        tile = item;
+        n_off = 0;
+        bn = 256;
+    } else {
+        const int r = item - p.full_items;
+        tile = p.full_items + (r >> 1);
+        n_off = (r & 1) * 128;
+        bn = 128;
     }
 }
 
@@ -358,7 +375,6 @@ gemm_bf16_pair_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_c
     const bool leader = rank == 0;
     const int cluster_id = blockIdx.x >> 1;
     const int num_clusters = gridDim.x >> 1;
-    const int num_tiles = p.tiles_m * p.tiles_n;
     const int num_kb = (p.K + kGemmBK - 1) / kGemmBK;
     constexpr uint32_t kTmemCols = 512;  // two 256-column accumulators
 
@@ -393,21 +409,23 @@ gemm_bf16_pair_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_c
             int stage = 0;
             uint32_t phase = 0;
             bool ok = true;
-            for (int tile = cluster_id; tile < num_tiles && ok; tile += num_clusters) {
-                int tm, tn;
+            for (int item = cluster_id; item < p.num_items && ok; item += num_clusters) {
+                int tile, n_off, bn, tm, tn;
+                gemm_pair_item(p, item, tile, n_off, bn);
                 gemm_tile_coords(p, tile, tm, tn);
                 const int m0 = tm * kPairBM + static_cast<int>(rank) * 128;
-                const int n0 = tn * kPairBN + static_cast<int>(rank) * 128;
+                const int n0 = tn * kPairBN + n_off + static_cast<int>(rank) * (bn >> 1);  // this CTA's bn/2 columns of B
+                const uint32_t tx = 2u * (L::kABytes + (bn >> 1) * kGemmBK * 2);
                 for (int kb = 0; kb < num_kb; ++kb) {
                     ok = mbar_wait(&empty[stage], phase ^ 1, abort_flag, 0x100 + stage);
                     if (!ok) break;
                     uint8_t* sa = smem + stage * L::kStageBytes;
                     uint8_t* sb = sa + L::kABytes;
-                    if (leader) mbar_arrive_expect_tx(&full[stage], 2 * L::kStageBytes);
+                    if (leader) mbar_arrive_expect_tx(&full[stage], tx);
                     const uint32_t bar = map_to_cta(smem_u32(&full[stage]), 0);
                     tma_load_2d_pair(sa, &tmap_a, bar, kb * kGemmBK, m0);
                     tma_load_2d_pair(sb, &tmap_b, bar, n0, kb * kGemmBK);
-                    tma_load_2d_pair(sb + kGemmBK * 128, &tmap_b, bar, n0 + 64, kb * kGemmBK);
+                    if (bn == 256) tma_load_2d_pair(sb + kGemmBK * 128, &tmap_b, bar, n0 + 64, kb * kGemmBK);
                     if (++stage == kStages) { stage = 0; phase ^= 1; }
                 }
             }
@@ -417,7 +435,8 @@ gemm_bf16_pair_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_c
         if (leader) {
             // whole warp, uniform control flow; one elected lane executes the tcgen05 instructions
             const bool issuer = elect_one();
-            const uint32_t idesc = gemm_idesc(kPairBM, kPairBN, p.f16_inputs);
+            const uint32_t idesc_full = gemm_idesc(kPairBM, kPairBN, p.f16_inputs);
+            const uint32_t idesc_half = gemm_idesc(kPairBM, kPairBN / 2, p.f16_inputs);
             const uint32_t a_lo0 = sdesc_lo(smem_u32(smem), 16);
             const uint32_t b_lo0 = sdesc_lo(smem_u32(smem + L::kABytes), kGemmBK * 128);
             int stage = 0;
@@ -425,10 +444,11 @@ gemm_bf16_pair_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_c
             int acc = 0;
             uint32_t acc_phase = 0;
             bool ok = true;
-            for (int tile = cluster_id; tile < num_tiles && ok; tile += num_clusters) {
+            for (int item = cluster_id; item < p.num_items && ok; item += num_clusters) {
                 ok = __all_sync(0xffffffffu, mbar_wait(&acc_empty[acc], acc_phase ^ 1, abort_flag, 0x300 + acc));
                 if (!ok) break;
                 tc_fence_after();
+                const uint32_t idesc = item < p.full_items ? idesc_full : idesc_half;
                 const uint32_t d_tmem = tmem_base + acc * kPairBN;
                 for (int kb = 0; kb < num_kb; ++kb) {
                     ok = __all_sync(0xffffffffu, mbar_wait(&full[stage], phase, abort_flag, 0x200 + stage));
@@ -456,17 +476,18 @@ gemm_bf16_pair_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_c
         int acc = 0;
         uint32_t acc_phase = 0;
         bool ok = true;
-        for (int tile = cluster_id; tile < num_tiles && ok; tile += num_clusters) {
-            int tm, tn;
+        for (int item = cluster_id; item < p.num_items && ok; item += num_clusters) {
+            int tile, n_off, bn, tm, tn;
+            gemm_pair_item(p, item, tile, n_off, bn);
             gemm_tile_coords(p, tile, tm, tn);
             const int row = tm * kPairBM + static_cast<int>(rank) * 128 + quarter * 32 + lane;
-            const int n0 = tn * kPairBN;
+            const int n0 = tn * kPairBN + n_off;
             ok = __all_sync(0xffffffffu, mbar_wait(&acc_full[acc], acc_phase, abort_flag, 0x400 + acc));
             if (!ok) break;
             tc_fence_after();
             const uint32_t t_row = tmem_base + (static_cast<uint32_t>(quarter * 32) << 16) + acc * kPairBN;
 #pragma unroll 1
-            for (int c = 0; c < kPairBN / 32; ++c) {
+            for (int c = 0; c < bn / 32; ++c) {
                 uint32_t v[32];
                 tmem_ld_32x32b_x32(t_row + c * 32, v);
                 tmem_wait_ld();

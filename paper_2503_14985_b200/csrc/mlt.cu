@@ -276,6 +276,7 @@ static int gemm_run(const void* A, const void* B, void* C, int64_t M, int64_t N,
     p.ldcf = ldc;
     p.accumulate = accumulate ? 1 : 0;
     p.f16_inputs = f16_in ? 1u : 0u;
+    p.full_items = p.num_items = 0;
     if (variant == 2 && workspace && !f32_out) {
         // Few tiles (skinny or small problem): cut K into slices so that about two work items per SM exist; the
         // weights are then streamed by all SMs at once.  FP32 partials go to the caller's scratch.
@@ -292,7 +293,13 @@ static int gemm_run(const void* A, const void* B, void* C, int64_t M, int64_t N,
     if (variant == 0) {
         // M-tiles per raster group: wide problems re-read B once per group, so fewer, taller groups pay
         p.group_m = debug_env_int("MLT_GEMM_GROUP_M", tiles_n >= 32 ? 16 : 8);
-        const int clusters = static_cast<int>(std::min<int64_t>(tiles_m * tiles_n, dev.sm_count / 2));
+        // A last wave that would occupy at most half of the SM pairs runs as twice as many 256 x 128 half tiles
+        const int pairs = dev.sm_count / 2;
+        const int num_tiles = static_cast<int>(tiles_m * tiles_n);
+        const int rem = num_tiles % pairs;
+        p.full_items = (rem > 0 && 2 * rem <= pairs && debug_env_int("MLT_GEMM_NO_HALF", 0) == 0) ? num_tiles - rem : num_tiles;
+        p.num_items = p.full_items + 2 * (num_tiles - p.full_items);
+        const int clusters = std::min(p.num_items, pairs);
         if (c_tma)
             gemm_bf16_pair_kernel<6, true><<<2 * clusters, kGemmThreads, GemmPairSmem<6>::kTotal, st>>>(ta, tb, tc, p);
         else
