@@ -151,8 +151,9 @@ int mlt_paged_attn_decode(const void* Q, const void* K_cache, const void* V_cach
  *
  * Arguments, layouts, results and errors are those of mlt_paged_attn_decode, without the workspace pair.  The
  * split over CTAs is the one mlt_paged_attn_decode makes with a full workspace, so the outputs are the same;
- * it needs num_seqs * H * splits * (4 * D + 8) bytes with splits <= 32 (splits = ceil(max_blocks_per_seq / 16),
- * or / 8 for few sequences), and a call that needs more than the array holds returns MLT_ERR_SCRATCH_LIMIT
+ * it needs num_seqs * H * splits * (4 * D + 8) bytes with splits <= 32 (splits = ceil(max_blocks_per_seq / 16), / 32
+ * with 4 or 8 query heads per KV head, half as many blocks per split for few sequences), and a call that needs more
+ * than the array holds returns MLT_ERR_SCRATCH_LIMIT
  * and launches nothing.
  *
  * The first call on each device looks up the array's device address (with that device current); make that first

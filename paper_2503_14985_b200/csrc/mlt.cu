@@ -422,8 +422,10 @@ int paged_prepare(const void* Q, const void* K_cache, const void* V_cache, const
     p->block_size = block_size;
     p->max_blocks = max_blocks_per_seq;
     p->num_blocks = num_blocks;
-    p->splits = paged_choose_splits(num_seqs, H_kv, max_blocks_per_seq, dev->sm_count);
+    p->splits = paged_choose_splits(num_seqs, H_kv, H / H_kv, max_blocks_per_seq, dev->sm_count);
+    p->splits = debug_env_int("MLT_PAGED_SPLITS", p->splits);
     p->scale_log2e = scale * 1.4426950408889634f;
+    p->head_groups = 1;
     *launch = true;
     return MLT_OK;
 }

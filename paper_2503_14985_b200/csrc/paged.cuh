@@ -45,6 +45,7 @@ struct PagedParams {
     int blocks_per_split;  // KV blocks each of them covers: the same for every sequence, so CTAs do equal work and
                            // the CTAs beyond a short sequence's end exit at once
     float scale_log2e;
+    int head_groups;       // CTAs per KV head (1, or 2 when 8 query heads per KV head run as two groups of 4)
 };
 
 __device__ __forceinline__ void bf16x8_to_f32(const uint4& v, float (&f)[8]) {
@@ -56,11 +57,59 @@ __device__ __forceinline__ void bf16x8_to_f32(const uint4& v, float (&f)[8]) {
     }
 }
 
+__device__ __forceinline__ void bf16x8_to_f32x2(const uint4& v, float2 (&f)[4]) {
+    const uint32_t w[4] = {v.x, v.y, v.z, v.w};
+#pragma unroll
+    for (int i = 0; i < 4; ++i) f[i] = make_float2(__uint_as_float(w[i] << 16), __uint_as_float(w[i] & 0xFFFF0000u));
+}
+
 // merge partial {m, l, o} states a and b (log2-domain maxima); -inf maxima stand for "nothing seen"
 __device__ __forceinline__ void paged_merge_scale(float ma, float mb, float& m, float& sa, float& sb) {
     m = fmaxf(ma, mb);
     sa = (ma == -INFINITY) ? 0.0f : fast_exp2(ma - m);
     sb = (mb == -INFINITY) ? 0.0f : fast_exp2(mb - m);
+}
+
+// Sum over the LPT lanes of a token of G partial dot products, scattered: every stage halves the number of values
+// a lane carries (lanes with the stage's bit clear keep the lower half of their list, the others the upper half)
+// until one is left, so G heads cost G - 1 + log2(LPT / G) shuffles instead of G * log2(LPT).  Returns the complete
+// sum of head paged_my_head(sub); lanes whose `sub` agree in the low log2(G) bits hold the same head.
+template <int G, int LPT>
+__device__ __forceinline__ float paged_reduce_scatter(float (&d)[G], int sub) {
+    int n = G;
+#pragma unroll
+    for (int mask = 1; mask < LPT; mask <<= 1) {
+        if (n > 1) {
+            const int half = n / 2;
+            const bool upper = (sub & mask) != 0;
+#pragma unroll
+            for (int j = 0; j < G / 2; ++j) {
+                if (j < half) {
+                    const float send = upper ? d[j] : d[j + half];
+                    const float keep = upper ? d[j + half] : d[j];
+                    d[j] = keep + __shfl_xor_sync(0xffffffffu, send, mask);
+                }
+            }
+            n = half;
+        } else {
+            d[0] += __shfl_xor_sync(0xffffffffu, d[0], mask);
+        }
+    }
+    return d[0];
+}
+template <int G>
+__device__ __forceinline__ int paged_my_head(int sub) {  // the head whose sum paged_reduce_scatter leaves in this lane
+    int g = 0, half = G / 2;
+    for (int mask = 1; half > 0; mask <<= 1, half >>= 1)
+        if (sub & mask) g += half;
+    return g;
+}
+template <int G>
+__device__ __forceinline__ int paged_head_sub(int g) {  // the lowest `sub` that holds head g
+    int sub = 0, half = G / 2;
+    for (int mask = 1; half > 0; mask <<= 1, half >>= 1)
+        if (g & half) sub |= mask;
+    return sub;
 }
 
 template <int D, int G, int BS>
@@ -74,7 +123,10 @@ paged_decode_kernel(const PagedParams p) {
     __shared__ float2 sm_ml[kPagedWarps][G];
 
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
-    const int sp = blockIdx.x, kvh = blockIdx.y, s = blockIdx.z;
+    // blockIdx.y = KV head x head group: with more query heads per KV head than G, several CTAs share a KV head
+    // (p.head_groups of them, G heads each; the second reads K and V from L2)
+    const int sp = blockIdx.x, kvh = blockIdx.y / p.head_groups, s = blockIdx.z;
+    const int head0 = kvh * (G * p.head_groups) + (blockIdx.y % p.head_groups) * G;  // first query head of this CTA
     const int sub = lane % LPT;   // which 8 columns of D this lane owns
     const int grp = lane / LPT;   // which token of a step
     const int len = p.seq_lens[s];
@@ -84,20 +136,23 @@ paged_decode_kernel(const PagedParams p) {
     if (p.splits > 1 && b0 >= nblk && !(sp == 0)) return;  // nothing of this sequence here (split 0 reports an empty one)
 
     // this lane's 8 columns of the G query rows
-    float q[G][8];
+    float2 q[G][4];  // pairs: the products below are packed (fma.rn.f32x2), two columns per instruction
 #pragma unroll
     for (int g = 0; g < G; ++g) {
-        const uint4 v = *reinterpret_cast<const uint4*>(p.Q + (static_cast<int64_t>(s) * p.H + kvh * G + g) * D + sub * 8);
-        bf16x8_to_f32(v, q[g]);
+        const uint4 v = *reinterpret_cast<const uint4*>(p.Q + (static_cast<int64_t>(s) * p.H + head0 + g) * D + sub * 8);
+        bf16x8_to_f32x2(v, q[g]);
     }
-    float m[G], l[G], o[G][8];
+    // Running max and sum are kept for one head per lane (the head whose scores the scattered reduction leaves
+    // here); the output accumulators cover this lane's 8 columns of all G heads.
+    const int my_g = paged_my_head<G>(sub);
+    float m_own = -INFINITY, l_own = 0.0f;
+    float2 o[G][4];
 #pragma unroll
     for (int g = 0; g < G; ++g) {
-        m[g] = -INFINITY;
-        l[g] = 0.0f;
 #pragma unroll
-        for (int e = 0; e < 8; ++e) o[g][e] = 0.0f;
+        for (int e = 0; e < 4; ++e) o[g][e] = make_float2(0.0f, 0.0f);
     }
+    (void)my_g;
 
     const int* table = p.block_table + static_cast<int64_t>(s) * p.max_blocks;
     for (int b = b0 + warp; b < b1; b += kPagedWarps) {
@@ -118,55 +173,74 @@ paged_decode_kernel(const PagedParams p) {
         for (int i = 0; i < STEPS; ++i) kr[i] = *reinterpret_cast<const uint4*>(kp + (i * TPS + grp) * D);
 #pragma unroll
         for (int i = 0; i < STEPS; ++i) vr[i] = *reinterpret_cast<const uint4*>(vp + (i * TPS + grp) * D);
-        // scores of this lane group's STEPS tokens for each head (log2 domain), masked beyond the length
-        float sc[G][STEPS];
+        // score of this lane's head for each of the lane group's STEPS tokens (log2 domain), masked beyond the length
+        float sc[STEPS];
 #pragma unroll
         for (int i = 0; i < STEPS; ++i) {
-            float kf[8];
-            bf16x8_to_f32(kr[i], kf);
+            float2 kf[4];
+            bf16x8_to_f32x2(kr[i], kf);
             const bool visible = b * BS + i * TPS + grp < len;
+            float d[G];
 #pragma unroll
             for (int g = 0; g < G; ++g) {
-                float d = 0.0f;
+                float2 d2 = make_float2(0.0f, 0.0f);
 #pragma unroll
-                for (int e = 0; e < 8; ++e) d = fmaf(q[g][e], kf[e], d);
-#pragma unroll
-                for (int w = LPT / 2; w > 0; w >>= 1) d += __shfl_xor_sync(0xffffffffu, d, w);
-                sc[g][i] = visible ? d * p.scale_log2e : -INFINITY;
+                for (int e = 0; e < 4; ++e) d2 = ffma2(q[g][e], kf[e], d2);
+                d[g] = d2.x + d2.y;
             }
+            const float dot = paged_reduce_scatter<G, LPT>(d, sub);
+            sc[i] = visible ? dot * p.scale_log2e : -INFINITY;
         }
-        // one online-softmax update per block and head
-        float pw[G][STEPS];
+        // one online-softmax update per block, for this lane's head: one exponential per (head, token) and lane
+        float pw[STEPS];
+        float alpha;
+        {
+            float mb = sc[0];
 #pragma unroll
-        for (int g = 0; g < G; ++g) {
-            float mb = sc[g][0];
-#pragma unroll
-            for (int i = 1; i < STEPS; ++i) mb = fmaxf(mb, sc[g][i]);
-            const float mn = fmaxf(m[g], mb);
-            const float alpha = (m[g] == -INFINITY) ? 0.0f : fast_exp2(m[g] - mn);
+            for (int i = 1; i < STEPS; ++i) mb = fmaxf(mb, sc[i]);
+            const float mn = fmaxf(m_own, mb);
+            alpha = (m_own == -INFINITY) ? 0.0f : fast_exp2(m_own - mn);
             const float ref = (mn == -INFINITY) ? 0.0f : mn;
             float sum = 0.0f;
 #pragma unroll
             for (int i = 0; i < STEPS; ++i) {
-                pw[g][i] = fast_exp2(sc[g][i] - ref);
-                sum += pw[g][i];
+                pw[i] = fast_exp2(sc[i] - ref);
+                sum += pw[i];
             }
-            m[g] = mn;
-            l[g] = l[g] * alpha + sum;
+            m_own = mn;
+            l_own = l_own * alpha + sum;
+        }
+        // rescale and accumulate all heads' outputs: the factors come from the lanes that hold each head
+        const int lane0 = grp * LPT;  // first lane of this token group
 #pragma unroll
-            for (int e = 0; e < 8; ++e) o[g][e] *= alpha;
+        for (int g = 0; g < G; ++g) {
+            const float ag = G == 1 ? alpha : __shfl_sync(0xffffffffu, alpha, lane0 + paged_head_sub<G>(g));
+#pragma unroll
+            for (int e = 0; e < 4; ++e) o[g][e] = make_float2(o[g][e].x * ag, o[g][e].y * ag);
         }
 #pragma unroll
         for (int i = 0; i < STEPS; ++i) {
-            float vf[8];
+            float2 vf[4];
             // bytes past the sequence's last token are whatever the cache holds: weight 0 must not meet a NaN
             if (b * BS + i * TPS + grp >= len) vr[i] = make_uint4(0u, 0u, 0u, 0u);
-            bf16x8_to_f32(vr[i], vf);
+            bf16x8_to_f32x2(vr[i], vf);
 #pragma unroll
-            for (int g = 0; g < G; ++g)
+            for (int g = 0; g < G; ++g) {
+                const float pg = G == 1 ? pw[i] : __shfl_sync(0xffffffffu, pw[i], lane0 + paged_head_sub<G>(g));
+                const float2 pg2 = make_float2(pg, pg);
 #pragma unroll
-                for (int e = 0; e < 8; ++e) o[g][e] = fmaf(pw[g][i], vf[e], o[g][e]);
+                for (int e = 0; e < 4; ++e) o[g][e] = ffma2(pg2, vf[e], o[g][e]);
+            }
         }
+    }
+
+    // every lane needs all heads' running max and sum for the merges below
+    float m[G], l[G];
+#pragma unroll
+    for (int g = 0; g < G; ++g) {
+        const int src = (lane / LPT) * LPT + paged_head_sub<G>(g);
+        m[g] = G == 1 ? m_own : __shfl_sync(0xffffffffu, m_own, src);
+        l[g] = G == 1 ? l_own : __shfl_sync(0xffffffffu, l_own, src);
     }
 
     // merge the TPS lane groups of the warp (lanes that own the same columns), then the warps through smem
@@ -180,15 +254,19 @@ paged_decode_kernel(const PagedParams p) {
             paged_merge_scale(m[g], mo, mn, sa, sb);
             l[g] = l[g] * sa + lo * sb;
 #pragma unroll
-            for (int e = 0; e < 8; ++e) {
-                const float oo = __shfl_xor_sync(0xffffffffu, o[g][e], w);
-                o[g][e] = o[g][e] * sa + oo * sb;
+            for (int e = 0; e < 4; ++e) {
+                const float ox = __shfl_xor_sync(0xffffffffu, o[g][e].x, w);
+                const float oy = __shfl_xor_sync(0xffffffffu, o[g][e].y, w);
+                o[g][e] = make_float2(o[g][e].x * sa + ox * sb, o[g][e].y * sa + oy * sb);
             }
             m[g] = mn;
         }
         if (grp == 0) {
 #pragma unroll
-            for (int e = 0; e < 8; ++e) sm_o[warp][g][sub * 8 + e] = o[g][e];
+            for (int e = 0; e < 4; ++e) {
+                sm_o[warp][g][sub * 8 + 2 * e] = o[g][e].x;
+                sm_o[warp][g][sub * 8 + 2 * e + 1] = o[g][e].y;
+            }
             if (sub == 0) sm_ml[warp][g] = make_float2(m[g], l[g]);
         }
     }
@@ -206,7 +284,7 @@ paged_decode_kernel(const PagedParams p) {
             lt += ml.y * sw;
             ot += sm_o[w][g][d] * sw;
         }
-        const int64_t row = static_cast<int64_t>(s) * p.H + kvh * G + g;
+        const int64_t row = static_cast<int64_t>(s) * p.H + head0 + g;
         if (p.splits == 1) {
             p.O[row * D + d] = __float2bfloat16(lt > 0.0f ? ot / lt : 0.0f);
             if (d == 0 && p.LSE) p.LSE[row] = lt > 0.0f ? (mt + log2f(lt)) * 0.6931471805599453f : -INFINITY;
@@ -269,17 +347,19 @@ inline size_t paged_workspace_bytes(int num_seqs, int H, int D, int splits) {
 // short sequence's end are empty: aim at 16 blocks (256 tokens) per CTA, which leaves enough busy CTAs per SM to
 // hide the HBM latency even when most sequences are shorter than the longest allowed; 8 blocks if that still
 // leaves SMs idle; no split when there are already many (sequence, KV head) pairs per SM.
-inline int paged_choose_splits(int num_seqs, int H_kv, int max_blocks, int sm_count) {
+// With 4 or 8 query heads per KV head a CTA computes more per byte and writes a larger partial: 32 blocks per CTA.
+inline int paged_choose_splits(int num_seqs, int H_kv, int group, int max_blocks, int sm_count) {
     const int64_t base = static_cast<int64_t>(num_seqs) * H_kv;
     if (base >= 16ll * sm_count) return 1;
-    int splits = (max_blocks + 15) / 16;
-    if (base * splits < 4ll * sm_count) splits = (max_blocks + 7) / 8;
+    const int per_cta = group >= 4 ? 32 : 16;
+    int splits = (max_blocks + per_cta - 1) / per_cta;
+    if (base * splits < 4ll * sm_count) splits = (max_blocks + per_cta / 2 - 1) / (per_cta / 2);
     return std::max(1, std::min(splits, kPagedMaxSplits));
 }
 
 template <int D, int G>
 int paged_launch_bs(const PagedParams& p, cudaStream_t st) {
-    const dim3 grid(p.splits, p.H_kv, p.num_seqs);
+    const dim3 grid(p.splits, p.H_kv * p.head_groups, p.num_seqs);
     switch (p.block_size) {
         case 8: paged_decode_kernel<D, G, 8><<<grid, kPagedThreads, 0, st>>>(p); break;
         case 16: paged_decode_kernel<D, G, 16><<<grid, kPagedThreads, 0, st>>>(p); break;
@@ -300,7 +380,12 @@ int paged_launch_g(const PagedParams& p, cudaStream_t st) {
         case 1: return paged_launch_bs<D, 1>(p, st);
         case 2: return paged_launch_bs<D, 2>(p, st);
         case 4: return paged_launch_bs<D, 4>(p, st);
-        case 8: return paged_launch_bs<D, 8>(p, st);
+        case 8: {
+            // 8 heads per CTA need 255 registers and leave two CTAs per SM; two CTAs of 4 heads run faster
+            PagedParams p2 = p;
+            p2.head_groups = 2;
+            return paged_launch_bs<D, 4>(p2, st);
+        }
         default: return 2;
     }
 }
