@@ -220,6 +220,8 @@ static int gemm_run(const void* A, const void* B, void* C, int64_t M, int64_t N,
         const double c1 = static_cast<double>((tiles1 + dev.sm_count - 1) / dev.sm_count) / 0.8;
         const double c2 = static_cast<double>((tiles2 + dev.sm_count - 1) / dev.sm_count) * 0.5 / 0.62;
         variant = (c0 <= c1 && c0 <= c2) ? 0 : (c1 <= c2 ? 1 : 2);
+    } else if (workspace && !f32_out && gemm_max_split(M, N, K) > 1) {
+        variant = 2;  // memory-bound with scratch: small tiles cut along K spread the stream of B evenly over the SMs
     } else if (pair_tiles >= dev.sm_count / 2) {
         variant = 0;
     } else if (tiles1 >= dev.sm_count) {
@@ -281,9 +283,22 @@ static int gemm_run(const void* A, const void* B, void* C, int64_t M, int64_t N,
         // Few tiles (skinny or small problem): cut K into slices so that about two work items per SM exist; the
         // weights are then streamed by all SMs at once.  FP32 partials go to the caller's scratch.
         const int num_kb = p.kb_per_split;
-        int split = static_cast<int>(std::min<int64_t>(gemm_max_split(M, N, K),
-                                                        (2ll * dev.sm_count + tiles_m * tiles_n - 1) / (tiles_m * tiles_n)));
-        while (split > 1 && static_cast<size_t>(split) * M * N * sizeof(float) > workspace_bytes) --split;
+        // Slices: the count that minimises rounds x (K blocks per slice + fill/drain of an item) plus the time to
+        // write and re-read the FP32 partials, all in units of one K block of one tile (16 KB of B per SM).
+        const int64_t tiles = tiles_m * tiles_n;
+        int max_split = gemm_max_split(M, N, K);
+        while (max_split > 1 && static_cast<size_t>(max_split) * M * N * sizeof(float) > workspace_bytes) --max_split;
+        int split = 1;
+        double best = 1e300;
+        for (int sl = 1; sl <= max_split; ++sl) {
+            const int kbps = (num_kb + sl - 1) / sl;
+            const int slices = (num_kb + kbps - 1) / kbps;
+            if (slices != sl) continue;  // the same slicing as a smaller count
+            const int64_t rounds = (tiles * slices + dev.sm_count - 1) / dev.sm_count;
+            const double partial = sl > 1 ? static_cast<double>(sl) * M * N * 8.0 / (16384.0 * dev.sm_count) : 0.0;
+            const double cost = static_cast<double>(rounds) * (kbps + 4) + partial;
+            if (cost < best) { best = cost; split = sl; }
+        }
         if (split > 1) {
             p.kb_per_split = (num_kb + split - 1) / split;
             p.split_k = (num_kb + p.kb_per_split - 1) / p.kb_per_split;  // no empty slice
