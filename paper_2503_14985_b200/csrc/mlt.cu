@@ -116,9 +116,23 @@ int forced_variant() {
     return v;
 }
 
-int debug_env_int(const char* name, int fallback) {
-    const char* e = std::getenv(name);
-    return e && std::atoi(e) > 0 ? std::atoi(e) : fallback;
+// Debug only: tuning overrides read once from the environment (0 = not set).  MLT_GEMM_GROUP_M: M-tiles per raster
+// group of the pair kernel; MLT_GEMM_NO_HALF: no half tiles in the last wave; MLT_MHA_HEAD_GROUP / MLT_MHA_GRID: item
+// list grouping and CTA count of the attention kernel; MLT_PAGED_SPLITS: CTAs per (sequence, KV head).
+struct DebugEnv {
+    int gemm_group_m, gemm_no_half, mha_head_group, mha_grid, paged_splits;
+};
+const DebugEnv& debug_env() {
+    static const DebugEnv env = [] {
+        auto get = [](const char* name) {
+            const char* e = std::getenv(name);
+            const int v = e ? std::atoi(e) : 0;
+            return v > 0 ? v : 0;
+        };
+        return DebugEnv{get("MLT_GEMM_GROUP_M"), get("MLT_GEMM_NO_HALF"), get("MLT_MHA_HEAD_GROUP"), get("MLT_MHA_GRID"),
+                        get("MLT_PAGED_SPLITS")};
+    }();
+    return env;
 }
 
 inline bool aligned16(const void* p) { return (reinterpret_cast<uintptr_t>(p) & 15u) == 0; }
@@ -307,12 +321,12 @@ static int gemm_run(const void* A, const void* B, void* C, int64_t M, int64_t N,
     }
     if (variant == 0) {
         // M-tiles per raster group: wide problems re-read B once per group, so fewer, taller groups pay
-        p.group_m = debug_env_int("MLT_GEMM_GROUP_M", tiles_n >= 32 ? 16 : 8);
+        p.group_m = debug_env().gemm_group_m ? debug_env().gemm_group_m : (tiles_n >= 32 ? 16 : 8);
         // A last wave that would occupy at most half of the SM pairs runs as twice as many 256 x 128 half tiles
         const int pairs = dev.sm_count / 2;
         const int num_tiles = static_cast<int>(tiles_m * tiles_n);
         const int rem = num_tiles % pairs;
-        p.full_items = (rem > 0 && 2 * rem <= pairs && debug_env_int("MLT_GEMM_NO_HALF", 0) == 0) ? num_tiles - rem : num_tiles;
+        p.full_items = (rem > 0 && 2 * rem <= pairs && !debug_env().gemm_no_half) ? num_tiles - rem : num_tiles;
         p.num_items = p.full_items + 2 * (num_tiles - p.full_items);
         const int clusters = std::min(p.num_items, pairs);
         if (c_tma)
@@ -393,8 +407,8 @@ int mlt_mha_fwd(const void* Q, const void* K, const void* V, void* O, float* LSE
         if (rc != MLT_OK) return rc;
     }
     return mha_launch(tq, tk, tv, to, LSE, B, H, Nq, Nk, D, causal != 0, scale,
-                      dev.sm_count, static_cast<cudaStream_t>(stream), debug_env_int("MLT_MHA_HEAD_GROUP", 0),
-                      debug_env_int("MLT_MHA_GRID", 0));
+                      dev.sm_count, static_cast<cudaStream_t>(stream), debug_env().mha_head_group,
+                      debug_env().mha_grid);
 }
 
 size_t mlt_paged_attn_workspace_bytes(int num_seqs, int H, int D) {
@@ -438,7 +452,7 @@ int paged_prepare(const void* Q, const void* K_cache, const void* V_cache, const
     p->max_blocks = max_blocks_per_seq;
     p->num_blocks = num_blocks;
     p->splits = paged_choose_splits(num_seqs, H_kv, H / H_kv, max_blocks_per_seq, dev->sm_count);
-    p->splits = debug_env_int("MLT_PAGED_SPLITS", p->splits);
+    if (debug_env().paged_splits) p->splits = std::min(debug_env().paged_splits, kPagedMaxSplits);
     p->scale_log2e = scale * 1.4426950408889634f;
     p->head_groups = 1;
     *launch = true;
