@@ -52,7 +52,9 @@ CASES = [(1, 1, 128, 128, 64, 0), (1, 1, 128, 128, 128, 1), (1, 2, 1, 1, 64, 0),
          (1, 3, 300, 300, 64, 0), (2, 2, 257, 640, 128, 1), (1, 1, 512, 384 + 1, 64, 0), (1, 9, 384, 384, 64, 1),
          (1, 1, 1, 700, 128, 1),
          # more work items than SMs: a CTA runs several items one after another (ragged last pairs among them)
-         (3, 70, 300, 300, 64, 1), (2, 80, 300, 420, 128, 1), (5, 40, 520, 260, 128, 0), (2, 90, 257, 257, 64, 0)]
+         (3, 70, 300, 300, 64, 1), (2, 80, 300, 420, 128, 1), (5, 40, 520, 260, 128, 0), (2, 90, 257, 257, 64, 0),
+         # ... with a single K/V block per item, and with the second 128-row tile absent in every item
+         (2, 100, 256, 128, 64, 0), (2, 100, 256, 100, 128, 0), (3, 60, 128, 128, 64, 1), (3, 60, 100, 228, 128, 1)]
 
 
 @pytest.mark.parametrize("B,H,Nq,Nk,D,causal", CASES)
