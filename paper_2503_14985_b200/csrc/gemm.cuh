@@ -8,6 +8,14 @@
 //   warps 2-5   epilogue: TMEM -> registers -> BF16 -> global, overlapped with the next tile's main loop
 // Tile 128 x BN x 64, kStages-deep smem ring guarded by full/empty mbarriers; two
 // accumulators in TMEM (2 x BN columns) guarded by acc_full/acc_empty mbarriers.
+// Large problems run on CTA pairs (256 x 256 tiles, tcgen05.mma.cta_group::2; see gemm_bf16_pair_kernel).
+//
+// The same kernels serve three destinations of the accumulators (gemm_store_chunk / gemm_store_chunk_tma):
+//   BF16 C        one rounding to nearest even, 16-byte stores from the thread that owns the row
+//   FP32 partial  split-K: work item = (tile, K slice), a second kernel sums the slices in a fixed order
+//   FP32 C        FP16 or BF16 operands, result through a shared-memory box and a TMA store, or a TMA
+//                 add-reduction for C += A * B (template parameter kCTma: its own instantiation, so the BF16
+//                 path keeps its registers and code size)
 #pragma once
 
 #include "ptx.cuh"
