@@ -126,13 +126,15 @@ def test_dominant_key_and_outlier_rows():
     check_mha(o, lse, o_ref, lse_ref, "dominant last key")
 
 
-def test_deterministic_across_runs():
-    Q, K, V = inputs.mha_inputs(1, 4, 512, 512, 128, seed=265)
+@pytest.mark.parametrize("B,H,N,D,causal", [(1, 4, 512, 128, True), (3, 70, 300, 64, True), (2, 90, 600, 128, False)])
+def test_deterministic_across_runs(B, H, N, D, causal):
+    # the second and third shapes have more work items than SMs (several items per persistent CTA)
+    Q, K, V = inputs.mha_inputs(B, H, N, N, D, seed=265)
     dQ, dK, dV = to_dev(Q), to_dev(K), to_dev(V)
-    o1, l1 = mlt.mha_fwd(dQ, dK, dV, causal=True, scale=scale_for(128))
-    o2, l2 = mlt.mha_fwd(dQ, dK, dV, causal=True, scale=scale_for(128))
+    runs = [mlt.mha_fwd(dQ, dK, dV, causal=causal, scale=scale_for(D)) for _ in range(4)]
     torch.cuda.synchronize()
-    assert torch.equal(o1.view(torch.int16), o2.view(torch.int16)) and torch.equal(l1, l2)
+    for o, l in runs[1:]:
+        assert torch.equal(runs[0][0].view(torch.int16), o.view(torch.int16)) and torch.equal(runs[0][1], l)
 
 
 @pytest.mark.parametrize("name", list(inputs.MHA_CONFIGS))
