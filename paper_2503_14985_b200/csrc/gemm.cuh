@@ -533,8 +533,27 @@ __global__ void gemm_splitk_reduce_kernel(const float* partial, __nv_bfloat16* C
         const int col = static_cast<int>(i % groups_per_row) * 8;
         float acc[8] = {0, 0, 0, 0, 0, 0, 0, 0};
         const bool full = col + 8 <= N && (N & 3) == 0;
-        for (int s = 0; s < split_k; ++s) {
-            const float* src = partial + (static_cast<int64_t>(s) * M + row) * N + col;
+        const int64_t slice_pitch = static_cast<int64_t>(M) * N;
+        const float* src0 = partial + static_cast<int64_t>(row) * N + col;
+        int s = 0;
+        if (full) {
+            // four slices' loads in flight before the first addition (the additions keep the ascending slice order)
+            for (; s + 4 <= split_k; s += 4) {
+                float4 a[4], b[4];
+#pragma unroll
+                for (int u = 0; u < 4; ++u) {
+                    a[u] = *reinterpret_cast<const float4*>(src0 + (s + u) * slice_pitch);
+                    b[u] = *reinterpret_cast<const float4*>(src0 + (s + u) * slice_pitch + 4);
+                }
+#pragma unroll
+                for (int u = 0; u < 4; ++u) {
+                    acc[0] += a[u].x; acc[1] += a[u].y; acc[2] += a[u].z; acc[3] += a[u].w;
+                    acc[4] += b[u].x; acc[5] += b[u].y; acc[6] += b[u].z; acc[7] += b[u].w;
+                }
+            }
+        }
+        for (; s < split_k; ++s) {
+            const float* src = src0 + s * slice_pitch;
             if (full) {
                 const float4 a = *reinterpret_cast<const float4*>(src), b = *reinterpret_cast<const float4*>(src + 4);
                 acc[0] += a.x; acc[1] += a.y; acc[2] += a.z; acc[3] += a.w;
