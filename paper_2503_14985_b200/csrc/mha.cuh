@@ -269,6 +269,10 @@ mha_fwd_kernel(const __grid_constant__ CUtensorMap tmap_q, const __grid_constant
     constexpr uint32_t kColP = kEarlyQK ? 384 : kColS;  // P_t at kColP + t*(kEarlyQK ? 64 : 128)
     constexpr uint32_t kStrideP = kEarlyQK ? 64 : kMhaBlock;
 
+    // Register hand-over: setmaxnreg moves registers inside the CTA's launch allocation (384 threads x 168), it cannot
+    // draw on the rest of the register file.  232 for the softmax warps needs every other warp down at 40; one
+    // register more anywhere and the increase below would wait for ever.
+    static_assert(8 * 32 * 232 + 4 * 32 * 40 <= kMhaThreads * 168, "setmaxnreg budget exceeds the launch allocation");
     if (warp >= 10) {
         setmaxnreg_dec<40>();  // only hand their registers over
     } else if (warp == 9) {
