@@ -29,6 +29,11 @@ def inputs_lines():
     Q, K, V = inputs.mha_inputs(1, 2, 16, 24, 64, seed=6, outlier_percent=1)
     out.append("mha seed6 1x2x16x24x64 outliers sha256 " + hashlib.sha256(Q.tobytes() + K.tobytes() + V.tobytes()).hexdigest())
     out.append("mha seed6 Q[0,0,0,:8] " + " ".join(f"{v:04x}" for v in Q[0, 0, 0, :8]))
+    A, B, C = inputs.gemm_f16_inputs(8, 8, 8, seed=3, kind="normal")
+    out.append("gemm_f16 normal seed3 A[0,:8] " + " ".join(f"{v:04x}" for v in A[0]))
+    out.append("gemm_f16 normal seed3 sha256 " + hashlib.sha256(A.tobytes() + B.tobytes() + C.tobytes()).hexdigest())
+    Qp, Kc, Vc, table, lens = inputs.paged_inputs(3, 4, 2, 64, 8, seed=9, min_len=5, max_len=40)[:5]
+    out.append("paged seed9 sha256 " + hashlib.sha256(Qp.tobytes() + Kc.tobytes() + Vc.tobytes() + table.tobytes() + lens.tobytes()).hexdigest())
     return out
 
 
@@ -42,6 +47,9 @@ def oracle_lines():
     O, L = oracle.mha_fwd(Q, K, V, causal=True, scale=np.float32(0.5))
     for row, l in zip(O, L):
         out.append("mha 3x5x4 causal " + " ".join(float(v).hex() for v in row) + " lse " + float(l).hex())
+    A, B, C0 = inputs.gemm_f16_inputs(3, 4, 5, seed=2, kind="uniform", lda=8, ldb=8, ldc=4)
+    for row in oracle.gemm_f16(A, B, 3, 4, 5, C_in=C0):
+        out.append("gemm_f16 3x4x5 accumulate " + " ".join(float(v).hex() for v in row))
     return out
 
 
