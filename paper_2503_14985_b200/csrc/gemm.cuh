@@ -527,6 +527,9 @@ gemm_bf16_pair_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_c
 __global__ void gemm_splitk_reduce_kernel(const float* partial, __nv_bfloat16* C, int64_t ldc, int M, int N, int split_k) {
     const int64_t groups_per_row = (N + 7) / 8;
     const int64_t total = static_cast<int64_t>(M) * groups_per_row;
+    // Launched with programmatic stream serialisation: the CTAs may start while the GEMM kernel is still running
+    // (which hides this kernel's launch latency) and wait here until all of its partial tiles are visible.
+    cudaGridDependencySynchronize();
     for (int64_t i = blockIdx.x * static_cast<int64_t>(blockDim.x) + threadIdx.x; i < total;
          i += static_cast<int64_t>(gridDim.x) * blockDim.x) {
         const int row = static_cast<int>(i / groups_per_row);

@@ -348,7 +348,18 @@ static int gemm_run(const void* A, const void* B, void* C, int64_t M, int64_t N,
             if (cudaGetLastError() != cudaSuccess) return MLT_ERR_CUDA;
             const int64_t groups = M * ((N + 7) / 8);
             const int blocks = static_cast<int>(std::min<int64_t>((groups + 255) / 256, 8 * dev.sm_count));
-            gemm_splitk_reduce_kernel<<<blocks, 256, 0, st>>>(p.partial, p.C, ldc, p.M, p.N, p.split_k);
+            cudaLaunchConfig_t cfg = {};
+            cfg.gridDim = dim3(blocks);
+            cfg.blockDim = dim3(256);
+            cfg.stream = st;
+            cudaLaunchAttribute attr;
+            attr.id = cudaLaunchAttributeProgrammaticStreamSerialization;
+            attr.val.programmaticStreamSerializationAllowed = 1;
+            cfg.attrs = &attr;
+            cfg.numAttrs = 1;
+            if (cudaLaunchKernelEx(&cfg, gemm_splitk_reduce_kernel, static_cast<const float*>(p.partial), p.C, ldc, p.M, p.N,
+                                   p.split_k) != cudaSuccess)
+                return MLT_ERR_CUDA;
         }
     }
     return cudaGetLastError() == cudaSuccess ? MLT_OK : MLT_ERR_CUDA;

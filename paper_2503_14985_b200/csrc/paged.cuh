@@ -307,6 +307,9 @@ paged_combine_kernel(const PagedParams p) {
     const int d = threadIdx.x;
     const int nblk = (p.seq_lens[row / p.H] + p.block_size - 1) / p.block_size;
     const int used = max(1, min(p.splits, (nblk + p.blocks_per_split - 1) / p.blocks_per_split));  // splits that wrote
+    // Launched with programmatic stream serialisation: the CTAs may start while the decode kernel is still
+    // running (which hides this kernel's launch latency) and wait here until all of its writes are visible.
+    cudaGridDependencySynchronize();
     if (d < 32) {
         const float2 ml = d < used ? p.part_ml[row * p.splits + d] : make_float2(-INFINITY, 0.0f);
         float mt = ml.x;
@@ -368,8 +371,16 @@ int paged_launch_bs(const PagedParams& p, cudaStream_t st) {
     }
     if (cudaGetLastError() != cudaSuccess) return 4;
     if (p.splits > 1) {
-        paged_combine_kernel<D><<<p.num_seqs * p.H, D, 0, st>>>(p);
-        if (cudaGetLastError() != cudaSuccess) return 4;
+        cudaLaunchConfig_t cfg = {};
+        cfg.gridDim = dim3(p.num_seqs * p.H);
+        cfg.blockDim = dim3(D);
+        cfg.stream = st;
+        cudaLaunchAttribute attr;
+        attr.id = cudaLaunchAttributeProgrammaticStreamSerialization;
+        attr.val.programmaticStreamSerializationAllowed = 1;
+        cfg.attrs = &attr;
+        cfg.numAttrs = 1;
+        if (cudaLaunchKernelEx(&cfg, paged_combine_kernel<D>, p) != cudaSuccess) return 4;
     }
     return 0;
 }
