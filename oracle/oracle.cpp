@@ -21,7 +21,14 @@
 // product of two BF16 values is exact in double, so the only rounding is in the
 // FP64 summations.  Outputs stay in FP64 (never rounded to BF16).
 //
-// Paged-attention decode (Sec. 3.2 / 4.3) is the same definition over keys gathered through a block table.
+// Paged-attention decode (Sec. 3.2 / 4.3) is the same definition over keys gathered through a block table.  The
+// paper's Listings 6 and 7 are schematic (they normalise per block and state no shapes or layouts): that the
+// operation is plain softmax attention of one query token, and the cache layout, are readings -- parity unpinned
+// by the paper for them; the function is pinned to the attention oracle above on the gathered tokens.
+//
+// FP16-operand GEMM with optional prior C (Listing 2 data types; C += A*B of the Sec. 2 problem statement): the
+// same sum over binary16 values (conversion written out field by field, checked against all 65536 patterns), the
+// prior C added after the sum.
 //
 // Pins (see tests/test_oracle_*.py): identity / permutation / all-ones /
 // single-non-zero / K-split additivity / exact rational brute force for GEMM;
