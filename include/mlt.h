@@ -180,6 +180,15 @@ int mlt_paged_attn_decode_static(const void* Q, const void* K_cache, const void*
  */
 int mlt_last_device_error(uint32_t* detail);
 
+/*
+ * Self-test of the bounded device-side waits (library addition; the paper has no counterpart).  Launches one warp
+ * that waits, with a budget of `budget_cycles` SM clocks (1 .. 1e9, i.e. at most about half a second), on a barrier
+ * that nothing completes.  The wait gives up, the kernel returns normally, and the next mlt_last_device_error
+ * reports MLT_ERR_TIMEOUT with detail = {code, barrier id 0x7E57, block 0, parity 0}.  Nothing traps; the context
+ * stays usable.  Returns MLT_OK when the launch was made, MLT_ERR_INVALID_ARG for a budget outside the range.
+ */
+int mlt_debug_wait_timeout_selftest(uint64_t budget_cycles, void* stream);
+
 /* Text for an mlt_status value (static storage). */
 const char* mlt_status_string(int status);
 

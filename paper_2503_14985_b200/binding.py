@@ -20,7 +20,7 @@ PAGED_STATIC_SCRATCH_BYTES = 16 * 1024 * 1024
 
 EXPORTS = ("mlt_gemm", "mlt_gemm_f16", "mlt_gemm_ex", "mlt_gemm_workspace_bytes", "mlt_mha_fwd", "mlt_paged_attn_decode", "mlt_paged_attn_decode_static",
            "mlt_paged_attn_workspace_bytes",
-           "mlt_last_device_error", "mlt_status_string", "mlt_version")
+           "mlt_last_device_error", "mlt_debug_wait_timeout_selftest", "mlt_status_string", "mlt_version")
 
 _lib = None
 
@@ -41,6 +41,8 @@ def load() -> ctypes.CDLL:
         i64, p, i32 = ctypes.c_int64, ctypes.c_void_p, ctypes.c_int
         lib.mlt_gemm.argtypes = [p, p, p, i64, i64, i64, i64, i64, i64, p]
         lib.mlt_gemm.restype = i32
+        lib.mlt_debug_wait_timeout_selftest.argtypes = [ctypes.c_uint64, p]
+        lib.mlt_debug_wait_timeout_selftest.restype = i32
         lib.mlt_gemm_f16.argtypes = [p, p, p, i64, i64, i64, i64, i64, i64, i32, p]
         lib.mlt_gemm_f16.restype = i32
         lib.mlt_gemm_ex.argtypes = [p, p, p, i64, i64, i64, i64, i64, i64, p, ctypes.c_size_t, p]
@@ -77,6 +79,11 @@ def version() -> int:
 def gemm_raw(A: int, B: int, C: int, M: int, N: int, K: int, lda: int, ldb: int, ldc: int, stream: int = 0) -> int:
     """mlt_gemm with raw device addresses; returns the status code."""
     return int(load().mlt_gemm(A, B, C, M, N, K, lda, ldb, ldc, stream))
+
+
+def debug_wait_timeout_selftest(budget_cycles: int, stream: int = 0) -> int:
+    """Launches the bounded-wait self-test (a wait that runs out after `budget_cycles` SM clocks); returns the status."""
+    return int(load().mlt_debug_wait_timeout_selftest(budget_cycles, stream))
 
 
 def gemm_f16_raw(A: int, B: int, C: int, M: int, N: int, K: int, lda: int, ldb: int, ldc: int, accumulate: int,

@@ -135,6 +135,21 @@ const DebugEnv& debug_env() {
     return env;
 }
 
+// Self-test of the bounded wait: one warp waits on a barrier that nothing will ever complete, with a short budget.
+// The wait gives up, records {timeout, barrier id 0x7E57, block, parity} in the status word and the kernel returns
+// like any other; nothing traps and the context stays usable.
+__global__ void debug_wait_timeout_kernel(long long budget) {
+    __shared__ uint64_t bar;
+    __shared__ uint32_t abort_word;
+    if (threadIdx.x == 0) {
+        mbar_init(&bar, 1);
+        abort_word = 0;
+        fence_mbar_init();
+    }
+    __syncthreads();
+    mbar_wait(&bar, 0, &abort_word, 0x7E57u, budget);
+}
+
 inline bool aligned16(const void* p) { return (reinterpret_cast<uintptr_t>(p) & 15u) == 0; }
 
 }  // namespace
@@ -156,6 +171,15 @@ const char* mlt_status_string(int status) {
         case MLT_ERR_SCRATCH_LIMIT: return "the call needs more scratch than the built-in array of mlt_paged_attn_decode_static holds";
         default: return "unknown status";
     }
+}
+
+int mlt_debug_wait_timeout_selftest(uint64_t budget_cycles, void* stream) {
+    if (budget_cycles == 0 || budget_cycles > 1000000000ull) return MLT_ERR_INVALID_ARG;  // at most about half a second
+    DeviceInfo dev;
+    const int rc = get_device(&dev);
+    if (rc != MLT_OK) return rc;
+    debug_wait_timeout_kernel<<<1, 32, 0, static_cast<cudaStream_t>(stream)>>>(static_cast<long long>(budget_cycles));
+    return cudaGetLastError() == cudaSuccess ? MLT_OK : MLT_ERR_CUDA;
 }
 
 int mlt_last_device_error(uint32_t* detail) {

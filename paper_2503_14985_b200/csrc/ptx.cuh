@@ -67,13 +67,13 @@ __device__ __forceinline__ bool mbar_try_wait(uint64_t* bar, uint32_t parity) {
 // Bounded wait for the phase with the given parity to complete.  `abort_flag`
 // is a CTA-shared word: non-zero means some role already gave up.
 __device__ __forceinline__ bool mbar_wait_slow(uint64_t* bar, uint32_t parity, volatile uint32_t* abort_flag,
-                                            uint32_t bar_id) {
+                                            uint32_t bar_id, long long budget = kWaitBudgetCycles) {
     const long long t0 = clock64();
     for (;;) {
         for (int i = 0; i < 256; ++i)
             if (mbar_try_wait(bar, parity)) return true;
         if (*abort_flag) return false;
-        if (clock64() - t0 > kWaitBudgetCycles) {
+        if (clock64() - t0 > budget) {
             *abort_flag = 1;
             if (atomicCAS(&g_status[0], 0u, kStatusTimeout) == 0u) {
                 g_status[1] = bar_id;
@@ -85,10 +85,10 @@ __device__ __forceinline__ bool mbar_wait_slow(uint64_t* bar, uint32_t parity, v
     }
 }
 __device__ __forceinline__ bool mbar_wait(uint64_t* bar, uint32_t parity, volatile uint32_t* abort_flag,
-                                          uint32_t bar_id) {
+                                          uint32_t bar_id, long long budget = kWaitBudgetCycles) {
     if (mbar_try_wait(bar, parity)) return true;
     if (mbar_try_wait(bar, parity)) return true;
-    return mbar_wait_slow(bar, parity, abort_flag, bar_id);
+    return mbar_wait_slow(bar, parity, abort_flag, bar_id, budget);
 }
 
 // ---------------------------------------------------------------------------
