@@ -2,6 +2,7 @@
 from __future__ import annotations
 
 import os
+import re
 import subprocess
 
 _HERE = os.path.dirname(os.path.abspath(__file__))
@@ -21,6 +22,30 @@ def is_stale() -> bool:
     return any(os.path.getmtime(os.path.join(CSRC, f)) > t for f in SOURCES + HEADERS)
 
 
+# The attention kernel moves registers between its warpgroups (setmaxnreg): 8 softmax warps at 232 and 4 other
+# warps at 40 must fit the launch allocation of 384 threads, i.e. ptxas has to assign at least this many per thread.
+MHA_MIN_REGISTERS = 168
+
+
+def check_mha_registers(ptxas_log: str) -> dict:
+    """Register counts of the mha_fwd_kernel instantiations in a `-Xptxas -v` log; raises if one is below the budget
+    the in-kernel register hand-over needs (launching such a build would wait for registers that never come)."""
+    found = {}
+    name = None
+    for line in ptxas_log.splitlines():
+        m = re.search(r"Compiling entry function '(\w+)'", line)
+        if m:
+            name = m.group(1)
+        m = re.search(r"Used (\d+) registers", line)
+        if m and name and "mha_fwd_kernel" in name:
+            found[name] = int(m.group(1))
+            name = None
+    low = {k: v for k, v in found.items() if v < MHA_MIN_REGISTERS}
+    if low:
+        raise RuntimeError(f"attention kernel compiled with fewer than {MHA_MIN_REGISTERS} registers per thread: {low}")
+    return found
+
+
 def build(force: bool = False, verbose: bool = False) -> str:
     """Compile the CUDA sources into libmlt.so next to this file; returns its path."""
     if force or is_stale():
@@ -30,6 +55,8 @@ def build(force: bool = False, verbose: bool = False) -> str:
         res = subprocess.run(cmd, capture_output=True, text=True)
         if res.returncode != 0:
             raise RuntimeError("nvcc failed:\n" + res.stdout + res.stderr)
+        if not check_mha_registers(res.stdout + res.stderr):
+            raise RuntimeError("no mha_fwd_kernel entry in the ptxas log")
         os.replace(tmp, LIB)
         if verbose:
             print(res.stdout + res.stderr)

@@ -89,10 +89,12 @@ __device__ __forceinline__ void mha_item(const MhaParams& p, int block, int& pai
 
 // 2^x for a pair of values on the FMA pipe (no MUFU): round-to-nearest split x = r + f, |f| <= 0.5, cubic for
 // 2^f (relative error < 8e-5, far below the BF16 rounding of P), then r is added to the exponent field.
-// x is clamped at -126 (2^x ~ 1e-38 stands for 0).
+// x is clamped to [-126, 127]: 2^-126 ~ 1e-38 stands for 0, and without the upper end the exponent add below
+// would carry into the sign bit (finite garbage that no overflow check sees); 2^127 is above the 2^64 limit, so
+// a score that far above the reference max still forces the true-max repeat pass.
 __device__ __forceinline__ float2 exp2_poly2(float2 x) {
-    x.x = fmaxf(x.x, -126.0f);
-    x.y = fmaxf(x.y, -126.0f);
+    x.x = fminf(fmaxf(x.x, -126.0f), 127.0f);
+    x.y = fminf(fmaxf(x.y, -126.0f), 127.0f);
     const float kMagic = 12582912.0f;  // 1.5 * 2^23: adding it leaves round(x) in the low mantissa bits
     const float2 t = fadd2(x, make_float2(kMagic, kMagic));
     const float2 r = fadd2(t, make_float2(-kMagic, -kMagic));
@@ -558,7 +560,10 @@ mha_fwd_kernel(const __grid_constant__ CUtensorMap tmap_q, const __grid_constant
                 const bool moved = !(blk < kRescaleLimit);  // also catches inf and NaN
                 if (__any_sync(0xffffffffu, moved)) {
                     // rare: rescale O_t and l by 2^((m_old - m_new)*c) (1 for rows whose reference stays) and redo P.
-                    // S_t(j) complete implies every earlier UMMA, so P_t(j-1) V has landed in O_t.
+                    // O_t may be rewritten in place because P_t(j-1) V has landed in it.  D = 128: S_t(j) complete
+                    // implies every UMMA issued before Q_t K_j^T, P_t(j-1) V among them.  D = 64: Q_t K_j^T is
+                    // issued BEFORE P_t(j-1) V, so s_full says nothing; the guarantee is the p_free[t] wait inside
+                    // the first exp_pass (w == 1), which every path to this point has passed.
                     float alpha = 1.0f;
                     if (moved) {
                         const float mxr = fmaxf(row_max(), m_run);
@@ -643,6 +648,12 @@ mha_fwd_kernel(const __grid_constant__ CUtensorMap tmap_q, const __grid_constant
     }
 }
 
+// Registers per thread the launch allocation must hold for the hand-over inside the kernel (8 softmax warps at
+// 232, 4 other warps at 40): with fewer, setmaxnreg.inc would wait for registers that never come.
+constexpr int kMhaMinRegsPerThread = (8 * 32 * 232 + 4 * 32 * 40 + kMhaThreads - 1) / kMhaThreads;
+
+// Returns 0, 1 (a CUDA call failed) or 2 (the compiled kernel's register count is below the hand-over budget, e.g.
+// after a compiler or flag change: nothing may be launched).
 inline int mha_configure() {
     if (cudaFuncSetAttribute(mha_fwd_kernel<64>, cudaFuncAttributeMaxDynamicSharedMemorySize, MhaSmem<64>::kTotal) !=
         cudaSuccess)
@@ -650,6 +661,11 @@ inline int mha_configure() {
     if (cudaFuncSetAttribute(mha_fwd_kernel<128>, cudaFuncAttributeMaxDynamicSharedMemorySize, MhaSmem<128>::kTotal) !=
         cudaSuccess)
         return 1;
+    cudaFuncAttributes a64, a128;
+    if (cudaFuncGetAttributes(&a64, mha_fwd_kernel<64>) != cudaSuccess ||
+        cudaFuncGetAttributes(&a128, mha_fwd_kernel<128>) != cudaSuccess)
+        return 1;
+    if (a64.numRegs < kMhaMinRegsPerThread || a128.numRegs < kMhaMinRegsPerThread) return 2;
     return 0;
 }
 

@@ -27,6 +27,7 @@ struct DeviceInfo {
     int sm_count = 0;
     int cc_major = 0;
     bool configured = false;
+    bool mha_ok = false;  // the attention kernels' compiled register count covers their in-kernel register hand-over
 };
 
 std::mutex g_mutex;
@@ -71,7 +72,9 @@ int get_device(DeviceInfo* out) {
             set_smem(gemm_bf16_kernel<128, 6, true>, GemmSmem<128, 6>::kTotal) != MLT_OK ||
             set_smem(gemm_bf16_pair_kernel<6, true>, GemmPairSmem<6>::kTotal) != MLT_OK)
             return MLT_ERR_CUDA;
-        if (mha_configure() != MLT_OK) return MLT_ERR_CUDA;
+        const int mha_rc = mha_configure();
+        if (mha_rc == 1) return MLT_ERR_CUDA;
+        d.mha_ok = mha_rc == 0;
         d.configured = true;
     }
     *out = d;
@@ -420,6 +423,7 @@ int mlt_mha_fwd(const void* Q, const void* K, const void* V, void* O, float* LSE
     DeviceInfo dev;
     int rc = get_device(&dev);
     if (rc != MLT_OK) return rc;
+    if (!dev.mha_ok) return MLT_ERR_UNSUPPORTED;  // this build of the kernel must not be launched (see mha_configure)
 
     CUtensorMap tq, tk, tv, to;
     const uint64_t bh = static_cast<uint64_t>(B) * H;

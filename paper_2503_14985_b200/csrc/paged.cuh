@@ -129,7 +129,8 @@ paged_decode_kernel(const PagedParams p) {
     const int head0 = kvh * (G * p.head_groups) + (blockIdx.y % p.head_groups) * G;  // first query head of this CTA
     const int sub = lane % LPT;   // which 8 columns of D this lane owns
     const int grp = lane / LPT;   // which token of a step
-    const int len = p.seq_lens[s];
+    // a length beyond what the block table can reach is cut at the table's end: no entry past the row is read
+    const int len = max(0, min(p.seq_lens[s], p.max_blocks * BS));
     const int nblk = (len + BS - 1) / BS;
     const int b0 = sp * p.blocks_per_split;
     const int b1 = min(nblk, b0 + p.blocks_per_split);
@@ -305,7 +306,8 @@ paged_combine_kernel(const PagedParams p) {
     __shared__ float sm_stat[2];             // common max, total l
     const int64_t row = blockIdx.x;
     const int d = threadIdx.x;
-    const int nblk = (p.seq_lens[row / p.H] + p.block_size - 1) / p.block_size;
+    const int len = max(0, min(p.seq_lens[row / p.H], p.max_blocks * p.block_size));  // as in the decode kernel
+    const int nblk = (len + p.block_size - 1) / p.block_size;
     const int used = max(1, min(p.splits, (nblk + p.blocks_per_split - 1) / p.blocks_per_split));  // splits that wrote
     // Launched with programmatic stream serialisation: the CTAs may start while the decode kernel is still
     // running (which hides this kernel's launch latency) and wait here until all of its writes are visible.

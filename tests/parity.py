@@ -42,3 +42,47 @@ def check_mha(o, lse, o_ref, lse_ref, what="", unit=1.0):
     assert np.isfinite(np.asarray(lse)).all()
     assert dl <= LSE_TOL, f"{what}: LSE max_abs {dl:.3e}"
     return rel, mx, dl
+
+
+def log_line(text: str) -> None:
+    """Appends one line to the parity log of this run (full-output comparisons are recorded there): the file named
+    by MLT_PARITY_LOG, else gpurun_out/parity_full_configs.log under the repository root.  Never fails a test."""
+    import os
+    path = os.environ.get("MLT_PARITY_LOG")
+    if not path:
+        root = os.path.dirname(os.path.dirname(os.path.abspath(__file__)))
+        path = os.path.join(root, "gpurun_out", "parity_full_configs.log")
+    try:
+        os.makedirs(os.path.dirname(path), exist_ok=True)
+        with open(path, "a") as f:
+            f.write(text.rstrip("\n") + "\n")
+    except OSError:
+        pass
+
+
+class RunningErrors:
+    """rel_fro / max_abs accumulated over chunks of rows, for outputs too large to hold twice in float64."""
+
+    def __init__(self):
+        self.d2 = self.r2 = 0.0
+        self.max_abs = 0.0
+        self.n = 0
+
+    def add(self, x, ref):
+        import numpy as np
+        x = np.asarray(x, dtype=np.float64)
+        ref = np.asarray(ref, dtype=np.float64)
+        assert x.shape == ref.shape, (x.shape, ref.shape)
+        assert np.isfinite(x).all(), "non-finite output"
+        diff = x - ref
+        self.d2 += float(np.sum(diff * diff))
+        self.r2 += float(np.sum(ref * ref))
+        if diff.size:
+            self.max_abs = max(self.max_abs, float(np.abs(diff).max()))
+        self.n += diff.size
+
+    def rel_fro(self):
+        return (self.d2 / self.r2) ** 0.5 if self.r2 > 0 else self.d2 ** 0.5
+
+    def rms_ref(self):
+        return (self.r2 / self.n) ** 0.5 if self.n else 1.0

@@ -62,3 +62,18 @@ def test_product_does_not_import_oracle():
             if f.endswith((".py", ".cu", ".cuh", ".h")):
                 text = open(os.path.join(dirpath, f)).read()
                 assert "import oracle" not in text and "from oracle" not in text and "oracle/" not in text, f
+
+
+def test_build_refuses_an_attention_kernel_below_its_register_budget():
+    # The attention kernel hands registers from its idle warps to its softmax warps; a build whose launch allocation
+    # is smaller than that hand-over needs must never be launched (the increase would wait for ever), so the build
+    # step reads the compiler's report and fails.  Checked here on report texts, no GPU involved.
+    from paper_2503_14985_b200 import build
+    ok = ("ptxas info    : Compiling entry function '_ZN3mlt14mha_fwd_kernelILi128EEEv' for 'sm_100a'\n"
+          "ptxas info    : Used 168 registers, used 1 barriers\n"
+          "ptxas info    : Compiling entry function '_ZN3mlt9other_fooEv' for 'sm_100a'\n"
+          "ptxas info    : Used 32 registers, used 0 barriers\n")
+    assert build.check_mha_registers(ok) == {"_ZN3mlt14mha_fwd_kernelILi128EEEv": 168}
+    with pytest.raises(RuntimeError):
+        build.check_mha_registers(ok.replace("Used 168", "Used 160"))
+    assert build.check_mha_registers("nothing here") == {}

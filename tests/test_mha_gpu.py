@@ -13,7 +13,7 @@ import paper_2503_14985_b200 as mlt  # noqa: E402
 from paper_2503_14985_b200 import inputs  # noqa: E402
 
 from gpu_util import assert_device_healthy, to_bits, to_dev, to_f64  # noqa: E402
-from parity import check_mha  # noqa: E402
+from parity import LSE_TOL, MAX_ABS_TOL, REL_FRO_TOL, RunningErrors, check_mha, log_line  # noqa: E402
 
 SENTINEL = 0x7FC1
 
@@ -109,21 +109,48 @@ def test_key_permutation_invariance_across_blocks():
     np.testing.assert_allclose(l1, l2, atol=1e-4)
 
 
-def test_dominant_key_and_outlier_rows():
-    # rows scaled x8 make the running max jump by far more than the lazy-rescale threshold
-    B, H, N, D = 1, 2, 640, 128
+@pytest.mark.parametrize("D", [128, 64])
+def test_dominant_key_and_outlier_rows(D):
+    # rows scaled x8 make the row max jump far above the reference max of the row's first block: the kernel has to
+    # notice (a block sum at or above 2^64), take the true max, rescale O and l and repeat the pass
+    B, H, N = 1, 2, 640
+    sc = scale_for(D)
     Q, K, V = inputs.mha_inputs(B, H, N, N, D, seed=264, outlier_percent=5)
     for causal in (0, 1):
+        o, lse = run_mha(Q, K, V, causal, sc)
+        o_ref, lse_ref = oracle.mha_fwd(Q, K, V, causal=bool(causal), scale=sc)
+        check_mha(o, lse, o_ref, lse_ref, f"outliers D={D} causal={causal}")
+    # One key of the last block dominates query row 5 by `gap` nats: every earlier block's contribution must be
+    # rescaled away.  2^64 = e^44.4, so a gap of 60 nats is sure to take the rescale branch; 120 nats (173 in
+    # base 2) is beyond the range a single-precision 2^x can hold.  Key positions 626 and 635 are 2 and 11 modulo
+    # 16: at D = 64 those exponentials are evaluated by the polynomial on the FMA pipe, 639 by the MUFU path.
+    q = inputs.bf16_bits_to_f64(Q); k0 = inputs.bf16_bits_to_f64(K)
+    for pos in (N - 1, 626, 635):
+        for gap in (60.0, 120.0):
+            k = k0.copy()
+            k[0, 0, pos] = (gap / float(sc)) * q[0, 0, 5] / np.dot(q[0, 0, 5], q[0, 0, 5])
+            K2 = inputs.f64_to_bf16_bits(k)
+            # the jump as the kernel sees it: the dominant score against the best score of the row's first block
+            s_row = float(sc) * inputs.bf16_bits_to_f64(K2)[0, 0] @ q[0, 0, 5]
+            assert s_row[pos] - s_row[:128].max() > 45.0, "the test input does not force the rescale branch"
+            o, lse = run_mha(Q, K2, V, 0, sc)
+            o_ref, lse_ref = oracle.mha_fwd(Q, K2, V, causal=False, scale=sc)
+            check_mha(o, lse, o_ref, lse_ref, f"dominant key at {pos}, gap {gap}, D={D}")
+
+
+def test_all_three_tensors_with_outlier_rows():
+    # The long-sequence recipe with the x8 rows in V as well (the other reading of "1 % of rows scaled x8"): outputs
+    # are no longer unit scale, so the max-abs bound is applied relative to s = max(1, max|O_ref|).  Reported
+    # separately from the benchmark configurations.
+    for (B, H, N, D, causal) in [(1, 4, 2048, 128, 1), (1, 4, 2048, 128, 0), (1, 4, 1024, 64, 1)]:
+        Q, K, V = inputs.mha_inputs(B, H, N, N, D, seed=266, outlier_percent=1, outlier_v=True)
+        assert inputs.outlier_rows(266, inputs.TENSOR_V, B * H * N, 1).any()
         o, lse = run_mha(Q, K, V, causal, scale_for(D))
         o_ref, lse_ref = oracle.mha_fwd(Q, K, V, causal=bool(causal), scale=scale_for(D))
-        check_mha(o, lse, o_ref, lse_ref, f"outliers causal={causal}")
-    # the largest key comes last: every earlier block's contribution must be rescaled away
-    q = inputs.bf16_bits_to_f64(Q); k = inputs.bf16_bits_to_f64(K)
-    k[0, 0, N - 1] = 40.0 * q[0, 0, 5] / np.linalg.norm(q[0, 0, 5])
-    K2 = inputs.f64_to_bf16_bits(k)
-    o, lse = run_mha(Q, K2, V, 0, scale_for(D))
-    o_ref, lse_ref = oracle.mha_fwd(Q, K2, V, causal=False, scale=scale_for(D))
-    check_mha(o, lse, o_ref, lse_ref, "dominant last key")
+        unit = max(1.0, float(np.abs(o_ref).max()))
+        rel, mx, dl = check_mha(o, lse, o_ref, lse_ref, f"Q/K/V outliers {(B, H, N, D, causal)}", unit=unit)
+        log_line(f"Q/K/V-all-scaled variant B{B} H{H} N{N} D{D} causal={causal}: every element, rel_fro={rel:.3e} "
+                 f"max_abs/s={mx:.3e} (s = max(1, max|O_ref|) = {unit:.2f}) lse={dl:.3e}")
 
 
 @pytest.mark.parametrize("B,H,N,D,causal", [(1, 4, 512, 128, True), (3, 70, 300, 64, True), (2, 90, 600, 128, False)])
@@ -137,30 +164,96 @@ def test_deterministic_across_runs(B, H, N, D, causal):
         assert torch.equal(runs[0][0].view(torch.int16), o.view(torch.int16)) and torch.equal(runs[0][1], l)
 
 
+def _compare_by_heads(O, LSE, Q, K, V, causal, sc, heads_per_chunk=4, rows_of_head=None):
+    """Every query row (or rows_of_head, the same row indices in every head) of O and LSE against the oracle, a few
+    heads at a time; returns (rel_fro, max_abs, max LSE error, rows compared)."""
+    Bn, H, Nq, D = Q.shape
+    acc = RunningErrors()
+    dl = 0.0
+    nrows = 0
+    O2 = O.reshape(Bn * H, Nq, D)
+    L2 = LSE.reshape(Bn * H, Nq)
+    for h0 in range(0, Bn * H, heads_per_chunk):
+        h1 = min(Bn * H, h0 + heads_per_chunk)
+        if rows_of_head is None:
+            rows = np.arange(h0 * Nq, h1 * Nq, dtype=np.int64)
+            got_o, got_l = to_f64(O2[h0:h1]).reshape(-1, D), L2[h0:h1].reshape(-1).cpu().numpy().astype(np.float64)
+        else:
+            rows = (np.arange(h0, h1, dtype=np.int64)[:, None] * Nq + rows_of_head[None, :]).reshape(-1)
+            idx = torch.from_numpy(rows_of_head).cuda()
+            got_o = to_f64(O2[h0:h1][:, idx]).reshape(-1, D)
+            got_l = L2[h0:h1][:, idx].reshape(-1).cpu().numpy().astype(np.float64)
+        o_ref, l_ref = oracle.mha_fwd(Q, K, V, causal=bool(causal), scale=sc, qrows=rows)
+        acc.add(got_o, o_ref)
+        assert np.isfinite(got_l).all()
+        dl = max(dl, float(np.abs(got_l - l_ref).max()))
+        nrows += len(rows)
+    return acc.rel_fro(), acc.max_abs, dl, nrows
+
+
 @pytest.mark.parametrize("name", list(inputs.MHA_CONFIGS))
-def test_benchmark_configs(name):
+def test_benchmark_configs_every_element(name):
+    # Every element of O and LSE against the FP64 oracle, launched exactly as bench.py launches it; the figures go
+    # to the parity log.
+    import time
     B, H, Nq, Nk, D, causal, seed, outl = inputs.MHA_CONFIGS[name]
     Q, K, V = inputs.mha_inputs(B, H, Nq, Nk, D, seed=seed, outlier_percent=outl)
+    dQ, dK, dV = to_dev(Q), to_dev(K), to_dev(V)
+    O = torch.empty_like(dQ)
+    LSE = torch.empty((B, H, Nq), dtype=torch.float32, device="cuda")
+    rc = mlt.mha_fwd_raw(dQ.data_ptr(), dK.data_ptr(), dV.data_ptr(), O.data_ptr(), LSE.data_ptr(), B, H, Nq, Nk, D,
+                         causal, float(scale_for(D)), torch.cuda.current_stream().cuda_stream)
+    assert rc == 0, mlt.status_string(rc)
+    assert_device_healthy()
+    t0 = time.perf_counter()
+    rel, mx, dl, nrows = _compare_by_heads(O, LSE, Q, K, V, causal, scale_for(D))
+    secs = time.perf_counter() - t0
+    log_line(f"{name}: all {nrows} query rows x {D}, rel_fro={rel:.3e} max_abs={mx:.3e} lse={dl:.3e} "
+             f"(limits {REL_FRO_TOL:.0e} / {MAX_ABS_TOL:.0e} / {LSE_TOL:.0e}); oracle {secs:.1f} s on "
+             f"{oracle.hardware_threads()} threads")
+    assert rel <= REL_FRO_TOL and mx <= MAX_ABS_TOL and dl <= LSE_TOL, (name, rel, mx, dl)
+
+
+# Sec. 4.2's benchmark shapes: 32k tokens in all, hidden size 2048 as 32 heads of 64 or 16 heads of 128, sequence
+# length up to 32k; the shapes below are the ones no other test reaches (D = 64 beyond 1k tokens, 32k tokens).
+SWEEP_SHAPES = [(4, 32, 8192, 64), (2, 32, 16384, 64), (1, 32, 32768, 64), (1, 16, 32768, 128)]
+
+
+@pytest.mark.parametrize("causal", [0, 1])
+@pytest.mark.parametrize("B,H,N,D", SWEEP_SHAPES)
+def test_paper_sweep_shapes_sampled_rows(B, H, N, D, causal):
+    Q, K, V = inputs.mha_inputs(B, H, N, N, D, seed=300 + N // 1024 + D)
     dQ, dK, dV = to_dev(Q), to_dev(K), to_dev(V)
     O, LSE = mlt.mha_fwd(dQ, dK, dV, causal=bool(causal), scale=scale_for(D))
     assert_device_healthy()
     assert torch.isfinite(O.float()).all() and torch.isfinite(LSE).all()
-    # sampled query rows: tile edges and interior rows in every head
-    rng = np.random.default_rng(seed)
-    per_head = 12 if Nq > 2048 else 24
-    rows = []
-    for bh in range(B * H):
-        pick = set(rng.integers(0, Nq, per_head).tolist()) | {0, Nq - 1}
-        t0 = int(rng.integers(0, Nq // 128)) * 128
-        pick |= {t0, t0 + 127}
-        rows += [bh * Nq + i for i in sorted(pick)]
-    rows = np.array(rows, dtype=np.int64)
-    o_ref, lse_ref = oracle.mha_fwd(Q, K, V, causal=bool(causal), scale=scale_for(D), qrows=rows)
-    idx = torch.from_numpy(rows).cuda()
-    got_o = to_f64(O.reshape(-1, D)[idx])
-    got_l = LSE.reshape(-1)[idx].cpu().numpy().astype(np.float64)
-    rel, mx, dl = check_mha(got_o, got_l, o_ref, lse_ref, name)
-    print(f"{name}: rel_fro={rel:.3e} max_abs={mx:.3e} lse={dl:.3e}")
+    # the same rows in every head: both ends, both sides of tile and 256-row item edges, and seeded interior rows
+    rng = np.random.default_rng(N + D + causal)
+    t0 = int(rng.integers(1, N // 256 - 1)) * 256
+    rows = np.unique(np.concatenate([[0, 1, 127, 128, 255, 256, t0 - 1, t0, t0 + 127, t0 + 128, N - 257, N - 256,
+                                      N - 129, N - 128, N - 1], rng.integers(0, N, 9)])).astype(np.int64)
+    rel, mx, dl, nrows = _compare_by_heads(O, LSE, Q, K, V, causal, scale_for(D), heads_per_chunk=B * H,
+                                           rows_of_head=rows)
+    log_line(f"sweep shape B{B} H{H} N{N} D{D} causal={causal}: {nrows} sampled query rows ({len(rows)} per head), "
+             f"rel_fro={rel:.3e} max_abs={mx:.3e} lse={dl:.3e}")
+    assert rel <= REL_FRO_TOL and mx <= MAX_ABS_TOL and dl <= LSE_TOL, (rel, mx, dl)
+
+
+@pytest.mark.parametrize("B,H,Nq,Nk,D,causal", [(2, 80, 16384, 128, 64, 0), (70, 148, 129, 129, 128, 1)])
+def test_more_items_than_the_decoded_table_holds(B, H, Nq, Nk, D, causal):
+    # A persistent CTA decodes its first 64 work items into shared memory ahead of time and the later ones on the
+    # fly, in the loader, the issuer and every softmax warp: these launches give every CTA more than 64 items.
+    props = torch.cuda.get_device_properties(0)
+    items = B * H * ((Nq + 255) // 256)
+    assert items > 64 * props.multi_processor_count
+    Q, K, V = inputs.mha_inputs(B, H, Nq, Nk, D, seed=270 + D)
+    dQ, dK, dV = to_dev(Q), to_dev(K), to_dev(V)
+    O, LSE = mlt.mha_fwd(dQ, dK, dV, causal=bool(causal), scale=scale_for(D))
+    assert_device_healthy()
+    rel, mx, dl, nrows = _compare_by_heads(O, LSE, Q, K, V, causal, scale_for(D), heads_per_chunk=16)
+    log_line(f"{items} work items (B{B} H{H} Nq{Nq} Nk{Nk} D{D} causal={causal}): all {nrows} query rows, "
+             f"rel_fro={rel:.3e} max_abs={mx:.3e} lse={dl:.3e}")
+    assert rel <= REL_FRO_TOL and mx <= MAX_ABS_TOL and dl <= LSE_TOL, (rel, mx, dl)
 
 
 def test_argument_errors_do_not_launch():

@@ -1,7 +1,8 @@
 """mlt_paged_attn_decode_static: the decode entry point for callers that cannot hand over scratch memory
 (an engine whose pool owns the whole device, a plug-in without an allocator, a loop where cudaMalloc is ruled
 out).  Its scratch is an array inside the library.  Checked here against mlt_paged_attn_decode, which takes the
-caller's workspace, on two calls in a row with different sequences (the array keeps the first call's contents).
+caller's workspace, on two calls in a row with different sequences (the array keeps the first call's contents),
+against the CPU oracle, and for the claim itself: the amount of free device memory does not move across a call.
 
 This file is named to be collected last, so that a run that stops at the first failure has already run every
 other test."""
@@ -14,6 +15,7 @@ pytestmark = pytest.mark.gpu
 
 torch = pytest.importorskip("torch")
 
+import oracle  # noqa: E402
 import paper_2503_14985_b200 as mlt  # noqa: E402
 from paper_2503_14985_b200 import inputs  # noqa: E402
 
@@ -46,6 +48,22 @@ def _run_both(S, H, Hkv, D, bs, lo, hi, seed):
     rel, mx = errors(o.reshape(-1, D), o_ref.reshape(-1, D))
     assert rel <= REL_FRO_TOL and mx <= MAX_ABS_TOL, (rel, mx)
     assert float((L - L_ref).abs().max()) <= LSE_TOL
+    # ... and against the oracle, so that the two CUDA entry points cannot be wrong in the same way unnoticed
+    o_cpu, l_cpu = oracle.paged_attn_decode(Q, Kc, Vc, table, lens, scale=scale)
+    rel, mx = errors(o.reshape(-1, D), o_cpu.reshape(-1, D))
+    assert rel <= REL_FRO_TOL and mx <= MAX_ABS_TOL, (rel, mx)
+    assert float(np.abs(L.cpu().numpy().astype(np.float64) - l_cpu).max()) <= LSE_TOL
+    # The claim itself.  The first call on a device has looked the array's address up; a further call must leave
+    # the device's free memory exactly where it was (outputs exist already, nothing is created in between).
+    torch.cuda.synchronize()
+    free_before, _ = torch.cuda.mem_get_info()
+    rc = mlt.paged_attn_decode_static_raw(dQ.data_ptr(), dK.data_ptr(), dV.data_ptr(), dT.data_ptr(), dL.data_ptr(),
+                                          O.data_ptr(), L.data_ptr(), S, H, Hkv, D, bs, table.shape[1], Kc.shape[0],
+                                          scale, sp)
+    assert rc == 0, mlt.status_string(rc)
+    torch.cuda.synchronize()
+    free_after, _ = torch.cuda.mem_get_info()
+    assert free_after == free_before, "the entry point that allocates nothing changed the free device memory"
     return bool(torch.equal(O.view(torch.int16), O_ref.view(torch.int16)))
 
 
