@@ -136,9 +136,7 @@ class ClockSampler:
     def summary(self):
         return {"sm_mhz": float(np.median(self.samples)) if self.samples else None, "sm_max_mhz": self.max_mhz,
                 "reasons": sorted(self.reasons), "samples": len(self.samples),
-                "power_w_max": max(self.power) if self.power else None,
-                "note": "under tensor-core load this pool's B200s run at 1.35-1.77 GHz (in-kernel clock64 / "
-                        "globaltimer and ncu agree); NVML reports sw_power_cap only intermittently"}
+                "power_w_max": max(self.power) if self.power else None}
 
 
 def measured_peaks():
@@ -352,10 +350,10 @@ def run_mlt(args):
     value = flop_all / (ms_max * 1e-3) / 1e12
     e2e_value = e2e_flop / (e2e_max * 1e-3) / 1e12
 
-    # ---- optional: every benchmark configuration on its own (rank 0 reports) ----
+    # ---- every benchmark configuration on its own (single-GPU runs; rank 0 reports) ----
     per_config = None
-    if args.all:
-        per_config = time_all_configs(mlt, torch, dev, stream)
+    if args.all or (world == 1 and not args.no_configs):
+        per_config = time_all_configs(mlt, torch, dev, stream, device_index=local)
 
     if rank != 0:
         return 0
@@ -367,7 +365,7 @@ def run_mlt(args):
     long_run = ms_total > 1000.0
     peak = peaks["sustained"] if long_run else peaks["burst"]
     roofline = {"bound": "tensor", "kernel": "gemm_bf16_pair_kernel<6, false>", "achieved": achieved, "peak": peak, "unit": UNIT,
-                "frac": achieved / peak, "traffic": NCU_TRAFFIC_BYTES.get("gemm"),
+                "frac": achieved / peak, "traffic": ncu_traffic_bytes(),
                 "peak_source": f"{peaks['source']} cuBLAS bf16 {'sustained' if long_run else 'burst'}",
                 "frac_of_nominal_2250": achieved / NOMINAL_BF16_TFLOPS,
                 "achieved_hbm_gbs": 2.0 * (M * K + K * N + M * N) / (gemm_avg_ms * 1e-3) / 1e9}
@@ -377,7 +375,17 @@ def run_mlt(args):
               "mha_fwd": {"config": MHA_NAME, "ms": mha_avg_ms, "ms_min": float(np.min(mha_ms)),
                           "tflops": mha_flop / (mha_avg_ms * 1e-3) / 1e12,
                           "tflops_best": mha_flop / (np.min(mha_ms) * 1e-3) / 1e12,
-                          "frac_of_2250": mha_flop / (mha_avg_ms * 1e-3) / 1e12 / NOMINAL_BF16_TFLOPS}}
+                          "frac_of_2250": mha_flop / (mha_avg_ms * 1e-3) / 1e12 / NOMINAL_BF16_TFLOPS,
+                          "timed": "inside the step, right after the GEMM (the GPU is under its power cap)"}}
+    if per_config is not None:
+        # the same kernels timed alone (pause, warm-up, L2 flushed between launches): see "configs"
+        for op, name in (("gemm", GEMM_NAME), ("mha_fwd", MHA_NAME)):
+            if name in per_config:
+                c = per_config[name]
+                per_op[op]["alone"] = {"ms_min": c["ms_min"], "ms_median": c["ms_median"], "tflops_best": c["tflops_best"],
+                                       "tflops_median": c["tflops_median"],
+                                       "frac_of_2250_best": c["tflops_best"] / NOMINAL_BF16_TFLOPS,
+                                       "frac_of_2250_median": c["tflops_median"] / NOMINAL_BF16_TFLOPS}
 
     cpu_baseline = None
     if world == 1 or rank == 0:
@@ -404,13 +412,28 @@ def run_mlt(args):
     return 0
 
 
-# dram__bytes_read.sum + dram__bytes_write.sum per launch of the GEMM kernel on the benchmark shape, from the ncu
-# capture summarised in profiles/gemm_pair_8192x28672x4096.md (algorithmic bytes: 0.772e9)
-NCU_TRAFFIC_BYTES = {"gemm": 0.795e9 + 0.453e9}
+def ncu_traffic_bytes():
+    """dram__bytes_read.sum + dram__bytes_write.sum per launch of the GEMM kernel on the benchmark shape, taken from
+    the rows of the committed ncu summary of that capture (None if the summary is not there)."""
+    import re
+    path = os.path.join(ROOT, "profiles", f"gemm_pair_{GEMM_NAME.split('_', 1)[1]}.md")
+    try:
+        text = open(path).read()
+    except OSError:
+        return None
+    total = 0.0
+    for key in ("dram__bytes_read.sum", "dram__bytes_write.sum"):
+        m = re.search(r"\|\s*" + re.escape(key) + r"\s*\|\s*([0-9.]+)\s*GB", text)
+        if not m:
+            return None
+        total += float(m.group(1)) * 1e9
+    return total
 
 
-def time_all_configs(mlt, torch, dev, stream, iters: int = 20, only: str | None = None, warm: int = 3):
-    """Min / median kernel time of every benchmark configuration (CUDA events, inputs resident)."""
+def time_all_configs(mlt, torch, dev, stream, iters: int = 20, only: str | None = None, warm: int = 3,
+                     device_index: int = 0):
+    """Min / median kernel time of every benchmark configuration alone (CUDA events, seeded inputs resident, a pause
+    and warm-up launches first, L2 evicted between timed launches, NVML clocks sampled per configuration)."""
     out = {}
     sp = stream.cuda_stream
 
@@ -425,6 +448,8 @@ def time_all_configs(mlt, torch, dev, stream, iters: int = 20, only: str | None 
         for _ in range(warm):
             fn()
         times = []
+        sampler = ClockSampler(device_index, period_s=0.002)
+        sampler.__enter__()
         for _ in range(iters):
             # evict L2 between timed launches: by writing a 256 MB buffer, or (for the HBM-bound decode kernel,
             # whose reads would otherwise have to push 126 MB of dirty lines out first) by reading it
@@ -438,9 +463,12 @@ def time_all_configs(mlt, torch, dev, stream, iters: int = 20, only: str | None 
             b.record(stream)
             torch.cuda.synchronize()
             times.append(a.elapsed_time(b))
+        sampler.__exit__()
+        ck = sampler.summary()
         tmin, tmed = float(np.min(times)), float(np.median(times))
         return {"ms_min": tmin, "ms_median": tmed, "tflops_best": flop / tmin / 1e9, "tflops_median": flop / tmed / 1e9,
-                "frac_of_2250_best": flop / tmin / 1e9 / NOMINAL_BF16_TFLOPS}
+                "frac_of_2250_best": flop / tmin / 1e9 / NOMINAL_BF16_TFLOPS, "launches": iters,
+                "clocks": {"sm_mhz": ck["sm_mhz"], "samples": ck["samples"], "reasons": ck["reasons"]}}
 
     for name, (M, N, K, kind, seed) in inputs.GEMM_CONFIGS.items():
         if only is not None and name != only:
@@ -456,24 +484,31 @@ def time_all_configs(mlt, torch, dev, stream, iters: int = 20, only: str | None 
         del dA, dB, dC
     # the same shapes in the data types of Listing 2 (FP16 operands, FP32 result), plain and as C += A * B
     for base, (M, N, K, kind, seed) in inputs.GEMM_CONFIGS.items():
-        for acc in (0, 1):
-            name = base.replace("gemm_", "gemm_f16_acc_" if acc else "gemm_f16_")
-            if (only is not None and name != only) or base == "gemm_512":
+        names = {acc: base.replace("gemm_", "gemm_f16_acc_" if acc else "gemm_f16_") for acc in (0, 1)}
+        if base == "gemm_512" or (only is not None and only not in names.values()):
+            continue
+        A, B, _ = inputs.gemm_f16_inputs(M, N, K, seed=seed, kind=kind, prior_c=False)
+        dA, dB = devbits(A), devbits(B)
+        dC = torch.zeros((M, N), dtype=torch.float32, device=dev)
+        for acc, name in names.items():
+            if only is not None and name != only:
                 continue
-            A, B, _ = inputs.gemm_f16_inputs(M, N, K, seed=seed, kind=kind, prior_c=False)
-            dA, dB = devbits(A), devbits(B)
-            dC = torch.zeros((M, N), dtype=torch.float32, device=dev)
 
             def fn():
                 rc = mlt.gemm_f16_raw(dA.data_ptr(), dB.data_ptr(), dC.data_ptr(), M, N, K, K, N, N, acc, sp)
                 assert rc == 0, rc
             out[name] = timeit(fn, inputs.gemm_flops(M, N, K))
-            del dA, dB, dC
+        del dA, dB, dC
+    mha_cache = {}
     for name, (Bn, H, Nq, Nk, D, causal, seed, outl) in inputs.MHA_CONFIGS.items():
         if only is not None and name != only:
             continue
-        Q, Kk, V = inputs.mha_inputs(Bn, H, Nq, Nk, D, seed=seed, outlier_percent=outl)
-        dQ, dK, dV = devbits(Q), devbits(Kk), devbits(V)
+        key = (Bn, H, Nq, Nk, D, seed, outl)
+        if key not in mha_cache:  # the causal and non-causal long-sequence configurations share their tensors
+            mha_cache.clear()
+            Q, Kk, V = inputs.mha_inputs(Bn, H, Nq, Nk, D, seed=seed, outlier_percent=outl)
+            mha_cache[key] = (devbits(Q), devbits(Kk), devbits(V))
+        dQ, dK, dV = mha_cache[key]
         dO = torch.empty_like(dQ)
         dL = torch.empty((Bn, H, Nq), dtype=torch.float32, device=dev)
         sc = float(np.float32(1.0 / np.sqrt(D)))
@@ -483,7 +518,8 @@ def time_all_configs(mlt, torch, dev, stream, iters: int = 20, only: str | None 
                                  D, causal, sc, sp)
             assert rc == 0, rc
         out[name] = timeit(fn, inputs.mha_flops(Bn, H, Nq, Nk, D, causal))
-        del dQ, dK, dV, dO, dL
+        del dO, dL
+    mha_cache.clear()
     hbm_peak = measured_peaks()["hbm_gbs"]
     # memory-bound GEMM shapes (Sec. 4.1, next-token prediction): split-K through mlt_gemm_ex, reported in GB/s of
     # A, B and C each moved once
@@ -502,7 +538,8 @@ def time_all_configs(mlt, torch, dev, stream, iters: int = 20, only: str | None 
         r = timeit(fn, inputs.gemm_flops(M, N, K), read_flush=True)
         out[name] = {"ms_min": r["ms_min"], "ms_median": r["ms_median"], "gbs_best": nbytes / r["ms_min"] / 1e6,
                      "gbs_median": nbytes / r["ms_median"] / 1e6, "tflops_best": r["tflops_best"],
-                     "frac_of_measured_hbm_best": nbytes / r["ms_min"] / 1e6 / hbm_peak}
+                     "frac_of_measured_hbm_best": nbytes / r["ms_min"] / 1e6 / hbm_peak, "launches": r["launches"],
+                     "clocks": r["clocks"]}
         del dA, dB, dC, ws
     # paged-attention decode (Sec. 3.2 / 4.3): bound by HBM, reported in GB/s of visible K and V
     for name, (S, H, Hkv, D, bs, lo, hi, seed) in inputs.PAGED_CONFIGS.items():
@@ -525,7 +562,8 @@ def time_all_configs(mlt, torch, dev, stream, iters: int = 20, only: str | None 
         r = timeit(fn, 4.0 * float(lens.sum()) * H * D, read_flush=True)
         out[name] = {"ms_min": r["ms_min"], "ms_median": r["ms_median"], "gbs_best": nbytes / r["ms_min"] / 1e6,
                      "gbs_median": nbytes / r["ms_median"] / 1e6, "kv_bytes": nbytes,
-                     "frac_of_measured_hbm_best": nbytes / r["ms_min"] / 1e6 / hbm_peak}
+                     "frac_of_measured_hbm_best": nbytes / r["ms_min"] / 1e6 / hbm_peak, "launches": r["launches"],
+                     "clocks": r["clocks"]}
         del dQ, dK, dV, dO, dL, ws
     return out
 
@@ -533,7 +571,7 @@ def time_all_configs(mlt, torch, dev, stream, iters: int = 20, only: str | None 
 def run_sweeps(mlt, torch, dev, stream, iters: int = 20):
     """Paper-shaped sweeps (Sec. 4.1 / 4.2): compute-bound GEMM with m = 1k..16k on Llama-like (n, k), and the
     attention forward with 32k tokens in total, sequence length 1k..32k, hidden size 2048 as 32 heads of 64 or 16
-    heads of 128.  Synthetic N(0,1) data generated on the device (timing only; parity is the test suite's job)."""
+    heads of 128.  Inputs come from the seeded generator, as in the parity tests of the same shapes."""
     sp = stream.cuda_stream
     flush = torch.empty(256 << 20, dtype=torch.int8, device=dev)
     rows = []
@@ -556,11 +594,16 @@ def run_sweeps(mlt, torch, dev, stream, iters: int = 20):
             ts.append(a.elapsed_time(b))
         return float(np.min(ts))
 
+    def devbits(bits):
+        return torch.from_numpy(np.ascontiguousarray(bits).view(np.int16)).to(dev)
+
     for (N, K) in ((4096, 4096), (14336, 4096), (4096, 14336), (8192, 8192)):
-        Bm = (torch.randn(K, N, device=dev) / np.sqrt(K)).to(torch.bfloat16)
+        scale = 1.0 / np.sqrt(K)
+        Bm = devbits(inputs.matrix_bf16(K, N, seed=40, tensor_id=inputs.TENSOR_B, scale=scale))
+        A_all = devbits(inputs.matrix_bf16(16384, K, seed=40, tensor_id=inputs.TENSOR_A, scale=scale))
         for M in (1024, 2048, 4096, 8192, 16384):
-            A = (torch.randn(M, K, device=dev) / np.sqrt(K)).to(torch.bfloat16)
-            C = torch.empty(M, N, dtype=torch.bfloat16, device=dev)
+            A = A_all[:M]  # the first M rows of the same seeded matrix
+            C = torch.empty(M, N, dtype=torch.int16, device=dev)
 
             def fn():
                 rc = mlt.gemm_raw(A.data_ptr(), Bm.data_ptr(), C.data_ptr(), M, N, K, K, N, N, sp)
@@ -568,13 +611,11 @@ def run_sweeps(mlt, torch, dev, stream, iters: int = 20):
             ms = best_ms(fn)
             rows.append({"op": "gemm", "M": M, "N": N, "K": K, "ms": ms, "tflops": 2.0 * M * N * K / ms / 1e9})
             del A, C
-        del Bm
+        del Bm, A_all
     for D, H in ((64, 32), (128, 16)):
         for N in (1024, 2048, 4096, 8192, 16384, 32768):
             Bn = 32768 // N
-            q = torch.randn(Bn, H, N, D, device=dev).to(torch.bfloat16)
-            k = torch.randn(Bn, H, N, D, device=dev).to(torch.bfloat16)
-            v = torch.randn(Bn, H, N, D, device=dev).to(torch.bfloat16)
+            q, k, v = (devbits(t) for t in inputs.mha_inputs(Bn, H, N, N, D, seed=300 + N // 1024 + D))
             o = torch.empty_like(q)
             lse = torch.empty(Bn, H, N, dtype=torch.float32, device=dev)
             for causal in (0, 1):
@@ -595,7 +636,8 @@ def main(argv=None):
     ap.add_argument("--steps", type=int, default=50)
     ap.add_argument("--warmup", type=int, default=5)
     ap.add_argument("--impl", choices=["mlt", "reference"], default="mlt")
-    ap.add_argument("--all", action="store_true", help="also time every benchmark configuration on its own")
+    ap.add_argument("--all", action="store_true", help="time every benchmark configuration on its own (the default on one GPU)")
+    ap.add_argument("--no-configs", action="store_true", help="skip the per-configuration timings (\"configs\")")
     ap.add_argument("--sweep", action="store_true", help="paper-shaped GEMM and attention sweeps (one JSON line)")
     ap.add_argument("--only", default=None, help="time one named configuration alone (kernel launches only; for profiling)")
     args = ap.parse_args(argv)

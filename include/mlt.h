@@ -123,7 +123,8 @@ int mlt_mha_fwd(const void* Q, const void* K, const void* V,
  *                logical blocks a sequence uses must lie in [0, num_blocks) (others are never read; a bad entry is
  *                skipped and reported through mlt_last_device_error, it is never dereferenced)
  *   seq_lens     device, int32, [num_seqs], 0 <= len <= max_blocks_per_seq * block_size; token i sits in logical
- *                block i / block_size at offset i % block_size
+ *                block i / block_size at offset i % block_size (a length outside that range is cut to it: no
+ *                table entry beyond a sequence's row is read)
  *   O            device, BF16 out, [num_seqs, H, D];  LSE device FP32 out [num_seqs, H] (natural log) or NULL
  *   H_kv         KV heads; H / H_kv in {1, 2, 4, 8}; query head h reads KV head h / (H / H_kv)
  *   D in {64, 128}; block_size in {8, 16, 32}; scale finite and > 0

@@ -104,6 +104,19 @@ def test_empty_and_single_token_sequences():
     check_mha(o[2:].reshape(-1, D), lse[2:].reshape(-1), o_ref[2:].reshape(-1, D), l_ref[2:].reshape(-1), "16 and 40")
 
 
+def test_length_beyond_the_table_is_cut_at_the_table_end():
+    # 75 table entries per sequence, split over CTAs of 8 blocks each (10 x 8 = 80 > 75): a stated length that the
+    # table cannot reach must not make any CTA read past the sequence's row (for the last sequence: past the table)
+    S, H, D, bs = 3, 4, 128, 16
+    Q, Kc, Vc, table, lens = inputs.paged_inputs(S, H, H, D, bs, seed=314, min_len=1200, max_len=1200)
+    assert table.shape[1] == 75 and (table >= 0).all()
+    too_long = lens.copy(); too_long[0] += 37; too_long[-1] += 500
+    scale = np.float32(1 / math.sqrt(D))
+    o, lse = run_paged(Q, Kc, Vc, table, too_long, scale)
+    o_ref, l_ref = oracle.paged_attn_decode(Q, Kc, Vc, table, lens, scale=scale)
+    check_mha(o, lse, o_ref.reshape(-1, D), l_ref.reshape(-1), "over-long lengths")
+
+
 def test_bad_block_table_entry_is_reported_not_dereferenced():
     S, H, D, bs = 1, 2, 64, 16
     Q, Kc, Vc, table, lens = inputs.paged_inputs(S, H, H, D, bs, seed=312, min_len=64, max_len=64)
