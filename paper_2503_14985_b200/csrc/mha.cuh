@@ -17,6 +17,8 @@
 //   warp  9     TMA loader (one lane): Q tiles, then K/V tiles through a ring; it also initialises the
 //               barriers and issues the first loads before the CTA-wide sync
 //   warps 10-11 idle (they complete the third warpgroup for the register hand-over)
+// One in eight of the exponentials of a D = 128 block (one in four at D = 64) is a cubic on the FMA pipe instead of
+// a MUFU operation (exp2_poly2): the MUFU pipe is the longest leg of a tile's chain S -> softmax -> P -> P V -> S.
 // Tensor memory (512 columns): S_0 | S_1 (128 FP32 columns each), O_0 | O_1 (D FP32 columns each).  D = 128:
 // the BF16 P of a tile overwrites the first 64 columns of its S and is consumed from there as the A operand of
 // P V.  D = 64: P_0 | P_1 have their own columns, and the next Q K^T of a tile is issued as soon as the softmax
@@ -46,8 +48,28 @@
 
 namespace mlt {
 
+// In-kernel clock trace (development builds only, -DMLT_TRACE): CTA 0 records the SM clock at fixed points of K/V
+// blocks 32..47 of its first work item; role 0 / 1 = first softmax warp of tile 0 / 1, role 2 = UMMA issuer.
+#ifdef MLT_TRACE
+__device__ unsigned int g_mha_trace[3][16][24];
+#define MLT_TR(role, j, ev)                                                                                  \
+    do {                                                                                                     \
+        if (blockIdx.x == 0 && r == 0 && (j) >= 32 && (j) < 48) g_mha_trace[role][(j) - 32][ev] = static_cast<unsigned int>(clock64()); \
+    } while (0)
+#else
+#define MLT_TR(role, j, ev) do { } while (0)
+#endif
+
 constexpr int kMhaBlock = 128;   // query rows per tile and keys per K/V block
 constexpr int kMhaThreads = 384; // three warpgroups
+#ifndef MLT_SOFTMAX_REGS
+#define MLT_SOFTMAX_REGS 208
+#endif
+#ifndef MLT_OTHER_REGS
+#define MLT_OTHER_REGS 88
+#endif
+constexpr int kMhaSoftmaxRegs = MLT_SOFTMAX_REGS;  // per thread of the 8 softmax warps after the hand-over
+constexpr int kMhaOtherRegs = MLT_OTHER_REGS;      // per thread of the 4 other warps
 constexpr float kLog2e = 1.4426950408889634f;
 constexpr float kRescaleLimit = 18446744073709551616.0f;  // 2^64: a block sum at or above it forces a new reference max
 
@@ -87,18 +109,27 @@ __device__ __forceinline__ void mha_item(const MhaParams& p, int block, int& pai
     bh = first + r % heads;
 }
 
-// 2^x for a pair of values on the FMA pipe (no MUFU): round-to-nearest split x = r + f, |f| <= 0.5, cubic for
-// 2^f (relative error < 8e-5, far below the BF16 rounding of P), then r is added to the exponent field.
-// x is clamped to [-126, 127]: 2^-126 ~ 1e-38 stands for 0, and without the upper end the exponent add below
-// would carry into the sign bit (finite garbage that no overflow check sees); 2^127 is above the 2^64 limit, so
-// a score that far above the reference max still forces the true-max repeat pass.
-__device__ __forceinline__ float2 exp2_poly2(float2 x) {
-    x.x = fminf(fmaxf(x.x, -126.0f), 127.0f);
-    x.y = fminf(fmaxf(x.y, -126.0f), 127.0f);
-    const float kMagic = 12582912.0f;  // 1.5 * 2^23: adding it leaves round(x) in the low mantissa bits
-    const float2 t = fadd2(x, make_float2(kMagic, kMagic));
-    const float2 r = fadd2(t, make_float2(-kMagic, -kMagic));
-    const float2 f = ffma2(r, make_float2(-1.0f, -1.0f), x);
+// 2^((s - m) * c) for a pair of scores on the FMA pipe (no MUFU).  The exponent x = (s - m) * c is clamped to
+// [-125, 127] by a saturating FMA: u = sat((x + 125) / 252) in [0, 1], so x + 125 = 252 u.  Round-to-nearest split
+// 252 u = N + f, |f| <= 0.5 (adding 1.5 * 2^23 leaves N in the low mantissa bits), a cubic for 2^f (relative error
+// below 9e-5, far below the BF16 rounding of P), and N - 125 is added to the exponent field: the constant is
+// folded into the magic number, whose low 9 mantissa bits then hold N - 125 in two's complement.
+// 2^-125 ~ 2e-38 stands for 0 (masked scores are -inf and saturate to it); the upper end keeps the exponent add
+// from carrying into the sign bit, and 2^127 is above the 2^64 limit, so a score that far above the reference max
+// still forces the true-max repeat pass.  `cs` = c / 252, `ns` = (125 - m c) / 252.
+constexpr float kPolySpan = 252.0f;
+constexpr float kPolyLow = 125.0f;
+__device__ __forceinline__ float fma_sat(float a, float b, float c) {
+    float d;
+    asm("fma.rn.sat.f32 %0, %1, %2, %3;" : "=f"(d) : "f"(a), "f"(b), "f"(c));
+    return d;
+}
+__device__ __forceinline__ float2 exp2_poly2(float s0, float s1, float cs, float ns) {
+    constexpr float kMagic = 12582912.0f - kPolyLow;  // 1.5 * 2^23 - 125
+    const float2 u = make_float2(fma_sat(s0, cs, ns), fma_sat(s1, cs, ns));
+    const float2 span = make_float2(kPolySpan, kPolySpan), magic = make_float2(kMagic, kMagic);
+    const float2 t = ffma2(u, span, magic);  // N + magic, exact integer grid
+    const float2 f = ffma2(u, span, fsub2(magic, t));
     float2 y = ffma2(f, make_float2(0.05508868396282196f, 0.05508868396282196f),
                      make_float2(0.24260404706001282f, 0.24260404706001282f));
     y = ffma2(y, f, make_float2(0.6932762265205383f, 0.6932762265205383f));
@@ -107,6 +138,14 @@ __device__ __forceinline__ float2 exp2_poly2(float2 x) {
     y.y = __int_as_float(__float_as_int(y.y) + (__float_as_int(t.y) << 23));
     return y;
 }
+
+// Which of the 8 score pairs of every 16 keys take the FMA-pipe exponential (bit i = pair i).
+#ifndef MLT_POLY_MASK_64
+#define MLT_POLY_MASK_64 0x22
+#endif
+#ifndef MLT_POLY_MASK_128
+#define MLT_POLY_MASK_128 0x10
+#endif
 
 template <int D>
 __global__ void __launch_bounds__(kMhaThreads, 1)
@@ -134,7 +173,10 @@ mha_fwd_kernel(const __grid_constant__ CUtensorMap tmap_q, const __grid_constant
     uint32_t* tmem_base_slot = reinterpret_cast<uint32_t*>(p_free + 2);
     volatile uint32_t* abort_flag = tmem_base_slot + 1;
 
-    const int warp = threadIdx.x >> 5;
+#ifndef MLT_ROLE_SHIFT
+#define MLT_ROLE_SHIFT 0
+#endif
+    const int warp = ((threadIdx.x >> 5) + MLT_ROLE_SHIFT) % 12;  // role index (see the table above)
     const int lane = threadIdx.x & 31;
 
     // Work items of this CTA: item list position r * gridDim.x + (c or gridDim.x - 1 - c), the direction alternating
@@ -272,14 +314,26 @@ mha_fwd_kernel(const __grid_constant__ CUtensorMap tmap_q, const __grid_constant
     constexpr uint32_t kStrideP = kEarlyQK ? 64 : kMhaBlock;
 
     // Register hand-over: setmaxnreg moves registers inside the CTA's launch allocation (384 threads x 168), it cannot
-    // draw on the rest of the register file.  232 for the softmax warps needs every other warp down at 40; one
-    // register more anywhere and the increase below would wait for ever.
-    static_assert(8 * 32 * 232 + 4 * 32 * 40 <= kMhaThreads * 168, "setmaxnreg budget exceeds the launch allocation");
+    // draw on the rest of the register file; if the two budgets together exceeded it, the increase below would wait
+    // for ever.  208 / 88 measured best: the softmax code does not use more (232 / 40 was 3 % slower: the issuing
+    // warp then spills).
+    static_assert(8 * 32 * kMhaSoftmaxRegs + 4 * 32 * kMhaOtherRegs <= kMhaThreads * 168, "setmaxnreg budget exceeds the launch allocation");
     if (warp >= 10) {
-        setmaxnreg_dec<40>();  // only hand their registers over
+        setmaxnreg_dec<kMhaOtherRegs>();  // only hand their registers over
+#ifdef MLT_TRACE
+        if (blockIdx.x == 0 && lane == 0) {  // spies: when do S_t(j) of the first item really complete?
+            const int t = warp - 10;
+            const int r = 0;
+            for (int j = 0; j < 48; ++j) {
+                int spins = 0;
+                while (!mbar_test_wait(&s_full[t], j & 1) && ++spins < 4000000) {}
+                MLT_TR(t, j, 8);
+            }
+        }
+#endif
     } else if (warp == 9) {
         // ------------------------------- loader -------------------------------
-        setmaxnreg_dec<40>();
+        setmaxnreg_dec<kMhaOtherRegs>();
         if (lane == 0) {
             bool ok = true;
             Item it;
@@ -302,7 +356,7 @@ mha_fwd_kernel(const __grid_constant__ CUtensorMap tmap_q, const __grid_constant
         // The whole warp runs this code (uniform control flow keeps addresses and descriptors in the uniform
         // datapath: an issue costs about 20 clocks instead of about 46 from a single divergent lane); one
         // elected lane executes the tcgen05 instructions.
-        setmaxnreg_dec<40>();
+        setmaxnreg_dec<kMhaOtherRegs>();
         {
             const bool leader = elect_one();
             constexpr uint32_t idesc_qk = make_idesc_bf16(kMhaBlock, kMhaBlock, false, false);
@@ -416,6 +470,7 @@ mha_fwd_kernel(const __grid_constant__ CUtensorMap tmap_q, const __grid_constant
 #pragma unroll 1
                 for (int j = -1; j < Jmax && ok; ++j) {
                     int vslot = 0;
+                    if (leader) MLT_TR(2, j, 0);
                     if (j >= 0) {
                         vslot = stage;
                         ok = wait_all(&kv_full[vslot], phase, 0x220 + vslot);
@@ -427,11 +482,14 @@ mha_fwd_kernel(const __grid_constant__ CUtensorMap tmap_q, const __grid_constant
                     for (int t = 0; t < 2 && ok; ++t) {
                         if (j >= 0 && j < it.J[t]) {
                             // P_t(0) of an item also tells that the softmax warps have read the previous item's O_t
+                            if (leader) MLT_TR(2, j, 1 + 4 * t);
                             ok = wait_all(&p_full[t], n_p[t] & 1, 0x230 + t);
                             if (!ok) break;
+                            if (leader) MLT_TR(2, j, 2 + 4 * t);
                             ++n_p[t];
                             tc_fence_after();
                             issue_pv(t, vslot, j == 0);
+                            if (leader) MLT_TR(2, j, 3 + 4 * t);
                             if (j == it.J[t] - 1 && leader) umma_commit(&o_full[t]);
                         }
                         if (j + 1 < it.J[t]) {
@@ -442,6 +500,7 @@ mha_fwd_kernel(const __grid_constant__ CUtensorMap tmap_q, const __grid_constant
                                 k_ready = true;
                             }
                             issue_qk(t, kslot);
+                            if (leader) MLT_TR(2, j, 4 + 4 * t);
                         }
                     }
                     if (!ok) break;
@@ -460,7 +519,7 @@ mha_fwd_kernel(const __grid_constant__ CUtensorMap tmap_q, const __grid_constant
         }
     } else {
         // ------------------- softmax, O rescale and epilogue of tile t -------------------
-        setmaxnreg_inc<232>();
+        setmaxnreg_inc<kMhaSoftmaxRegs>();
         const int t = warp >> 2;
         const int quarter = warp & 3;
         const int row_in_tile = quarter * 32 + lane;
@@ -481,14 +540,17 @@ mha_fwd_kernel(const __grid_constant__ CUtensorMap tmap_q, const __grid_constant
         float l_run = 0.0f;
 
         for (int j = 0; j < Jt; ++j) {
+            if (quarter == 0 && lane == 0) MLT_TR(t, j, 0);
             ok = __all_sync(0xffffffffu, mbar_wait(&s_full[t], n_s & 1, abort_flag, 0x300 + t));
             if (!ok) break;
+            if (quarter == 0 && lane == 0) MLT_TR(t, j, 1);
             ++n_s;
             tc_fence_after();
             uint32_t s[4][32];  // this thread's row of S: 4 chunks of 32 keys
 #pragma unroll
             for (int q = 0; q < 4; ++q) tmem_ld_32x32b_x32(s_addr + q * 32, s[q]);
             tmem_wait_ld();
+            if (quarter == 0 && lane == 0) MLT_TR(t, j, 2);
             if constexpr (kEarlyQK) {  // S_t is in registers: the next Q K^T of this tile may overwrite it
                 tc_fence_before();
                 __syncwarp();
@@ -520,25 +582,27 @@ mha_fwd_kernel(const __grid_constant__ CUtensorMap tmap_q, const __grid_constant
                 return fmaxf(fmaxf(mx[0], mx[1]), fmaxf(mx[2], mx[3]));
             };
             auto exp_pass = [&](float neg_mc) {
+                constexpr int kPolyMask = (D == 64) ? MLT_POLY_MASK_64 : MLT_POLY_MASK_128;
                 const float2 c2 = make_float2(c, c), n2 = make_float2(neg_mc, neg_mc);
+                const float cs = c * (1.0f / kPolySpan), ns = (neg_mc + kPolyLow) * (1.0f / kPolySpan);
                 acc0 = make_float2(0.0f, 0.0f);
                 acc1 = make_float2(0.0f, 0.0f);
                 uint32_t pk[16];
+                auto exp_pair = [&](int k, bool poly) {  // keys k, k + 1 of the block
+                    const float s0 = __uint_as_float(s[k >> 5][k & 31]), s1 = __uint_as_float(s[k >> 5][(k & 31) + 1]);
+                    if (poly) return exp2_poly2(s0, s1, cs, ns);
+                    float2 x = ffma2(make_float2(s0, s1), c2, n2);
+                    x.x = fast_exp2(x.x);
+                    x.y = fast_exp2(x.y);
+                    return x;
+                };
 #pragma unroll
                 for (int w = 0; w < 8; ++w) {  // waves of 16 keys
 #pragma unroll
                     for (int i = 0; i < 8; i += 2) {
                         const int k = w * 16 + 2 * i;
-                        float2 x0 = ffma2(make_float2(__uint_as_float(s[k >> 5][k & 31]), __uint_as_float(s[k >> 5][(k & 31) + 1])), c2, n2);
-                        float2 x1 = ffma2(make_float2(__uint_as_float(s[k >> 5][(k & 31) + 2]), __uint_as_float(s[k >> 5][(k & 31) + 3])), c2, n2);
-                        x0.x = fast_exp2(x0.x);
-                        x0.y = fast_exp2(x0.y);
-                        if (D == 64 && (i / 2) % 2 == 0) {  // D = 64 is MUFU-bound: a quarter of the exponentials go to the FMA pipe
-                            x1 = exp2_poly2(x1);
-                        } else {
-                            x1.x = fast_exp2(x1.x);
-                            x1.y = fast_exp2(x1.y);
-                        }
+                        const float2 x0 = exp_pair(k, (kPolyMask >> i) & 1);
+                        const float2 x1 = exp_pair(k + 2, (kPolyMask >> (i + 1)) & 1);
                         acc0 = fadd2(acc0, x0);
                         acc1 = fadd2(acc1, x1);
                         pk[(w & 1) * 8 + i] = pack_bf16x2(x0.x, x0.y);
@@ -555,6 +619,7 @@ mha_fwd_kernel(const __grid_constant__ CUtensorMap tmap_q, const __grid_constant
             // The first block of a row takes its max first and then runs the same pass as every other block.
             if (j == 0) m_run = row_max();
             exp_pass((m_run == -INFINITY) ? 0.0f : -m_run * c);
+            if (quarter == 0 && lane == 0) MLT_TR(t, j, 3);
             if (j > 0) {
                 const float blk = (acc0.x + acc0.y) + (acc1.x + acc1.y);
                 const bool moved = !(blk < kRescaleLimit);  // also catches inf and NaN
@@ -585,10 +650,13 @@ mha_fwd_kernel(const __grid_constant__ CUtensorMap tmap_q, const __grid_constant
             }
             if (!ok) break;
             l_run += (acc0.x + acc0.y) + (acc1.x + acc1.y);
+            if (quarter == 0 && lane == 0) MLT_TR(t, j, 5);
             tmem_wait_st();
+            if (quarter == 0 && lane == 0) MLT_TR(t, j, 6);
             tc_fence_before();
             __syncwarp();
             if (lane == 0) mbar_arrive(&p_full[t]);
+            if (quarter == 0 && lane == 0) MLT_TR(t, j, 4);
         }
 
         if (!ok) break;
@@ -650,7 +718,7 @@ mha_fwd_kernel(const __grid_constant__ CUtensorMap tmap_q, const __grid_constant
 
 // Registers per thread the launch allocation must hold for the hand-over inside the kernel (8 softmax warps at
 // 232, 4 other warps at 40): with fewer, setmaxnreg.inc would wait for registers that never come.
-constexpr int kMhaMinRegsPerThread = (8 * 32 * 232 + 4 * 32 * 40 + kMhaThreads - 1) / kMhaThreads;
+constexpr int kMhaMinRegsPerThread = (8 * 32 * kMhaSoftmaxRegs + 4 * 32 * kMhaOtherRegs + kMhaThreads - 1) / kMhaThreads;
 
 // Returns 0, 1 (a CUDA call failed) or 2 (the compiled kernel's register count is below the hand-over budget, e.g.
 // after a compiler or flag change: nothing may be launched).

@@ -185,6 +185,13 @@ int mlt_debug_wait_timeout_selftest(uint64_t budget_cycles, void* stream) {
     return cudaGetLastError() == cudaSuccess ? MLT_OK : MLT_ERR_CUDA;
 }
 
+#ifdef MLT_TRACE
+int mlt_debug_read_trace(unsigned int* host) {  // development builds only: copies the attention kernel's clock trace
+    if (cudaDeviceSynchronize() != cudaSuccess) return MLT_ERR_CUDA;
+    return cudaMemcpyFromSymbol(host, g_mha_trace, sizeof(g_mha_trace)) == cudaSuccess ? MLT_OK : MLT_ERR_CUDA;
+}
+#endif
+
 int mlt_last_device_error(uint32_t* detail) {
     if (cudaDeviceSynchronize() != cudaSuccess) return MLT_ERR_CUDA;
     unsigned int host[4] = {0, 0, 0, 0};
