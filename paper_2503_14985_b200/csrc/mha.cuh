@@ -11,12 +11,15 @@
 //   warps 0-3   softmax / O-rescale / epilogue of tile 0 (one thread per query row)
 //   warps 4-7   the same for tile 1
 //   warp  8     UMMA issuer (the whole warp runs the loop, one elected lane issues) and owner of the
-//               tensor-memory allocation; it serves the tiles in a fixed order, which keeps the two softmax
-//               warpgroups half a period apart (one issuer per tile was tried: the tiles fall into step and
-//               D = 128 loses 18 %)
+//               tensor-memory allocation; at D = 128 it serves both tiles in a fixed order, which keeps the two
+//               softmax warpgroups half a period apart (one issuer per tile was tried there: the tiles fall into
+//               step and D = 128 loses 18 %); at D = 64 it serves tile 0 only
 //   warp  9     TMA loader (one lane): Q tiles, then K/V tiles through a ring; it also initialises the
 //               barriers and issues the first loads before the CTA-wide sync
-//   warps 10-11 idle (they complete the third warpgroup for the register hand-over)
+//   warp  10    D = 64: UMMA issuer of tile 1 (there S_t(j+1) does not wait for P_t(j) V, so a tile's products
+//               follow its own softmax only; one warp serving both tiles in turn made each wait for the other's
+//               softmax: 724 -> 760 TFLOP/s at 16k tokens); D = 128: idle
+//   warp  11    idle (completes the third warpgroup for the register hand-over)
 // One in eight of the exponentials of a D = 128 block (one in four at D = 64) is a cubic on the FMA pipe instead of
 // a MUFU operation (exp2_poly2): the MUFU pipe is the longest leg of a tile's chain S -> softmax -> P -> P V -> S.
 // Tensor memory (512 columns): S_0 | S_1 (128 FP32 columns each), O_0 | O_1 (D FP32 columns each).  D = 128:
@@ -153,6 +156,7 @@ mha_fwd_kernel(const __grid_constant__ CUtensorMap tmap_q, const __grid_constant
                const __grid_constant__ CUtensorMap tmap_v, const __grid_constant__ CUtensorMap tmap_o,
                const MhaParams p) {
     using L = MhaSmem<D>;
+    constexpr int kIssuers = (D == 64) ? 2 : 1;  // UMMA-issuing warps (see the role table)
     constexpr int kStages = L::kStages;
     constexpr int kChunks = D / 64;
     extern __shared__ uint8_t smem_raw[];
@@ -268,10 +272,11 @@ mha_fwd_kernel(const __grid_constant__ CUtensorMap tmap_q, const __grid_constant
     int pre_tiles = 0;  // ring tiles of the first item already requested
     if (warp == 9 && lane == 0) {
         mbar_init(q_full, 1);
-        mbar_init(q_empty, 1);
+        // D = 64 has one issuing warp per query tile: each of them releases every K/V slot and the Q tiles
+        mbar_init(q_empty, kIssuers);
         for (int s = 0; s < kStages; ++s) {
             mbar_init(&kv_full[s], 1);
-            mbar_init(&kv_empty[s], 1);
+            mbar_init(&kv_empty[s], kIssuers);
         }
         for (int t = 0; t < 2; ++t) {
             mbar_init(&s_full[t], 1);
@@ -318,7 +323,7 @@ mha_fwd_kernel(const __grid_constant__ CUtensorMap tmap_q, const __grid_constant
     // for ever.  208 / 88 measured best: the softmax code does not use more (232 / 40 was 3 % slower: the issuing
     // warp then spills).
     static_assert(8 * 32 * kMhaSoftmaxRegs + 4 * 32 * kMhaOtherRegs <= kMhaThreads * 168, "setmaxnreg budget exceeds the launch allocation");
-    if (warp >= 10) {
+    if (warp == 11 || (warp == 10 && kIssuers == 1)) {
         setmaxnreg_dec<kMhaOtherRegs>();  // only hand their registers over
 #ifdef MLT_TRACE
         if (blockIdx.x == 0 && lane == 0) {  // spies: when do S_t(j) of the first item really complete?
@@ -351,8 +356,14 @@ mha_fwd_kernel(const __grid_constant__ CUtensorMap tmap_q, const __grid_constant
                 }
             }
         }
-    } else if (warp == 8) {
+    } else if (warp == 8 || warp == 10) {
         // ------------------------------- UMMA issuer -------------------------------
+        // D = 128: warp 8 serves both tiles in a fixed order (which keeps them half a period apart).  D = 64: warp 8
+        // serves tile 0 and warp 10 tile 1, each in its tile's own order (Q_t K_{j+1}^T when S_t(j) has been read,
+        // P_t(j) V_j when P_t(j) is there), so that neither tile ever waits for the other's softmax; both walk
+        // the same K/V ring and both release every slot.
+        const int t_lo = (kIssuers == 2 && warp == 10) ? 1 : 0;
+        const int t_hi = (kIssuers == 2 && warp == 8) ? 1 : 2;
         // The whole warp runs this code (uniform control flow keeps addresses and descriptors in the uniform
         // datapath: an issue costs about 20 clocks instead of about 46 from a single divergent lane); one
         // elected lane executes the tcgen05 instructions.
@@ -407,25 +418,29 @@ mha_fwd_kernel(const __grid_constant__ CUtensorMap tmap_q, const __grid_constant
                 for (int r = 0; ok && item_at(r, it); ++r) {
                     const int Jmax = it.Jmax;
                     ok = wait_all(q_full, r & 1, 0x200);
-                    // Step j: Q_t K_{j+1}^T for both tiles as soon as S_t(j) has been read, then P_t(j) V_j.
+                    // Step j: Q_t K_{j+1}^T as soon as S_t(j) has been read, then P_t(j) V_j, for this warp's tile(s).
                     // Step -1 issues the first Q K^T products only (same instructions, no cold copy).
 #pragma unroll 1
                     for (int j = -1; j < Jmax && ok; ++j) {
+                        if (leader && warp == 8) MLT_TR(2, j, 0);
                         if (j + 1 < Jmax) {
                             const int kslot = stage;
                             ok = wait_all(&kv_full[kslot], phase, 0x240 + kslot);
                             if (!ok) break;
+                            if (leader && warp == 8) MLT_TR(2, j, 1);
                             if (++stage == kStages) { stage = 0; phase ^= 1; }
                             tc_fence_after();
-                            for (int t = 0; t < 2 && ok; ++t) {
+                            for (int t = t_lo; t < t_hi && ok; ++t) {
                                 if (j + 1 >= it.J[t]) continue;
                                 if (n_qk[t] > 0) {  // S_t is free once the softmax warps hold its previous contents
                                     ok = wait_all(&s_free[t], (n_qk[t] - 1) & 1, 0x250 + t);
                                     if (!ok) break;
                                     tc_fence_after();
                                 }
+                                if (leader && warp == 8) MLT_TR(2, j, 2);
                                 ++n_qk[t];
                                 issue_qk(t, kslot);
+                                if (leader && warp == 8) MLT_TR(2, j, 3);
                             }
                             if (!ok) break;
                             if (leader) {
@@ -439,14 +454,17 @@ mha_fwd_kernel(const __grid_constant__ CUtensorMap tmap_q, const __grid_constant
                             ok = wait_all(&kv_full[vslot], phase, 0x220 + vslot);
                             if (!ok) break;
                             if (++stage == kStages) { stage = 0; phase ^= 1; }
-                            for (int t = 0; t < 2 && ok; ++t) {
+                            if (leader && warp == 8) MLT_TR(2, j, 4);
+                            for (int t = t_lo; t < t_hi && ok; ++t) {
                                 if (j >= it.J[t]) continue;
                                 // P_t(0) of an item also tells that the softmax warps have read the previous O_t
                                 ok = wait_all(&p_full[t], n_p[t] & 1, 0x230 + t);
                                 if (!ok) break;
+                                if (leader && warp == 8) MLT_TR(2, j, 5);
                                 ++n_p[t];
                                 tc_fence_after();
                                 issue_pv(t, vslot, j == 0);
+                                if (leader && warp == 8) MLT_TR(2, j, 6);
                                 if (leader) {
                                     umma_commit(&p_free[t]);
                                     if (j == it.J[t] - 1) umma_commit(&o_full[t]);
@@ -629,6 +647,7 @@ mha_fwd_kernel(const __grid_constant__ CUtensorMap tmap_q, const __grid_constant
                     // implies every UMMA issued before Q_t K_j^T, P_t(j-1) V among them.  D = 64: Q_t K_j^T is
                     // issued BEFORE P_t(j-1) V, so s_full says nothing; the guarantee is the p_free[t] wait inside
                     // the first exp_pass (w == 1), which every path to this point has passed.
+                    // (A single copy of the pass inside a retry loop was measured 7 % slower.)
                     float alpha = 1.0f;
                     if (moved) {
                         const float mxr = fmaxf(row_max(), m_run);
