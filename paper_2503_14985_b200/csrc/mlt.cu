@@ -72,6 +72,7 @@ int get_device(DeviceInfo* out) {
             set_smem(gemm_bf16_kernel<128, 6, true>, GemmSmem<128, 6>::kTotal) != MLT_OK ||
             set_smem(gemm_bf16_pair_kernel<6, true>, GemmPairSmem<6>::kTotal) != MLT_OK)
             return MLT_ERR_CUDA;
+        if (paged_configure() != 0) return MLT_ERR_CUDA;
         const int mha_rc = mha_configure();
         if (mha_rc == 1) return MLT_ERR_CUDA;
         d.mha_ok = mha_rc == 0;
@@ -520,7 +521,7 @@ int mlt_paged_attn_decode(const void* Q, const void* K_cache, const void* V_cach
     // use as many splits as the caller's scratch allows
     if (!workspace) workspace_bytes = 0;
     while (p.splits > 1 && paged_workspace_bytes(num_seqs, H, D, p.splits) > workspace_bytes) --p.splits;
-    p.blocks_per_split = (max_blocks_per_seq + p.splits - 1) / p.splits;
+    p.blocks_per_split = paged_blocks_per_split(max_blocks_per_seq, p.splits, block_size, H / H_kv);
     return paged_launch(p, D, workspace, static_cast<cudaStream_t>(stream));
 }
 
@@ -571,7 +572,7 @@ extern "C" int mlt_paged_attn_decode_static(const void* Q, const void* K_cache, 
     // the same split as mlt_paged_attn_decode makes with a full workspace; it must fit the built-in array
     if (paged_workspace_bytes(num_seqs, H, D, p.splits) > static_cast<size_t>(MLT_PAGED_STATIC_SCRATCH_BYTES))
         return MLT_ERR_SCRATCH_LIMIT;
-    p.blocks_per_split = (max_blocks_per_seq + p.splits - 1) / p.splits;
+    p.blocks_per_split = paged_blocks_per_split(max_blocks_per_seq, p.splits, block_size, H / H_kv);
     void* scratch = nullptr;
     rc = paged_static_scratch(&scratch);
     if (rc != MLT_OK) return rc;

@@ -296,6 +296,282 @@ paged_decode_kernel(const PagedParams p) {
     }
 }
 
+// ---------------------------------------------------------------------------------------------------------
+// Grouped heads (4 or 8 query heads per KV head) on the tensor cores.
+//
+// With G query heads reading the same keys and values, the FP32-pipe kernel above spends G times the
+// instructions per byte and runs out of issue slots long before HBM is busy (8 heads: 0.38 of the copy
+// bandwidth).  Here the G heads are the rows of a warp-level MMA (mma.sync m16n8k16, rows G..15 are zero):
+//   scores  S[16 x 16 tokens] = Q[16 x D] K^T   (2 column tiles of 8 tokens, D/16 steps)
+//   output  O[16 x D]        += P[16 x 16 tokens] V   (D/8 column tiles, one step)
+// per unit of 16 tokens and warp: 32 MMAs at D = 128 instead of about 500 packed FMAs.  K and V go from global
+// memory straight into the B fragments with 16-byte loads; no shared memory, no transposes:
+//  * the order of the summation index of an MMA is free as long as both operands use the same order, and so is
+//    the order of its output columns.  For Q K^T the 16 index slots of two consecutive steps are mapped to the 8
+//    consecutive elements of D a lane loads (lane (g, tg): elements pp*32 + tg*8 .. +7 of token column g), for Q and
+//    K alike.  The 8 output columns of score tile e are mapped to tokens 4*(c/2) + c%2 + 2e, so that lane (g, tg)
+//    ends up with the scores of head g for the 4 consecutive tokens 4 tg .. 4 tg + 3;
+//  * for P V the index slots 2tg, 2tg+1, 2tg+8, 2tg+9 of a lane are exactly those 4 tokens, so the score
+//    accumulators, exponentiated and packed, ARE the A fragment.  Output column n of tile (h, nt) is mapped to
+//    element h*64 + n*8 + nt of D: lane (g, tg) loads 8 consecutive elements (16 bytes) of each of its 4 tokens and
+//    pairs the same element of two tokens into one register with a byte permute.
+// Splits, partial format and the combine kernel are those of the kernel above.
+// ---------------------------------------------------------------------------------------------------------
+constexpr int kPagedRing = 3;  // units of 16 tokens per warp in the shared-memory ring (one being used, two in flight)
+template <int D>
+constexpr size_t paged_mma_smem_bytes() {
+    return static_cast<size_t>(kPagedWarps) * kPagedRing * (2 * (D / 32) + (D / 64) * 4) * 32 * 16;
+}
+// 16 bytes global -> shared, asynchronously; `valid` false: 16 zero bytes, the source is not read
+__device__ __forceinline__ void cp_async_16(void* smem_dst, const void* gmem_src, bool valid) {
+    asm volatile("cp.async.cg.shared.global [%0], [%1], 16, %2;" ::"r"(smem_u32(smem_dst)), "l"(gmem_src), "r"(valid ? 16 : 0)
+                 : "memory");
+}
+__device__ __forceinline__ void cp_async_commit() { asm volatile("cp.async.commit_group;" ::: "memory"); }
+template <int kPending>
+__device__ __forceinline__ void cp_async_wait() { asm volatile("cp.async.wait_group %0;" ::"n"(kPending) : "memory"); }
+
+__device__ __forceinline__ void mma_bf16_16816(float (&c)[4], uint32_t a0, uint32_t a1, uint32_t a2, uint32_t a3, uint32_t b0,
+                                               uint32_t b1) {
+    asm volatile("mma.sync.aligned.m16n8k16.row.col.f32.bf16.bf16.f32 {%0, %1, %2, %3}, {%4, %5, %6, %7}, {%8, %9}, {%0, %1, %2, %3};"
+                 : "+f"(c[0]), "+f"(c[1]), "+f"(c[2]), "+f"(c[3])
+                 : "r"(a0), "r"(a1), "r"(a2), "r"(a3), "r"(b0), "r"(b1));
+}
+
+template <int D, int G, int BS>
+__global__ void __launch_bounds__(kPagedThreads)
+paged_decode_mma_kernel(const PagedParams p) {
+    static_assert(G == 4 || G == 8, "rows of the MMA: 4 or 8 query heads");
+    constexpr int PP = D / 32;  // pairs of 16-element steps of Q K^T
+    constexpr int HV = D / 64;  // halves of D in the P V output mapping
+    __shared__ float sm_o[kPagedWarps][G][D];
+    __shared__ float2 sm_ml[kPagedWarps][G];
+
+    const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+    const int g = lane >> 2, tg = lane & 3;  // MMA fragment coordinates: row / column group, position in the group
+    const int sp = blockIdx.x, kvh = blockIdx.y, s = blockIdx.z;
+    const int head0 = kvh * G;
+    const int len = max(0, min(p.seq_lens[s], p.max_blocks * BS));
+    const int nblk = (len + BS - 1) / BS;
+    const int b0 = sp * p.blocks_per_split;
+    const int b1 = min(nblk, b0 + p.blocks_per_split);
+    if (p.splits > 1 && b0 >= nblk && !(sp == 0)) return;
+    const int tok_begin = b0 * BS;                     // a multiple of 16 (the host keeps blocks_per_split even for BS = 8)
+    const int tok_end = min(len, b1 * BS);
+
+    // Q as A fragments: rows g < G hold head head0 + g, the others are zero
+    uint32_t qa[PP][4];
+#pragma unroll
+    for (int pp = 0; pp < PP; ++pp) {
+        uint4 v = make_uint4(0u, 0u, 0u, 0u);
+        if (g < G) v = *reinterpret_cast<const uint4*>(p.Q + (static_cast<int64_t>(s) * p.H + head0 + g) * D + pp * 32 + tg * 8);
+        qa[pp][0] = v.x; qa[pp][1] = v.y; qa[pp][2] = v.z; qa[pp][3] = v.w;
+    }
+    float oacc[HV][8][4];
+#pragma unroll
+    for (int h = 0; h < HV; ++h)
+#pragma unroll
+        for (int nt = 0; nt < 8; ++nt)
+#pragma unroll
+            for (int i = 0; i < 4; ++i) oacc[h][nt][i] = 0.0f;
+    float m_run = -INFINITY, l_part = 0.0f;  // head g: running max (log2 units, equal in the 4 lanes of a group), this lane's share of the sum
+
+    const int* table = p.block_table + static_cast<int64_t>(s) * p.max_blocks;
+    const int64_t head_off = static_cast<int64_t>(kvh) * BS * D;
+    const int64_t blk_stride = static_cast<int64_t>(p.H_kv) * BS * D;
+    constexpr int NB = BS >= 16 ? 1 : 16 / BS;  // cache blocks per unit of 16 tokens
+
+    struct Unit {  // the K and V registers of one unit of 16 tokens
+        uint4 kr[2][PP], vr[HV][4];
+    };
+    // K and V travel global -> shared -> registers with cp.async: a warp keeps kRing - 1 units (8 KB each at D = 128)
+    // on their way from HBM while it computes, whatever the compiler does with the register loads.  Every lane copies
+    // exactly the 16-byte pieces it will read back itself (slot-major, lane-minor: no bank conflicts, and no
+    // synchronisation beyond the lane's own cp.async.wait_group).
+    constexpr int kSlots = 2 * PP + HV * 4;  // 16-byte pieces per lane and unit
+    extern __shared__ uint4 paged_ring[];    // [warp][kRing][kSlots][32]
+    uint4* my_ring = paged_ring + static_cast<size_t>(warp) * kPagedRing * kSlots * 32 + lane;
+    // Unit k of this warp starts at token first + k * kStep.  The table entries of 32 units at a time are read by
+    // one coalesced load (lane i: unit tab_base + i) and handed out by shuffles: a table load in every unit's path
+    // would put a second memory latency in front of its K/V loads.
+    constexpr int kStep = kPagedWarps * 16;
+    const int first = tok_begin + warp * 16;
+    const int n_units = first < tok_end ? (tok_end - first + kStep - 1) / kStep : 0;
+    int tab[NB];
+    int tab_base = -64;
+    auto issue_unit = [&](int stage, int k) -> bool {  // returns false if a bad table entry makes the unit unusable
+        const int u0 = first + k * kStep;
+        if (k >= tab_base + 32) {
+            tab_base = k;
+#pragma unroll
+            for (int i = 0; i < NB; ++i) {
+                const int b = (first + (k + lane) * kStep) / BS + i;
+                tab[i] = (k + lane < n_units && b < b1) ? table[b] : 0;
+            }
+        }
+        int phys[NB];
+        bool usable = true;
+#pragma unroll
+        for (int i = 0; i < NB; ++i) {
+            const int b = u0 / BS + i;
+            phys[i] = __shfl_sync(0xffffffffu, tab[i], k - tab_base);
+            if (b < b1 && (phys[i] < 0 || phys[i] >= p.num_blocks)) {  // never dereference a bad table entry
+                usable = false;
+                if (lane == 0 && atomicCAS(&g_status[0], 0u, kStatusBadBlock) == 0u) {
+                    g_status[1] = static_cast<unsigned int>(b);
+                    g_status[2] = static_cast<unsigned int>(s);
+                    g_status[3] = static_cast<unsigned int>(phys[i]);
+                }
+            }
+        }
+        if (!usable) return false;
+        auto token_ptr = [&](const __nv_bfloat16* cache, int tok) {  // tok: index inside the unit
+            const int blk = NB == 1 ? phys[0] : phys[(tok * NB) >> 4];
+            return cache + static_cast<int64_t>(blk) * blk_stride + head_off + static_cast<int64_t>((u0 + tok) % BS) * D;
+        };
+        uint4* dst = my_ring + stage * kSlots * 32;
+#pragma unroll
+        for (int e = 0; e < 2; ++e) {
+            const int tok = 4 * (g >> 1) + (g & 1) + 2 * e;
+            const bool in = u0 + tok < tok_end;  // beyond the sequence's end: zero fill, nothing is read
+            const __nv_bfloat16* kp = token_ptr(p.K_cache, in ? tok : 0) + tg * 8;
+#pragma unroll
+            for (int pp = 0; pp < PP; ++pp) cp_async_16(dst + (e * PP + pp) * 32, kp + pp * 32, in);
+        }
+#pragma unroll
+        for (int i = 0; i < 4; ++i) {
+            const int tok = 4 * tg + i;
+            const bool in = u0 + tok < tok_end;
+            const __nv_bfloat16* vp = token_ptr(p.V_cache, in ? tok : 0) + g * 8;
+#pragma unroll
+            for (int h = 0; h < HV; ++h) cp_async_16(dst + (2 * PP + h * 4 + i) * 32, vp + h * 64, in);
+        }
+        return true;
+    };
+    auto fetch_unit = [&](Unit& un, int stage) {
+        const uint4* src = my_ring + stage * kSlots * 32;
+#pragma unroll
+        for (int e = 0; e < 2; ++e)
+#pragma unroll
+            for (int pp = 0; pp < PP; ++pp) un.kr[e][pp] = src[(e * PP + pp) * 32];
+#pragma unroll
+        for (int h = 0; h < HV; ++h)
+#pragma unroll
+            for (int i = 0; i < 4; ++i) un.vr[h][i] = src[(2 * PP + h * 4 + i) * 32];
+    };
+    auto compute_unit = [&](const Unit& un, int u0) {
+        // ---- scores of head g for tokens 4 tg .. 4 tg + 3 ----
+        float sc[2][4];
+#pragma unroll
+        for (int e = 0; e < 2; ++e) {
+#pragma unroll
+            for (int i = 0; i < 4; ++i) sc[e][i] = 0.0f;
+#pragma unroll
+            for (int pp = 0; pp < PP; ++pp) {
+                mma_bf16_16816(sc[e], qa[pp][0], 0u, qa[pp][1], 0u, un.kr[e][pp].x, un.kr[e][pp].y);
+                mma_bf16_16816(sc[e], qa[pp][2], 0u, qa[pp][3], 0u, un.kr[e][pp].z, un.kr[e][pp].w);
+            }
+        }
+        float x[4];
+#pragma unroll
+        for (int i = 0; i < 4; ++i)
+            x[i] = (u0 + 4 * tg + i < tok_end) ? sc[i >> 1][i & 1] * p.scale_log2e : -INFINITY;
+        float mb = fmaxf(fmaxf(x[0], x[1]), fmaxf(x[2], x[3]));
+        mb = fmaxf(mb, __shfl_xor_sync(0xffffffffu, mb, 1));
+        mb = fmaxf(mb, __shfl_xor_sync(0xffffffffu, mb, 2));
+        const float mn = fmaxf(m_run, mb);  // finite: token u0 of this unit is inside the sequence
+        const float alpha = fast_exp2(m_run - mn);  // 0 for the first unit (m_run = -inf)
+        float pw[4];
+#pragma unroll
+        for (int i = 0; i < 4; ++i) pw[i] = fast_exp2(x[i] - mn);
+        l_part = l_part * alpha + (pw[0] + pw[1]) + (pw[2] + pw[3]);
+        if (__any_sync(0xffffffffu, mn != m_run)) {  // the maximum rarely moves after the first units
+#pragma unroll
+            for (int h = 0; h < HV; ++h)
+#pragma unroll
+                for (int nt = 0; nt < 8; ++nt) {
+                    oacc[h][nt][0] *= alpha;
+                    oacc[h][nt][1] *= alpha;
+                }
+        }
+        m_run = mn;
+        // ---- O += P V: the probabilities are the A fragment as they stand ----
+        const uint32_t pa0 = pack_bf16x2(pw[0], pw[1]), pa2 = pack_bf16x2(pw[2], pw[3]);
+#pragma unroll
+        for (int h = 0; h < HV; ++h) {
+            const uint32_t w0[4] = {un.vr[h][0].x, un.vr[h][0].y, un.vr[h][0].z, un.vr[h][0].w};
+            const uint32_t w1[4] = {un.vr[h][1].x, un.vr[h][1].y, un.vr[h][1].z, un.vr[h][1].w};
+            const uint32_t w2[4] = {un.vr[h][2].x, un.vr[h][2].y, un.vr[h][2].z, un.vr[h][2].w};
+            const uint32_t w3[4] = {un.vr[h][3].x, un.vr[h][3].y, un.vr[h][3].z, un.vr[h][3].w};
+#pragma unroll
+            for (int nt = 0; nt < 8; ++nt) {
+                const uint32_t sel = (nt & 1) ? 0x7632u : 0x5410u;  // the same element of D from two tokens
+                const uint32_t vb0 = __byte_perm(w0[nt >> 1], w1[nt >> 1], sel);
+                const uint32_t vb1 = __byte_perm(w2[nt >> 1], w3[nt >> 1], sel);
+                mma_bf16_16816(oacc[h][nt], pa0, 0u, pa2, 0u, vb0, vb1);
+            }
+        }
+    };
+    // One cp.async group per unit, committed even when empty so that "all but the newest kRing - 1 groups" is always "unit k has landed".
+    uint32_t usable = 0;  // bit (k % 32): unit k may be used
+#pragma unroll
+    for (int k = 0; k < kPagedRing - 1; ++k) {
+        if (k < n_units && issue_unit(k, k)) usable |= 1u << k;
+        cp_async_commit();
+    }
+    for (int k = 0; k < n_units; ++k) {
+        const int kk = k + kPagedRing - 1;
+        if (kk < n_units) {
+            if (issue_unit(kk % kPagedRing, kk)) usable |= 1u << (kk & 31);
+            else usable &= ~(1u << (kk & 31));
+        }
+        cp_async_commit();
+        cp_async_wait<kPagedRing - 1>();
+        if (usable & (1u << (k & 31))) {
+            Unit un;
+            fetch_unit(un, k % kPagedRing);
+            compute_unit(un, first + k * kStep);
+        }
+    }
+
+    // ---- warp result: sum of the group's shares of l; output element of (h, nt, column 2 tg + i) is h*64 + (2 tg + i)*8 + nt ----
+    l_part += __shfl_xor_sync(0xffffffffu, l_part, 1);
+    l_part += __shfl_xor_sync(0xffffffffu, l_part, 2);
+    if (g < G) {
+#pragma unroll
+        for (int h = 0; h < HV; ++h)
+#pragma unroll
+            for (int nt = 0; nt < 8; ++nt) {
+                sm_o[warp][g][h * 64 + (2 * tg) * 8 + nt] = oacc[h][nt][0];
+                sm_o[warp][g][h * 64 + (2 * tg + 1) * 8 + nt] = oacc[h][nt][1];
+            }
+        if (tg == 0) sm_ml[warp][g] = make_float2(m_run, l_part);
+    }
+    __syncthreads();
+    for (int idx = threadIdx.x; idx < G * D; idx += kPagedThreads) {
+        const int gg = idx / D, d = idx % D;
+        float mt = -INFINITY;
+#pragma unroll
+        for (int w = 0; w < kPagedWarps; ++w) mt = fmaxf(mt, sm_ml[w][gg].x);
+        float lt = 0.0f, ot = 0.0f;
+#pragma unroll
+        for (int w = 0; w < kPagedWarps; ++w) {
+            const float2 ml = sm_ml[w][gg];
+            const float sw = (ml.x == -INFINITY) ? 0.0f : fast_exp2(ml.x - mt);
+            lt += ml.y * sw;
+            ot += sm_o[w][gg][d] * sw;
+        }
+        const int64_t row = static_cast<int64_t>(s) * p.H + head0 + gg;
+        if (p.splits == 1) {
+            p.O[row * D + d] = __float2bfloat16(lt > 0.0f ? ot / lt : 0.0f);
+            if (d == 0 && p.LSE) p.LSE[row] = lt > 0.0f ? (mt + log2f(lt)) * 0.6931471805599453f : -INFINITY;
+        } else {
+            p.part_o[(row * p.splits + sp) * D + d] = ot;
+            if (d == 0) p.part_ml[row * p.splits + sp] = make_float2(mt, lt);
+        }
+    }
+}
+
 // O[row] = sum over splits of the partials, rescaled to the common max; one CTA of D threads per (seq, head).
 // The {m, l} pairs go through shared memory once, and the partial outputs are read with independent loads
 // (eight in flight per thread), so the kernel is a few microseconds of latency rather than a chain of them.
@@ -362,14 +638,32 @@ inline int paged_choose_splits(int num_seqs, int H_kv, int group, int max_blocks
     return std::max(1, std::min(splits, kPagedMaxSplits));
 }
 
+// KV blocks per CTA of a split sequence.  The grouped-head kernel works in units of 16 tokens, so with 8-token
+// blocks every CTA starts at an even block.
+inline int paged_blocks_per_split(int max_blocks, int splits, int block_size, int group) {
+    int bps = (max_blocks + splits - 1) / splits;
+    if (group >= 4 && block_size == 8) bps = (bps + 1) & ~1;
+    return bps;
+}
+
 template <int D, int G>
 int paged_launch_bs(const PagedParams& p, cudaStream_t st) {
     const dim3 grid(p.splits, p.H_kv * p.head_groups, p.num_seqs);
-    switch (p.block_size) {
-        case 8: paged_decode_kernel<D, G, 8><<<grid, kPagedThreads, 0, st>>>(p); break;
-        case 16: paged_decode_kernel<D, G, 16><<<grid, kPagedThreads, 0, st>>>(p); break;
-        case 32: paged_decode_kernel<D, G, 32><<<grid, kPagedThreads, 0, st>>>(p); break;
-        default: return 2;
+    if constexpr (G >= 4) {  // grouped heads: rows of a tensor-core MMA
+        constexpr size_t smem = paged_mma_smem_bytes<D>();
+        switch (p.block_size) {
+            case 8: paged_decode_mma_kernel<D, G, 8><<<grid, kPagedThreads, smem, st>>>(p); break;
+            case 16: paged_decode_mma_kernel<D, G, 16><<<grid, kPagedThreads, smem, st>>>(p); break;
+            case 32: paged_decode_mma_kernel<D, G, 32><<<grid, kPagedThreads, smem, st>>>(p); break;
+            default: return 2;
+        }
+    } else {
+        switch (p.block_size) {
+            case 8: paged_decode_kernel<D, G, 8><<<grid, kPagedThreads, 0, st>>>(p); break;
+            case 16: paged_decode_kernel<D, G, 16><<<grid, kPagedThreads, 0, st>>>(p); break;
+            case 32: paged_decode_kernel<D, G, 32><<<grid, kPagedThreads, 0, st>>>(p); break;
+            default: return 2;
+        }
     }
     if (cudaGetLastError() != cudaSuccess) return 4;
     if (p.splits > 1) {
@@ -393,14 +687,23 @@ int paged_launch_g(const PagedParams& p, cudaStream_t st) {
         case 1: return paged_launch_bs<D, 1>(p, st);
         case 2: return paged_launch_bs<D, 2>(p, st);
         case 4: return paged_launch_bs<D, 4>(p, st);
-        case 8: {
-            // 8 heads per CTA need 255 registers and leave two CTAs per SM; two CTAs of 4 heads run faster
-            PagedParams p2 = p;
-            p2.head_groups = 2;
-            return paged_launch_bs<D, 4>(p2, st);
-        }
+        case 8: return paged_launch_bs<D, 8>(p, st);
         default: return 2;
     }
+}
+
+// Once per device: the grouped-head kernels' shared-memory ring is larger than the default limit.
+template <int D, int G>
+int paged_configure_one() {
+    const int bytes = static_cast<int>(paged_mma_smem_bytes<D>());
+    if (cudaFuncSetAttribute(paged_decode_mma_kernel<D, G, 8>, cudaFuncAttributeMaxDynamicSharedMemorySize, bytes) != cudaSuccess ||
+        cudaFuncSetAttribute(paged_decode_mma_kernel<D, G, 16>, cudaFuncAttributeMaxDynamicSharedMemorySize, bytes) != cudaSuccess ||
+        cudaFuncSetAttribute(paged_decode_mma_kernel<D, G, 32>, cudaFuncAttributeMaxDynamicSharedMemorySize, bytes) != cudaSuccess)
+        return 1;
+    return 0;
+}
+inline int paged_configure() {
+    return paged_configure_one<64, 4>() | paged_configure_one<64, 8>() | paged_configure_one<128, 4>() | paged_configure_one<128, 8>();
 }
 
 // workspace layout: part_o floats first, then part_ml pairs
