@@ -68,6 +68,10 @@ def poison_unused(Kc, Vc, table, lens, bs):
 CASES = [  # S, H, H_kv, D, block_size, min_len, max_len
     (3, 4, 4, 128, 16, 1, 100), (2, 8, 8, 64, 16, 17, 300), (5, 8, 2, 128, 16, 50, 700), (4, 8, 1, 64, 8, 1, 90),
     (2, 4, 2, 128, 32, 200, 1500), (1, 2, 2, 128, 16, 5000, 5000), (7, 16, 8, 64, 32, 1, 2000), (3, 2, 2, 64, 8, 1, 7),
+    # 4 or 8 query heads per KV head (the tensor-core kernel), every block size and head dimension, lengths that end
+    # inside a 16-token unit, and (8-token blocks) splits that must start at an even block
+    (3, 16, 2, 128, 32, 100, 3000), (4, 8, 2, 64, 8, 1, 500), (2, 32, 4, 128, 8, 700, 2900), (5, 16, 4, 64, 16, 1, 1100),
+    (2, 8, 1, 128, 16, 4000, 6000), (6, 4, 1, 64, 32, 1, 40),
 ]
 
 
