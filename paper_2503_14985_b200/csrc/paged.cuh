@@ -304,8 +304,9 @@ paged_decode_kernel(const PagedParams p) {
 // bandwidth).  Here the G heads are the rows of a warp-level MMA (mma.sync m16n8k16, rows G..15 are zero):
 //   scores  S[16 x 16 tokens] = Q[16 x D] K^T   (2 column tiles of 8 tokens, D/16 steps)
 //   output  O[16 x D]        += P[16 x 16 tokens] V   (D/8 column tiles, one step)
-// per unit of 16 tokens and warp: 32 MMAs at D = 128 instead of about 500 packed FMAs.  K and V go from global
-// memory straight into the B fragments with 16-byte loads; no shared memory, no transposes:
+// per unit of 16 tokens and warp: 32 MMAs at D = 128 instead of about 500 packed FMAs.  K and V rows go from global
+// memory into a per-warp shared-memory ring by bulk copies and from there into the B fragments as they are, with
+// 16-byte loads and no transposes:
 //  * the order of the summation index of an MMA is free as long as both operands use the same order, and so is
 //    the order of its output columns.  For Q K^T the 16 index slots of two consecutive steps are mapped to the 8
 //    consecutive elements of D a lane loads (lane (g, tg): elements pp*32 + tg*8 .. +7 of token column g), for Q and
@@ -317,19 +318,30 @@ paged_decode_kernel(const PagedParams p) {
 //    pairs the same element of two tokens into one register with a byte permute.
 // Splits, partial format and the combine kernel are those of the kernel above.
 // ---------------------------------------------------------------------------------------------------------
-constexpr int kPagedRing = 3;  // units of 16 tokens per warp in the shared-memory ring (one being used, two in flight)
+// Units of 16 tokens per warp in the shared-memory ring (one being used, one in flight), and CTAs per SM the
+// grouped-head kernel is compiled for (168 registers).  Measured (32 / 128 sequences, H = 32, H_kv = 4, 2k-4k
+// tokens): ring 2 with 3 CTAs per SM 50 / 155 us; ring 3 with 2 CTAs 52 / 169; ring 4 with 2 CTAs 67 / 237; ring 2
+// with 4 CTAs (128 registers) 56 / 171.
+constexpr int kPagedRing = 2;
+constexpr int kPagedMmaCtasPerSm = 3;
+// A unit in shared memory: 16 K rows then 16 V rows of D BF16 each, as they lie in the cache (one bulk copy per
+// tensor and cache block).  The fragment loads meet 2-way (K) and 4-way (V) bank conflicts; the load/store unit has
+// the room (a quarter busy without them), and copies of single padded rows were far slower (256-byte bulk copies:
+// 1.8-2.1 TB/s).
+template <int D>
+struct PagedRow {
+    static constexpr int kPitch = D * 2;
+};
 template <int D>
 constexpr size_t paged_mma_smem_bytes() {
-    return static_cast<size_t>(kPagedWarps) * kPagedRing * (2 * (D / 32) + (D / 64) * 4) * 32 * 16;
+    return static_cast<size_t>(kPagedWarps) * kPagedRing * 32 * PagedRow<D>::kPitch + 128;
 }
-// 16 bytes global -> shared, asynchronously; `valid` false: 16 zero bytes, the source is not read
-__device__ __forceinline__ void cp_async_16(void* smem_dst, const void* gmem_src, bool valid) {
-    asm volatile("cp.async.cg.shared.global [%0], [%1], 16, %2;" ::"r"(smem_u32(smem_dst)), "l"(gmem_src), "r"(valid ? 16 : 0)
+// global -> shared bulk copy of `bytes` (a multiple of 16, both addresses 16-byte aligned), completion counted on `bar`
+__device__ __forceinline__ void bulk_load(void* smem_dst, const void* gmem_src, uint32_t bytes, uint64_t* bar) {
+    asm volatile("cp.async.bulk.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1], %2, [%3];"
+                 ::"r"(smem_u32(smem_dst)), "l"(gmem_src), "r"(bytes), "r"(smem_u32(bar))
                  : "memory");
 }
-__device__ __forceinline__ void cp_async_commit() { asm volatile("cp.async.commit_group;" ::: "memory"); }
-template <int kPending>
-__device__ __forceinline__ void cp_async_wait() { asm volatile("cp.async.wait_group %0;" ::"n"(kPending) : "memory"); }
 
 __device__ __forceinline__ void mma_bf16_16816(float (&c)[4], uint32_t a0, uint32_t a1, uint32_t a2, uint32_t a3, uint32_t b0,
                                                uint32_t b1) {
@@ -339,12 +351,11 @@ __device__ __forceinline__ void mma_bf16_16816(float (&c)[4], uint32_t a0, uint3
 }
 
 template <int D, int G, int BS>
-__global__ void __launch_bounds__(kPagedThreads)
+__global__ void __launch_bounds__(kPagedThreads, kPagedMmaCtasPerSm)
 paged_decode_mma_kernel(const PagedParams p) {
     static_assert(G == 4 || G == 8, "rows of the MMA: 4 or 8 query heads");
     constexpr int PP = D / 32;  // pairs of 16-element steps of Q K^T
     constexpr int HV = D / 64;  // halves of D in the P V output mapping
-    __shared__ float sm_o[kPagedWarps][G][D];
     __shared__ float2 sm_ml[kPagedWarps][G];
 
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
@@ -384,13 +395,24 @@ paged_decode_mma_kernel(const PagedParams p) {
     struct Unit {  // the K and V registers of one unit of 16 tokens
         uint4 kr[2][PP], vr[HV][4];
     };
-    // K and V travel global -> shared -> registers with cp.async: a warp keeps kRing - 1 units (8 KB each at D = 128)
-    // on their way from HBM while it computes, whatever the compiler does with the register loads.  Every lane copies
-    // exactly the 16-byte pieces it will read back itself (slot-major, lane-minor: no bank conflicts, and no
-    // synchronisation beyond the lane's own cp.async.wait_group).
-    constexpr int kSlots = 2 * PP + HV * 4;  // 16-byte pieces per lane and unit
-    extern __shared__ uint4 paged_ring[];    // [warp][kRing][kSlots][32]
-    uint4* my_ring = paged_ring + static_cast<size_t>(warp) * kPagedRing * kSlots * 32 + lane;
+    // K and V travel global -> shared by bulk copies (the TMA engine: no address generation, no load/store-unit
+    // queue entries in the SM; with per-lane 16-byte cp.async the same ring streamed 4.3-4.6 TB/s at best), one copy
+    // per tensor and cache block (a unit of 16 tokens is one block, half a block, or two blocks).  Each warp has its
+    // own ring of kPagedRing units and one mbarrier per ring stage.
+    constexpr int kPitch = PagedRow<D>::kPitch;
+    constexpr int kUnitBytes = 32 * kPitch;
+    extern __shared__ uint8_t paged_ring_raw[];
+    uint8_t* ring_base = reinterpret_cast<uint8_t*>((reinterpret_cast<uintptr_t>(paged_ring_raw) + 127) & ~uintptr_t(127));
+    uint8_t* my_ring = ring_base + static_cast<size_t>(warp) * kPagedRing * kUnitBytes;
+    __shared__ uint64_t ring_bar[kPagedWarps][kPagedRing];
+    __shared__ uint32_t ring_abort;
+    if (lane == 0) {
+#pragma unroll
+        for (int i = 0; i < kPagedRing; ++i) mbar_init(&ring_bar[warp][i], 1);
+        if (warp == 0) ring_abort = 0;
+        fence_mbar_init();
+    }
+    __syncthreads();
     // Unit k of this warp starts at token first + k * kStep.  The table entries of 32 units at a time are read by
     // one coalesced load (lane i: unit tab_base + i) and handed out by shuffles: a table load in every unit's path
     // would put a second memory latency in front of its K/V loads.
@@ -425,39 +447,47 @@ paged_decode_mma_kernel(const PagedParams p) {
             }
         }
         if (!usable) return false;
-        auto token_ptr = [&](const __nv_bfloat16* cache, int tok) {  // tok: index inside the unit
-            const int blk = NB == 1 ? phys[0] : phys[(tok * NB) >> 4];
-            return cache + static_cast<int64_t>(blk) * blk_stride + head_off + static_cast<int64_t>((u0 + tok) % BS) * D;
-        };
-        uint4* dst = my_ring + stage * kSlots * 32;
-#pragma unroll
-        for (int e = 0; e < 2; ++e) {
-            const int tok = 4 * (g >> 1) + (g & 1) + 2 * e;
-            const bool in = u0 + tok < tok_end;  // beyond the sequence's end: zero fill, nothing is read
-            const __nv_bfloat16* kp = token_ptr(p.K_cache, in ? tok : 0) + tg * 8;
-#pragma unroll
-            for (int pp = 0; pp < PP; ++pp) cp_async_16(dst + (e * PP + pp) * 32, kp + pp * 32, in);
+        // every lane must be done reading the stage's previous contents before the copies overwrite them
+        __syncwarp();
+        const int rows_in = min(16, tok_end - u0);  // rows beyond the sequence's end are not copied but zeroed
+        uint64_t* bar = &ring_bar[warp][stage];
+        if (lane == 0) mbar_arrive_expect_tx(bar, 2u * rows_in * (D * 2));
+        __syncwarp();
+        uint8_t* dst = my_ring + stage * kUnitBytes;
+        constexpr int kPieceRows = 16 / NB;  // token rows per bulk copy: a cache block, or the half of one that the unit covers
+        if (lane < 2 * NB) {  // lanes 0 .. NB-1: the K pieces, lanes NB .. 2 NB - 1: the V pieces
+            const int piece = lane % NB, is_v = lane / NB;
+            const int rows = min(kPieceRows, rows_in - piece * kPieceRows);
+            if (rows > 0) {
+                const int t0 = u0 + piece * kPieceRows;
+                const __nv_bfloat16* src = (is_v ? p.V_cache : p.K_cache) + static_cast<int64_t>(phys[piece]) * blk_stride + head_off +
+                                           static_cast<int64_t>(t0 % BS) * D;
+                bulk_load(dst + (is_v * 16 + piece * kPieceRows) * kPitch, src, rows * (D * 2), bar);
+            }
         }
-#pragma unroll
-        for (int i = 0; i < 4; ++i) {
-            const int tok = 4 * tg + i;
-            const bool in = u0 + tok < tok_end;
-            const __nv_bfloat16* vp = token_ptr(p.V_cache, in ? tok : 0) + g * 8;
-#pragma unroll
-            for (int h = 0; h < HV; ++h) cp_async_16(dst + (2 * PP + h * 4 + i) * 32, vp + h * 64, in);
+        if (rows_in < 16) {  // a weight of 0 must not meet whatever the cache holds beyond the sequence's end
+            for (int i = lane; i < (16 - rows_in) * (kPitch / 16); i += 32) {
+                reinterpret_cast<uint4*>(dst + rows_in * kPitch)[i] = make_uint4(0u, 0u, 0u, 0u);
+                reinterpret_cast<uint4*>(dst + (16 + rows_in) * kPitch)[i] = make_uint4(0u, 0u, 0u, 0u);
+            }
+            __syncwarp();
         }
         return true;
     };
     auto fetch_unit = [&](Unit& un, int stage) {
-        const uint4* src = my_ring + stage * kSlots * 32;
+        const uint8_t* src = my_ring + stage * kUnitBytes;
 #pragma unroll
-        for (int e = 0; e < 2; ++e)
+        for (int e = 0; e < 2; ++e) {
+            const int tok = 4 * (g >> 1) + (g & 1) + 2 * e;
 #pragma unroll
-            for (int pp = 0; pp < PP; ++pp) un.kr[e][pp] = src[(e * PP + pp) * 32];
+            for (int pp = 0; pp < PP; ++pp)
+                un.kr[e][pp] = *reinterpret_cast<const uint4*>(src + tok * kPitch + (pp * 32 + tg * 8) * 2);
+        }
 #pragma unroll
         for (int h = 0; h < HV; ++h)
 #pragma unroll
-            for (int i = 0; i < 4; ++i) un.vr[h][i] = src[(2 * PP + h * 4 + i) * 32];
+            for (int i = 0; i < 4; ++i)
+                un.vr[h][i] = *reinterpret_cast<const uint4*>(src + (16 + 4 * tg + i) * kPitch + (h * 64 + g * 8) * 2);
     };
     auto compute_unit = [&](const Unit& un, int u0) {
         // ---- scores of head g for tokens 4 tg .. 4 tg + 3 ----
@@ -512,28 +542,32 @@ paged_decode_mma_kernel(const PagedParams p) {
             }
         }
     };
-    // One cp.async group per unit, committed even when empty so that "all but the newest kRing - 1 groups" is always "unit k has landed".
+    // Stage k % kPagedRing holds unit k; its barrier completes once per use, so the parity to wait for is that of
+    // (k / kPagedRing).
     uint32_t usable = 0;  // bit (k % 32): unit k may be used
+    bool ok = true;
 #pragma unroll
-    for (int k = 0; k < kPagedRing - 1; ++k) {
+    for (int k = 0; k < kPagedRing - 1; ++k)
         if (k < n_units && issue_unit(k, k)) usable |= 1u << k;
-        cp_async_commit();
-    }
-    for (int k = 0; k < n_units; ++k) {
+    for (int k = 0; k < n_units && ok; ++k) {
         const int kk = k + kPagedRing - 1;
         if (kk < n_units) {
             if (issue_unit(kk % kPagedRing, kk)) usable |= 1u << (kk & 31);
             else usable &= ~(1u << (kk & 31));
         }
-        cp_async_commit();
-        cp_async_wait<kPagedRing - 1>();
         if (usable & (1u << (k & 31))) {
+            ok = __all_sync(0xffffffffu, mbar_wait(&ring_bar[warp][k % kPagedRing], (k / kPagedRing) & 1, &ring_abort, 0x500 + warp)) != 0;
+            if (!ok) break;
             Unit un;
             fetch_unit(un, k % kPagedRing);
             compute_unit(un, first + k * kStep);
         }
     }
 
+    // The warps' partial outputs go where the ring was (every warp's copies have landed and been read by now).
+    __syncthreads();
+    float (*sm_o)[G][D] = reinterpret_cast<float (*)[G][D]>(ring_base);
+    static_assert(sizeof(float) * kPagedWarps * G * D <= kPagedWarps * kPagedRing * 32 * PagedRow<D>::kPitch, "partials fit the ring");
     // ---- warp result: sum of the group's shares of l; output element of (h, nt, column 2 tg + i) is h*64 + (2 tg + i)*8 + nt ----
     l_part += __shfl_xor_sync(0xffffffffu, l_part, 1);
     l_part += __shfl_xor_sync(0xffffffffu, l_part, 2);
