@@ -502,6 +502,8 @@ int paged_prepare(const void* Q, const void* K_cache, const void* V_cache, const
     if (debug_env().paged_splits) p->splits = std::min(debug_env().paged_splits, kPagedMaxSplits);
     p->scale_log2e = scale * 1.4426950408889634f;
     p->head_groups = 1;
+    p->balanced = 0;
+    p->balanced_ctas = 0;
     *launch = true;
     return MLT_OK;
 }
@@ -520,6 +522,8 @@ int mlt_paged_attn_decode(const void* Q, const void* K_cache, const void* V_cach
     if (rc != MLT_OK || !launch) return rc;
     // use as many splits as the caller's scratch allows
     if (!workspace) workspace_bytes = 0;
+    if (paged_use_balanced(p, dev.sm_count) && paged_workspace_bytes(num_seqs, H, D, kPagedMaxSplits) <= workspace_bytes)
+        paged_set_balanced(&p, dev.sm_count);
     while (p.splits > 1 && paged_workspace_bytes(num_seqs, H, D, p.splits) > workspace_bytes) --p.splits;
     p.blocks_per_split = paged_blocks_per_split(max_blocks_per_seq, p.splits, block_size, H / H_kv);
     return paged_launch(p, D, workspace, static_cast<cudaStream_t>(stream));
@@ -570,6 +574,9 @@ extern "C" int mlt_paged_attn_decode_static(const void* Q, const void* K_cache, 
                            max_blocks_per_seq, num_blocks, scale, &p, &dev, &launch);
     if (rc != MLT_OK || !launch) return rc;
     // the same split as mlt_paged_attn_decode makes with a full workspace; it must fit the built-in array
+    if (paged_use_balanced(p, dev.sm_count) &&
+        paged_workspace_bytes(num_seqs, H, D, kPagedMaxSplits) <= static_cast<size_t>(MLT_PAGED_STATIC_SCRATCH_BYTES))
+        paged_set_balanced(&p, dev.sm_count);
     if (paged_workspace_bytes(num_seqs, H, D, p.splits) > static_cast<size_t>(MLT_PAGED_STATIC_SCRATCH_BYTES))
         return MLT_ERR_SCRATCH_LIMIT;
     p.blocks_per_split = paged_blocks_per_split(max_blocks_per_seq, p.splits, block_size, H / H_kv);

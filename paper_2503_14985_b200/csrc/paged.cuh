@@ -46,6 +46,8 @@ struct PagedParams {
                            // the CTAs beyond a short sequence's end exit at once
     float scale_log2e;
     int head_groups;       // CTAs per KV head (1, or 2 when 8 query heads per KV head run as two groups of 4)
+    int balanced;          // grouped-head kernel: equal work per CTA (see paged_decode_mma_kernel); splits = kPagedMaxSplits
+    int balanced_ctas;     // ... and the grid it is launched with (the combine kernel repeats the arithmetic)
 };
 
 __device__ __forceinline__ void bf16x8_to_f32(const uint4& v, float (&f)[8]) {
@@ -350,25 +352,146 @@ __device__ __forceinline__ void mma_bf16_16816(float (&c)[4], uint32_t a0, uint3
                  : "r"(a0), "r"(a1), "r"(a2), "r"(a3), "r"(b0), "r"(b1));
 }
 
+// Equal work per CTA (p.balanced): the live chunks of kPagedChunkTokens tokens of all (sequence, KV head) rows, in
+// the order sequence, KV head, chunk, are numbered 0 .. n-1 and CTA c takes numbers c*q .. (c+1)*q - 1, whatever
+// rows they belong to; it writes one partial per row it touches, into slot c - (first CTA of that row).  The numbers
+// come from seq_lens, which only the device knows: every CTA scans them itself.  q is at least n / gridDim.x and at
+// least a 30th of the longest row, so that no row has more than kPagedMaxSplits partials.
+constexpr int kPagedChunkTokens = 128;
+constexpr int kPagedBalanceMaxSeqs = 1024;  // the scan's shared-memory table; beyond it the static split is used
+__device__ __forceinline__ int paged_chunks(const PagedParams& p, int s) {
+    const int len = max(0, min(p.seq_lens[s], p.max_blocks * p.block_size));
+    return (len + kPagedChunkTokens - 1) / kPagedChunkTokens;
+}
+__device__ __forceinline__ int paged_quota(long long n, int max_row, int ctas) {
+    const long long q = max(max((n + ctas - 1) / ctas, static_cast<long long>((max_row + 29) / 30)), 1ll);
+    return static_cast<int>(q);
+}
+
 template <int D, int G, int BS>
 __global__ void __launch_bounds__(kPagedThreads, kPagedMmaCtasPerSm)
 paged_decode_mma_kernel(const PagedParams p) {
     static_assert(G == 4 || G == 8, "rows of the MMA: 4 or 8 query heads");
     constexpr int PP = D / 32;  // pairs of 16-element steps of Q K^T
     constexpr int HV = D / 64;  // halves of D in the P V output mapping
+    constexpr int NB = BS >= 16 ? 1 : 16 / BS;  // cache blocks per unit of 16 tokens
     __shared__ float2 sm_ml[kPagedWarps][G];
+    __shared__ int sm_pre[kPagedBalanceMaxSeqs + 1];  // balanced: chunks of all sequences before s
+    __shared__ int sm_red[2 * kPagedWarps];
 
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
     const int g = lane >> 2, tg = lane & 3;  // MMA fragment coordinates: row / column group, position in the group
-    const int sp = blockIdx.x, kvh = blockIdx.y, s = blockIdx.z;
+
+    // K and V travel global -> shared by bulk copies (the TMA engine: no address generation, no load/store-unit
+    // queue entries in the SM; with per-lane 16-byte cp.async the same ring streamed 4.3-4.6 TB/s at best), one copy
+    // per tensor and cache block (a unit of 16 tokens is one block, half a block, or two blocks).  Each warp has its
+    // own ring of kPagedRing units and one mbarrier per ring stage.
+    constexpr int kPitch = PagedRow<D>::kPitch;
+    constexpr int kUnitBytes = 32 * kPitch;
+    extern __shared__ uint8_t paged_ring_raw[];
+    uint8_t* ring_base = reinterpret_cast<uint8_t*>((reinterpret_cast<uintptr_t>(paged_ring_raw) + 127) & ~uintptr_t(127));
+    uint8_t* my_ring = ring_base + static_cast<size_t>(warp) * kPagedRing * kUnitBytes;
+    __shared__ uint64_t ring_bar[kPagedWarps][kPagedRing];
+    __shared__ uint32_t ring_abort;
+    if (lane == 0) {
+#pragma unroll
+        for (int i = 0; i < kPagedRing; ++i) mbar_init(&ring_bar[warp][i], 1);
+        if (warp == 0) ring_abort = 0;
+        fence_mbar_init();
+    }
+
+    // ---- which segments (row, token range, partial slot) this CTA works on ----
+    int seg_s, seg_kvh, seg_tok_begin, seg_tok_end, seg_slot;
+    long long bal_i = 0, bal_hi = 0;  // balanced: next live chunk number, end of this CTA's numbers
+    int bal_q = 1;
+    if (!p.balanced) {
+        seg_s = blockIdx.z;
+        seg_kvh = blockIdx.y;
+        const int len = max(0, min(p.seq_lens[seg_s], p.max_blocks * BS));
+        const int nblk = (len + BS - 1) / BS;
+        const int b0 = blockIdx.x * p.blocks_per_split;  // even for BS = 8 (the host sees to it): a multiple of 16 tokens
+        const int b1 = min(nblk, b0 + p.blocks_per_split);
+        if (p.splits > 1 && b0 >= nblk && blockIdx.x != 0) return;  // nothing of this sequence here (split 0 reports an empty one)
+        seg_tok_begin = b0 * BS;
+        seg_tok_end = min(len, b1 * BS);
+        seg_slot = blockIdx.x;
+        __syncthreads();  // the ring barriers are initialised
+    } else {
+        // inclusive scan of the sequences' chunk counts into sm_pre, and their maximum
+        const int S = p.num_seqs;
+        const int per = (S + kPagedThreads - 1) / kPagedThreads;
+        const int s_lo = min(S, static_cast<int>(threadIdx.x) * per), s_hi = min(S, s_lo + per);
+        int sum = 0, mx = 0;
+        for (int s2 = s_lo; s2 < s_hi; ++s2) {
+            const int c = paged_chunks(p, s2);
+            sum += c;
+            mx = max(mx, c);
+        }
+        int incl = sum;
+#pragma unroll
+        for (int w = 1; w < 32; w <<= 1) {
+            const int v = __shfl_up_sync(0xffffffffu, incl, w);
+            if (lane >= w) incl += v;
+            mx = max(mx, __shfl_xor_sync(0xffffffffu, mx, w));
+        }
+        if (lane == 31) sm_red[warp] = incl;
+        if (lane == 0) sm_red[kPagedWarps + warp] = mx;
+        __syncthreads();  // also: the ring barriers are initialised
+        int before = incl - sum;
+        int total = 0, max_row = 0;
+#pragma unroll
+        for (int w = 0; w < kPagedWarps; ++w) {
+            if (w < warp) before += sm_red[w];
+            total += sm_red[w];
+            max_row = max(max_row, sm_red[kPagedWarps + w]);
+        }
+        if (threadIdx.x == 0) sm_pre[0] = 0;
+        for (int s2 = s_lo; s2 < s_hi; ++s2) {
+            before += paged_chunks(p, s2);
+            sm_pre[s2 + 1] = before;
+        }
+        __syncthreads();
+        const long long n = static_cast<long long>(total) * p.H_kv;
+        bal_q = paged_quota(n, max_row, static_cast<int>(gridDim.x));
+        bal_i = static_cast<long long>(blockIdx.x) * bal_q;
+        bal_hi = min(n, bal_i + bal_q);
+        if (bal_i >= n) return;
+        // the sequence that holds chunk number bal_i: the last s with H_kv * pre[s] <= bal_i
+        int lo = 0, hi = S;  // invariant: H_kv * pre[lo] <= bal_i < H_kv * pre[hi]
+        while (hi - lo > 1) {
+            const int mid = (lo + hi) >> 1;
+            if (static_cast<long long>(sm_pre[mid]) * p.H_kv <= bal_i) lo = mid; else hi = mid;
+        }
+        seg_s = lo;
+        seg_kvh = 0; seg_tok_begin = 0; seg_tok_end = 0; seg_slot = 0;  // set by next_segment below
+    }
+    // balanced: the segment that starts at chunk number bal_i (inside sequence seg_s); false when the CTA is done
+    auto next_segment = [&]() -> bool {
+        if (bal_i >= bal_hi) return false;
+        while (static_cast<long long>(sm_pre[seg_s + 1]) * p.H_kv <= bal_i) ++seg_s;  // skips empty sequences too
+        const int n_s = sm_pre[seg_s + 1] - sm_pre[seg_s];
+        const long long r = bal_i - static_cast<long long>(sm_pre[seg_s]) * p.H_kv;
+        seg_kvh = static_cast<int>(r / n_s);
+        const int ch0 = static_cast<int>(r % n_s);
+        const int ch1 = static_cast<int>(min(static_cast<long long>(n_s), ch0 + (bal_hi - bal_i)));
+        const int len = max(0, min(p.seq_lens[seg_s], p.max_blocks * BS));
+        seg_tok_begin = ch0 * kPagedChunkTokens;
+        seg_tok_end = min(len, ch1 * kPagedChunkTokens);
+        const long long row_start = bal_i - ch0;
+        seg_slot = static_cast<int>(blockIdx.x - row_start / bal_q);
+        bal_i += ch1 - ch0;
+        return true;
+    };
+    if (p.balanced && !next_segment()) return;
+
+    uint32_t kbase = 0;        // units this warp has been through so far (the ring stage follows it)
+    uint32_t ring_parity = 0;  // bit st: parity of the next completion of stage st's barrier
+    bool ok = true;
+    for (;;) {
+    // =============================== one segment ===============================
+    const int s = seg_s, kvh = seg_kvh, tok_begin = seg_tok_begin, tok_end = seg_tok_end;
     const int head0 = kvh * G;
-    const int len = max(0, min(p.seq_lens[s], p.max_blocks * BS));
-    const int nblk = (len + BS - 1) / BS;
-    const int b0 = sp * p.blocks_per_split;
-    const int b1 = min(nblk, b0 + p.blocks_per_split);
-    if (p.splits > 1 && b0 >= nblk && !(sp == 0)) return;
-    const int tok_begin = b0 * BS;                     // a multiple of 16 (the host keeps blocks_per_split even for BS = 8)
-    const int tok_end = min(len, b1 * BS);
+    const int b1 = (tok_end + BS - 1) / BS;  // cache blocks of the sequence this segment may touch end here
 
     // Q as A fragments: rows g < G hold head head0 + g, the others are zero
     uint32_t qa[PP][4];
@@ -390,29 +513,10 @@ paged_decode_mma_kernel(const PagedParams p) {
     const int* table = p.block_table + static_cast<int64_t>(s) * p.max_blocks;
     const int64_t head_off = static_cast<int64_t>(kvh) * BS * D;
     const int64_t blk_stride = static_cast<int64_t>(p.H_kv) * BS * D;
-    constexpr int NB = BS >= 16 ? 1 : 16 / BS;  // cache blocks per unit of 16 tokens
 
     struct Unit {  // the K and V registers of one unit of 16 tokens
         uint4 kr[2][PP], vr[HV][4];
     };
-    // K and V travel global -> shared by bulk copies (the TMA engine: no address generation, no load/store-unit
-    // queue entries in the SM; with per-lane 16-byte cp.async the same ring streamed 4.3-4.6 TB/s at best), one copy
-    // per tensor and cache block (a unit of 16 tokens is one block, half a block, or two blocks).  Each warp has its
-    // own ring of kPagedRing units and one mbarrier per ring stage.
-    constexpr int kPitch = PagedRow<D>::kPitch;
-    constexpr int kUnitBytes = 32 * kPitch;
-    extern __shared__ uint8_t paged_ring_raw[];
-    uint8_t* ring_base = reinterpret_cast<uint8_t*>((reinterpret_cast<uintptr_t>(paged_ring_raw) + 127) & ~uintptr_t(127));
-    uint8_t* my_ring = ring_base + static_cast<size_t>(warp) * kPagedRing * kUnitBytes;
-    __shared__ uint64_t ring_bar[kPagedWarps][kPagedRing];
-    __shared__ uint32_t ring_abort;
-    if (lane == 0) {
-#pragma unroll
-        for (int i = 0; i < kPagedRing; ++i) mbar_init(&ring_bar[warp][i], 1);
-        if (warp == 0) ring_abort = 0;
-        fence_mbar_init();
-    }
-    __syncthreads();
     // Unit k of this warp starts at token first + k * kStep.  The table entries of 32 units at a time are read by
     // one coalesced load (lane i: unit tab_base + i) and handed out by shuffles: a table load in every unit's path
     // would put a second memory latency in front of its K/V loads.
@@ -542,27 +646,30 @@ paged_decode_mma_kernel(const PagedParams p) {
             }
         }
     };
-    // Stage k % kPagedRing holds unit k; its barrier completes once per use, so the parity to wait for is that of
-    // (k / kPagedRing).
+    // Unit k of the segment is the warp's unit kbase + k and uses ring stage (kbase + k) % kPagedRing.  A stage's
+    // barrier completes once per use; a unit that is left out (bad table entry) does not use its stage, so the parity
+    // to wait for is kept per stage (ring_parity) and flips with every wait.
     uint32_t usable = 0;  // bit (k % 32): unit k may be used
-    bool ok = true;
 #pragma unroll
     for (int k = 0; k < kPagedRing - 1; ++k)
-        if (k < n_units && issue_unit(k, k)) usable |= 1u << k;
+        if (k < n_units && issue_unit((kbase + k) % kPagedRing, k)) usable |= 1u << k;
     for (int k = 0; k < n_units && ok; ++k) {
         const int kk = k + kPagedRing - 1;
         if (kk < n_units) {
-            if (issue_unit(kk % kPagedRing, kk)) usable |= 1u << (kk & 31);
+            if (issue_unit((kbase + kk) % kPagedRing, kk)) usable |= 1u << (kk & 31);
             else usable &= ~(1u << (kk & 31));
         }
         if (usable & (1u << (k & 31))) {
-            ok = __all_sync(0xffffffffu, mbar_wait(&ring_bar[warp][k % kPagedRing], (k / kPagedRing) & 1, &ring_abort, 0x500 + warp)) != 0;
+            const uint32_t st = (kbase + k) % kPagedRing;
+            ok = __all_sync(0xffffffffu, mbar_wait(&ring_bar[warp][st], (ring_parity >> st) & 1, &ring_abort, 0x500 + warp)) != 0;
             if (!ok) break;
+            ring_parity ^= 1u << st;
             Unit un;
-            fetch_unit(un, k % kPagedRing);
+            fetch_unit(un, st);
             compute_unit(un, first + k * kStep);
         }
     }
+    kbase += n_units;
 
     // The warps' partial outputs go where the ring was (every warp's copies have landed and been read by now).
     __syncthreads();
@@ -600,10 +707,14 @@ paged_decode_mma_kernel(const PagedParams p) {
             p.O[row * D + d] = __float2bfloat16(lt > 0.0f ? ot / lt : 0.0f);
             if (d == 0 && p.LSE) p.LSE[row] = lt > 0.0f ? (mt + log2f(lt)) * 0.6931471805599453f : -INFINITY;
         } else {
-            p.part_o[(row * p.splits + sp) * D + d] = ot;
-            if (d == 0) p.part_ml[row * p.splits + sp] = make_float2(mt, lt);
+            p.part_o[(row * p.splits + seg_slot) * D + d] = ot;
+            if (d == 0) p.part_ml[row * p.splits + seg_slot] = make_float2(mt, lt);
         }
     }
+    if (!p.balanced || !ok) break;
+    __syncthreads();  // the partials have left shared memory: the ring may be filled again
+    if (!next_segment()) break;
+    }  // segments
 }
 
 // O[row] = sum over splits of the partials, rescaled to the common max; one CTA of D threads per (seq, head).
@@ -616,12 +727,46 @@ paged_combine_kernel(const PagedParams p) {
     __shared__ float sm_stat[2];             // common max, total l
     const int64_t row = blockIdx.x;
     const int d = threadIdx.x;
-    const int len = max(0, min(p.seq_lens[row / p.H], p.max_blocks * p.block_size));  // as in the decode kernel
-    const int nblk = (len + p.block_size - 1) / p.block_size;
-    const int used = max(1, min(p.splits, (nblk + p.blocks_per_split - 1) / p.blocks_per_split));  // splits that wrote
+    int used;  // partials the decode kernel wrote for this row
+    if (!p.balanced) {
+        const int len = max(0, min(p.seq_lens[row / p.H], p.max_blocks * p.block_size));  // as in the decode kernel
+        const int nblk = (len + p.block_size - 1) / p.block_size;
+        used = max(1, min(p.splits, (nblk + p.blocks_per_split - 1) / p.blocks_per_split));
+    } else {
+        // the decode kernel's arithmetic again: chunks before this row's sequence, in all, and the longest row's
+        __shared__ int sm_bal[3][D / 32];
+        const int s = static_cast<int>(row / p.H), kvh = static_cast<int>(row % p.H) / (p.H / p.H_kv);
+        int below = 0, total = 0, mx = 0;
+        for (int s2 = d; s2 < p.num_seqs; s2 += D) {
+            const int c = paged_chunks(p, s2);
+            total += c;
+            mx = max(mx, c);
+            if (s2 < s) below += c;
+        }
+#pragma unroll
+        for (int w = 16; w > 0; w >>= 1) {
+            below += __shfl_xor_sync(0xffffffffu, below, w);
+            total += __shfl_xor_sync(0xffffffffu, total, w);
+            mx = max(mx, __shfl_xor_sync(0xffffffffu, mx, w));
+        }
+        if ((d & 31) == 0) { sm_bal[0][d >> 5] = below; sm_bal[1][d >> 5] = total; sm_bal[2][d >> 5] = mx; }
+        __syncthreads();
+        below = total = mx = 0;
+#pragma unroll
+        for (int w = 0; w < D / 32; ++w) { below += sm_bal[0][w]; total += sm_bal[1][w]; mx = max(mx, sm_bal[2][w]); }
+        const int n_s = paged_chunks(p, s);
+        const int q = paged_quota(static_cast<long long>(total) * p.H_kv, mx, p.balanced_ctas);
+        const long long row_start = static_cast<long long>(below) * p.H_kv + static_cast<long long>(kvh) * n_s;
+        used = n_s > 0 ? static_cast<int>((row_start + n_s - 1) / q - row_start / q + 1) : 0;
+    }
     // Launched with programmatic stream serialisation: the CTAs may start while the decode kernel is still
     // running (which hides this kernel's launch latency) and wait here until all of its writes are visible.
     cudaGridDependencySynchronize();
+    // the first 8 partial outputs are requested before the weights are known: one memory latency instead of two
+    const float* po = p.part_o + row * p.splits * D + d;
+    float v0[8];
+#pragma unroll
+    for (int i = 0; i < 8; ++i) v0[i] = i < used ? po[i * D] : 0.0f;
     if (d < 32) {
         const float2 ml = d < used ? p.part_ml[row * p.splits + d] : make_float2(-INFINITY, 0.0f);
         float mt = ml.x;
@@ -638,9 +783,10 @@ paged_combine_kernel(const PagedParams p) {
         }
     }
     __syncthreads();
-    const float* po = p.part_o + row * p.splits * D + d;
     float ot = 0.0f;
-    int sp = 0;
+#pragma unroll
+    for (int i = 0; i < 8; ++i) ot = fmaf(v0[i], sm_w[i], ot);  // slots beyond `used` have weight 0
+    int sp = 8;
     for (; sp + 8 <= used; sp += 8) {
         float v[8];
 #pragma unroll
@@ -672,6 +818,21 @@ inline int paged_choose_splits(int num_seqs, int H_kv, int group, int max_blocks
     return std::max(1, std::min(splits, kPagedMaxSplits));
 }
 
+// Equal work per CTA is used by the grouped-head kernel whenever it would split sequences at all (and the
+// sequences fit the scan's table): one CTA per slot the kernel can occupy, or fewer if there is not that much work.
+inline bool paged_use_balanced(const PagedParams& p, int sm_count) {
+    (void)sm_count;
+    const int group = p.H / p.H_kv;
+    return group >= 4 && p.splits > 1 && p.num_seqs <= kPagedBalanceMaxSeqs;
+}
+inline void paged_set_balanced(PagedParams* p, int sm_count) {
+    const long long max_chunks = static_cast<long long>(p->num_seqs) * p->H_kv *
+                                 ((static_cast<long long>(p->max_blocks) * p->block_size + kPagedChunkTokens - 1) / kPagedChunkTokens);
+    p->balanced = 1;
+    p->balanced_ctas = static_cast<int>(std::max<long long>(1, std::min<long long>(static_cast<long long>(kPagedMmaCtasPerSm) * sm_count, max_chunks)));
+    p->splits = kPagedMaxSplits;  // partial slots per row
+}
+
 // KV blocks per CTA of a split sequence.  The grouped-head kernel works in units of 16 tokens, so with 8-token
 // blocks every CTA starts at an even block.
 inline int paged_blocks_per_split(int max_blocks, int splits, int block_size, int group) {
@@ -682,7 +843,8 @@ inline int paged_blocks_per_split(int max_blocks, int splits, int block_size, in
 
 template <int D, int G>
 int paged_launch_bs(const PagedParams& p, cudaStream_t st) {
-    const dim3 grid(p.splits, p.H_kv * p.head_groups, p.num_seqs);
+    dim3 grid(p.splits, p.H_kv * p.head_groups, p.num_seqs);
+    if (p.balanced) grid = dim3(p.balanced_ctas);
     if constexpr (G >= 4) {  // grouped heads: rows of a tensor-core MMA
         constexpr size_t smem = paged_mma_smem_bytes<D>();
         switch (p.block_size) {
