@@ -96,6 +96,42 @@ def test_any_workspace_size_gives_the_same_answer(workspace_bytes):
     check_mha(o, lse, o_ref.reshape(-1, D), l_ref.reshape(-1), f"workspace {workspace_bytes}")
 
 
+@pytest.mark.parametrize("workspace_bytes", [0, 20000, None])
+def test_grouped_heads_any_workspace_size(workspace_bytes):
+    # 8 query heads per KV head: with the full workspace the CTAs get equal shares of the live tokens, with less the
+    # sequences are cut into as many fixed pieces as the scratch allows, with none there is one CTA per sequence and head
+    S, H, Hkv, D, bs = 3, 16, 2, 128, 16
+    Q, Kc, Vc, table, lens = inputs.paged_inputs(S, H, Hkv, D, bs, seed=315, min_len=700, max_len=2100)
+    scale = np.float32(1 / math.sqrt(D))
+    o, lse = run_paged(Q, Kc, Vc, table, lens, scale, workspace_bytes=workspace_bytes)
+    o_ref, l_ref = oracle.paged_attn_decode(Q, Kc, Vc, table, lens, scale=scale)
+    check_mha(o, lse, o_ref.reshape(-1, D), l_ref.reshape(-1), f"grouped heads, workspace {workspace_bytes}")
+
+
+def test_grouped_heads_empty_short_and_long_sequences_together():
+    # equal shares of work per CTA: rows without any token, rows shorter than a chunk, and one row much longer
+    # than all others together (it bounds the share size: no row may need more than 32 partial results)
+    S, H, Hkv, D, bs = 9, 16, 2, 64, 16
+    Q, Kc, Vc, table, _ = inputs.paged_inputs(S, H, Hkv, D, bs, seed=316, min_len=9000, max_len=9000)
+    lens = np.array([0, 1, 9000, 0, 17, 300, 128, 129, 0], dtype=np.int32)
+    o, lse = run_paged(Q, Kc, Vc, table, lens, 0.125)
+    o_ref, l_ref = oracle.paged_attn_decode(Q, Kc, Vc, table, lens, scale=0.125)
+    o = o.reshape(S, H, D); lse = lse.reshape(S, H)
+    for s_ in (0, 3, 8):
+        assert (o[s_] == 0).all() and np.isneginf(lse[s_]).all()
+    live = lens > 0
+    check_mha(o[live].reshape(-1, D), lse[live].reshape(-1), o_ref[live].reshape(-1, D), l_ref[live].reshape(-1), "mixed rows")
+
+
+def test_grouped_heads_more_sequences_than_the_balancing_table():
+    # beyond 1024 sequences the grouped-head kernel falls back to fixed pieces per sequence
+    S, H, Hkv, D, bs = 1100, 8, 2, 64, 16
+    Q, Kc, Vc, table, lens = inputs.paged_inputs(S, H, Hkv, D, bs, seed=317, min_len=1, max_len=1100)
+    o, lse = run_paged(Q, Kc, Vc, table, lens, 0.125)
+    o_ref, l_ref = oracle.paged_attn_decode(Q, Kc, Vc, table, lens, scale=0.125)
+    check_mha(o, lse, o_ref.reshape(-1, D), l_ref.reshape(-1), "1100 sequences")
+
+
 def test_empty_and_single_token_sequences():
     S, H, D, bs = 4, 2, 64, 16
     Q, Kc, Vc, table, lens = inputs.paged_inputs(S, H, H, D, bs, seed=311, min_len=40, max_len=40)
@@ -134,6 +170,30 @@ def test_bad_block_table_entry_is_reported_not_dereferenced():
     status, detail = mlt.last_device_error()
     assert status == 7 and detail[0] == 7 and detail[1] == 2 and detail[2] == 0
     assert mlt.last_device_error()[0] == 0      # cleared
+
+
+def test_bad_entry_with_grouped_heads_leaves_the_pipeline_in_step():
+    # the tensor-core kernel leaves out the 16-token unit of a bad entry; its shared-memory ring must stay in step
+    # (a wrong barrier parity would show as a timeout), and the next call must be clean
+    S, H, Hkv, D, bs = 2, 8, 2, 128, 16
+    Q, Kc, Vc, table, lens = inputs.paged_inputs(S, H, Hkv, D, bs, seed=318, min_len=1500, max_len=1500)
+    bad = table.copy(); bad[1, 5] = -7; bad[0, 40] = Kc.shape[0]
+    o, _ = None, None
+    dQ, dK, dV = to_dev(Q), to_dev(Kc), to_dev(Vc)
+    dL = torch.from_numpy(lens).cuda()
+    O = torch.empty(S * H * D, dtype=torch.int16, device="cuda")
+    ws = torch.empty(mlt.paged_attn_workspace_bytes(S, H, D), dtype=torch.uint8, device="cuda")
+    for tab, want in ((bad, 7), (table, 0)):
+        dT = torch.from_numpy(tab).cuda()
+        rc = mlt.paged_attn_decode_raw(dQ.data_ptr(), dK.data_ptr(), dV.data_ptr(), dT.data_ptr(), dL.data_ptr(), O.data_ptr(),
+                                       0, S, H, Hkv, D, bs, tab.shape[1], Kc.shape[0], 0.09, ws.data_ptr(), ws.numel())
+        assert rc == 0
+        status, detail = mlt.last_device_error()
+        assert status == want, (status, detail)
+        assert torch.isfinite(O.view(torch.bfloat16).float()).all()
+    o_ref, _ = oracle.paged_attn_decode(Q, Kc, Vc, table, lens, scale=0.09)
+    got = inputs.bf16_bits_to_f64(O.cpu().numpy().view(np.uint16)).reshape(-1, D)
+    check_mha(got, np.zeros(0), o_ref.reshape(-1, D), np.zeros(0), "after a bad entry")
 
 
 def test_deterministic_across_runs():
