@@ -285,6 +285,9 @@ def run_mlt(args):
     ms_total = t_begin.elapsed_time(t_end)
     gemm_ms = [e[0].elapsed_time(e[1]) for e in ev]
     mha_ms = [e[1].elapsed_time(e[2]) for e in ev]
+    # the SM clock the last GEMM / attention launch of the timed region really ran at (cycle counter over ns timer
+    # inside the kernels; NVML's figure does not show this part's power management)
+    kernel_mhz = {"gemm": mlt.last_clock_mhz(0), "mha_fwd": mlt.last_clock_mhz(1)}
     rc, detail = mlt.last_device_error()
     if rc:
         raise mlt.MltError(rc, f"device status {detail}")
@@ -400,7 +403,7 @@ def run_mlt(args):
             "config": {"workload": WORKLOAD, "gemm": {"M": M, "N": N, "K": K}, "mha": {"B": Bn, "H": H, "Nq": Nq, "Nk": Nk,
                        "D": D, "causal": bool(causal)}, "l2": "inputs larger than L2 (302 MB GEMM operands; the GEMM's 772 MB stream evicts Q/K/V between steps)",
                        "flop_convention": "2MNK; 4*B*H*Nq*Nk*D halved when causal", "parallelism": f"replicas x{world}"},
-            "clocks": clocks.summary(),
+            "clocks": {**clocks.summary(), "sm_mhz_in_kernel": kernel_mhz},
             "e2e": {"value": e2e_value, "unit": UNIT, "h2d_bytes_per_step": h2d, "d2h_bytes_per_step": d2h,
                     "ms_per_step": e2e_max / e2e_steps, "steps": e2e_steps,
                     "overlap": "upload of step i, kernels of step i-1 and download of step i-2 on three streams, "
@@ -468,7 +471,8 @@ def time_all_configs(mlt, torch, dev, stream, iters: int = 20, only: str | None 
         tmin, tmed = float(np.min(times)), float(np.median(times))
         return {"ms_min": tmin, "ms_median": tmed, "tflops_best": flop / tmin / 1e9, "tflops_median": flop / tmed / 1e9,
                 "frac_of_2250_best": flop / tmin / 1e9 / NOMINAL_BF16_TFLOPS, "launches": iters,
-                "clocks": {"sm_mhz": ck["sm_mhz"], "samples": ck["samples"], "reasons": ck["reasons"]}}
+                "clocks": {"sm_mhz": ck["sm_mhz"], "samples": ck["samples"], "reasons": ck["reasons"],
+                           "sm_mhz_in_kernel": {"gemm": mlt.last_clock_mhz(0), "mha_fwd": mlt.last_clock_mhz(1)}}}
 
     for name, (M, N, K, kind, seed) in inputs.GEMM_CONFIGS.items():
         if only is not None and name != only:

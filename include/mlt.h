@@ -172,6 +172,15 @@ int mlt_paged_attn_decode_static(const void* Q, const void* K_cache, const void*
                                  void* stream);
 
 /*
+ * The SM clock the last GEMM (which = 0) or attention (which = 1) launch on the current device really ran at, in
+ * MHz: CTA 0 of those kernels notes the SM cycle counter and the nanosecond timer at its start and at its end.  (No
+ * counterpart in the paper; a measurement aid: under tensor-core load this part runs well below the clock NVML
+ * reports, and throughput is only comparable across runs together with it.)  Synchronises the device.  *mhz is 0
+ * if no such kernel has run yet.  Concurrent launches of the same kind overwrite each other's notes.
+ */
+int mlt_debug_last_clock_mhz(int which, double* mhz);
+
+/*
  * Device-side health word.  Kernels never trap: a wait that exceeds its bound
  * records {code, barrier id, block} in a per-device status word and the kernel
  * drains and returns.  This call synchronises the current device, reads and

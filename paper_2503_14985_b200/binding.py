@@ -20,7 +20,8 @@ PAGED_STATIC_SCRATCH_BYTES = 16 * 1024 * 1024
 
 EXPORTS = ("mlt_gemm", "mlt_gemm_f16", "mlt_gemm_ex", "mlt_gemm_workspace_bytes", "mlt_mha_fwd", "mlt_paged_attn_decode", "mlt_paged_attn_decode_static",
            "mlt_paged_attn_workspace_bytes",
-           "mlt_last_device_error", "mlt_debug_wait_timeout_selftest", "mlt_status_string", "mlt_version")
+           "mlt_last_device_error", "mlt_debug_wait_timeout_selftest", "mlt_debug_last_clock_mhz", "mlt_status_string",
+           "mlt_version")
 
 _lib = None
 
@@ -43,6 +44,8 @@ def load() -> ctypes.CDLL:
         lib.mlt_gemm.restype = i32
         lib.mlt_debug_wait_timeout_selftest.argtypes = [ctypes.c_uint64, p]
         lib.mlt_debug_wait_timeout_selftest.restype = i32
+        lib.mlt_debug_last_clock_mhz.argtypes = [i32, ctypes.POINTER(ctypes.c_double)]
+        lib.mlt_debug_last_clock_mhz.restype = i32
         lib.mlt_gemm_f16.argtypes = [p, p, p, i64, i64, i64, i64, i64, i64, i32, p]
         lib.mlt_gemm_f16.restype = i32
         lib.mlt_gemm_ex.argtypes = [p, p, p, i64, i64, i64, i64, i64, i64, p, ctypes.c_size_t, p]
@@ -134,6 +137,15 @@ def last_device_error():
     detail = (ctypes.c_uint32 * 4)()
     rc = int(load().mlt_last_device_error(ctypes.cast(detail, ctypes.c_void_p)))
     return rc, list(detail)
+
+
+def last_clock_mhz(which: int) -> float:
+    """SM clock in MHz that the last GEMM (which = 0) or attention (which = 1) launch ran at; 0.0 if none has run."""
+    mhz = ctypes.c_double(0.0)
+    rc = int(load().mlt_debug_last_clock_mhz(which, ctypes.byref(mhz)))
+    if rc != MLT_OK:
+        raise MltError(rc, "mlt_debug_last_clock_mhz")
+    return float(mhz.value)
 
 
 def _stream(stream) -> int:

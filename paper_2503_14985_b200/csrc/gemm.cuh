@@ -196,6 +196,7 @@ gemm_bf16_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_consta
     volatile uint32_t* abort_flag = tmem_base_slot + 1;
 
     const int warp = threadIdx.x >> 5;
+    if (blockIdx.x == 0 && threadIdx.x == 0) clock_probe(0, 0);
     const int lane = threadIdx.x & 31;
     const int num_items = p.tiles_m * p.tiles_n * p.split_k;
     const int num_kb = (p.K + kGemmBK - 1) / kGemmBK;
@@ -329,6 +330,7 @@ gemm_bf16_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_consta
     // common exit: every role reaches this, also after an aborted wait
     tc_fence_before();
     __syncthreads();
+    if (blockIdx.x == 0 && threadIdx.x == 0) clock_probe(0, 1);
     if (warp == 1) {
         __syncwarp();
         tc_fence_after();
@@ -378,6 +380,7 @@ gemm_bf16_pair_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_c
     volatile uint32_t* abort_flag = tmem_base_slot + 1;
 
     const int warp = threadIdx.x >> 5;
+    if (blockIdx.x == 0 && threadIdx.x == 0) clock_probe(0, 0);
     const int lane = threadIdx.x & 31;
     const uint32_t rank = cluster_ctarank();
     const bool leader = rank == 0;
@@ -516,6 +519,7 @@ gemm_bf16_pair_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_c
     // common exit: no CTA of the pair leaves while its peer may still touch its memory
     tc_fence_before();
     cluster_sync_all();
+    if (blockIdx.x == 0 && threadIdx.x == 0) clock_probe(0, 1);
     if (warp == 1) {
         __syncwarp();
         tc_fence_after();

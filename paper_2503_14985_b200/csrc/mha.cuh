@@ -182,6 +182,7 @@ mha_fwd_kernel(const __grid_constant__ CUtensorMap tmap_q, const __grid_constant
 #endif
     const int warp = ((threadIdx.x >> 5) + MLT_ROLE_SHIFT) % 12;  // role index (see the table above)
     const int lane = threadIdx.x & 31;
+    if (blockIdx.x == 0 && threadIdx.x == 0) clock_probe(1, 0);
 
     // Work items of this CTA: item list position r * gridDim.x + (c or gridDim.x - 1 - c), the direction alternating
     // from round to round, so that with the list sorted by length the CTAs' sums stay within about one item.
@@ -728,6 +729,7 @@ mha_fwd_kernel(const __grid_constant__ CUtensorMap tmap_q, const __grid_constant
     // common exit: every role reaches this, also after an aborted wait
     tc_fence_before();
     __syncthreads();
+    if (blockIdx.x == 0 && threadIdx.x == 0) clock_probe(1, 1);
     if (warp == 8) {
         __syncwarp();
         tc_fence_after();

@@ -193,6 +193,16 @@ int mlt_debug_read_trace(unsigned int* host) {  // development builds only: copi
 }
 #endif
 
+int mlt_debug_last_clock_mhz(int which, double* mhz) {
+    if ((which != 0 && which != 1) || !mhz) return MLT_ERR_INVALID_ARG;
+    if (cudaDeviceSynchronize() != cudaSuccess) return MLT_ERR_CUDA;
+    unsigned long long host[2][4];
+    if (cudaMemcpyFromSymbol(host, g_clock_probe, sizeof host) != cudaSuccess) return MLT_ERR_CUDA;
+    const unsigned long long* h = host[which];
+    *mhz = (h[3] > h[1] && h[2] > h[0]) ? 1000.0 * static_cast<double>(h[2] - h[0]) / static_cast<double>(h[3] - h[1]) : 0.0;
+    return MLT_OK;
+}
+
 int mlt_last_device_error(uint32_t* detail) {
     if (cudaDeviceSynchronize() != cudaSuccess) return MLT_ERR_CUDA;
     unsigned int host[4] = {0, 0, 0, 0};

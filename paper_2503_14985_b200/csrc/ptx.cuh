@@ -20,6 +20,17 @@ namespace mlt {
 // ---------------------------------------------------------------------------
 __device__ unsigned int g_status[4];  // {code, barrier id, block, aux}
 
+// SM clock under load: CTA 0 of the GEMM and attention kernels notes the SM cycle counter and the nanosecond timer
+// when it starts and when it ends (slot 0: GEMM kernels, slot 1: attention), so the host can report the clock the
+// last launch really ran at (NVML's figure does not show the power management on this part).
+__device__ unsigned long long g_clock_probe[2][4];  // {cycles at start, ns at start, cycles at end, ns at end}
+__device__ __forceinline__ void clock_probe(int slot, int which) {
+    unsigned long long ns;
+    asm volatile("mov.u64 %0, %%globaltimer;" : "=l"(ns));
+    g_clock_probe[slot][2 * which] = static_cast<unsigned long long>(clock64());
+    g_clock_probe[slot][2 * which + 1] = ns;
+}
+
 constexpr unsigned int kStatusTimeout = 6;
 constexpr long long kWaitBudgetCycles = 4000000000ll;  // about 2 s at boost clock
 
