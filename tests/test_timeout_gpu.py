@@ -37,3 +37,19 @@ def test_budget_outside_the_range_is_refused_without_a_launch():
     assert mlt.debug_wait_timeout_selftest(0) == 1
     assert mlt.debug_wait_timeout_selftest(2_000_000_000) == 1
     assert mlt.last_device_error()[0] == 0
+
+
+def test_kernels_report_the_clock_they_ran_at():
+    # CTA 0 of the GEMM and attention kernels notes the SM cycle counter and the nanosecond timer at both ends
+    import numpy as np
+    from paper_2503_14985_b200 import inputs
+    A, B = inputs.gemm_inputs(2048, 2048, 2048, seed=3)
+    dA = torch.from_numpy(A.view(np.int16)).cuda().view(torch.bfloat16)
+    dB = torch.from_numpy(B.view(np.int16)).cuda().view(torch.bfloat16)
+    mlt.gemm(dA, dB)
+    q = torch.randn(1, 8, 2048, 128, device="cuda").to(torch.bfloat16)
+    mlt.mha_fwd(q, q, q, causal=True, scale=0.088)
+    for which in (0, 1):
+        mhz = mlt.last_clock_mhz(which)
+        assert 300.0 < mhz < 2500.0, (which, mhz)
+    assert mlt.binding.load().mlt_debug_last_clock_mhz(2, None) == 1
