@@ -445,7 +445,7 @@ def time_all_configs(mlt, torch, dev, stream, iters: int = 20, only: str | None 
 
     flush = torch.empty(256 << 20, dtype=torch.int8, device=dev)
 
-    def timeit(fn, flop, read_flush=False):
+    def timeit(fn, flop, read_flush=False, kind=None):
         torch.cuda.synchronize()
         time.sleep(0.3)  # burst timing: let the power governor recover from the configuration before
         for _ in range(warm):
@@ -472,7 +472,8 @@ def time_all_configs(mlt, torch, dev, stream, iters: int = 20, only: str | None 
         return {"ms_min": tmin, "ms_median": tmed, "tflops_best": flop / tmin / 1e9, "tflops_median": flop / tmed / 1e9,
                 "frac_of_2250_best": flop / tmin / 1e9 / NOMINAL_BF16_TFLOPS, "launches": iters,
                 "clocks": {"sm_mhz": ck["sm_mhz"], "samples": ck["samples"], "reasons": ck["reasons"],
-                           "sm_mhz_in_kernel": {"gemm": mlt.last_clock_mhz(0), "mha_fwd": mlt.last_clock_mhz(1)}}}
+                           # the clock the last timed launch really ran at (kernels that carry the probe)
+                           "sm_mhz_in_kernel": mlt.last_clock_mhz({"gemm": 0, "mha_fwd": 1}[kind]) if kind else None}}
 
     for name, (M, N, K, kind, seed) in inputs.GEMM_CONFIGS.items():
         if only is not None and name != only:
@@ -484,7 +485,7 @@ def time_all_configs(mlt, torch, dev, stream, iters: int = 20, only: str | None 
         def fn():
             rc = mlt.gemm_raw(dA.data_ptr(), dB.data_ptr(), dC.data_ptr(), M, N, K, K, N, N, sp)
             assert rc == 0, rc
-        out[name] = timeit(fn, inputs.gemm_flops(M, N, K))
+        out[name] = timeit(fn, inputs.gemm_flops(M, N, K), kind="gemm")
         del dA, dB, dC
     # the same shapes in the data types of Listing 2 (FP16 operands, FP32 result), plain and as C += A * B
     for base, (M, N, K, kind, seed) in inputs.GEMM_CONFIGS.items():
@@ -501,7 +502,7 @@ def time_all_configs(mlt, torch, dev, stream, iters: int = 20, only: str | None 
             def fn():
                 rc = mlt.gemm_f16_raw(dA.data_ptr(), dB.data_ptr(), dC.data_ptr(), M, N, K, K, N, N, acc, sp)
                 assert rc == 0, rc
-            out[name] = timeit(fn, inputs.gemm_flops(M, N, K))
+            out[name] = timeit(fn, inputs.gemm_flops(M, N, K), kind="gemm")
         del dA, dB, dC
     mha_cache = {}
     for name, (Bn, H, Nq, Nk, D, causal, seed, outl) in inputs.MHA_CONFIGS.items():
@@ -521,7 +522,7 @@ def time_all_configs(mlt, torch, dev, stream, iters: int = 20, only: str | None 
             rc = mlt.mha_fwd_raw(dQ.data_ptr(), dK.data_ptr(), dV.data_ptr(), dO.data_ptr(), dL.data_ptr(), Bn, H, Nq, Nk,
                                  D, causal, sc, sp)
             assert rc == 0, rc
-        out[name] = timeit(fn, inputs.mha_flops(Bn, H, Nq, Nk, D, causal))
+        out[name] = timeit(fn, inputs.mha_flops(Bn, H, Nq, Nk, D, causal), kind="mha_fwd")
         del dO, dL
     mha_cache.clear()
     hbm_peak = measured_peaks()["hbm_gbs"]
@@ -539,7 +540,7 @@ def time_all_configs(mlt, torch, dev, stream, iters: int = 20, only: str | None 
             rc = mlt.gemm_ex_raw(dA.data_ptr(), dB.data_ptr(), dC.data_ptr(), M, N, K, K, N, N, ws.data_ptr(), ws.numel(), sp)
             assert rc == 0, rc
         nbytes = 2.0 * (M * K + K * N + M * N)
-        r = timeit(fn, inputs.gemm_flops(M, N, K), read_flush=True)
+        r = timeit(fn, inputs.gemm_flops(M, N, K), read_flush=True, kind="gemm")
         out[name] = {"ms_min": r["ms_min"], "ms_median": r["ms_median"], "gbs_best": nbytes / r["ms_min"] / 1e6,
                      "gbs_median": nbytes / r["ms_median"] / 1e6, "tflops_best": r["tflops_best"],
                      "frac_of_measured_hbm_best": nbytes / r["ms_min"] / 1e6 / hbm_peak, "launches": r["launches"],
