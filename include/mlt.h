@@ -71,14 +71,17 @@ int mlt_gemm_f16(const void* A, const void* B, float* C,
 /*
  * mlt_gemm with caller-provided scratch, for the memory-bound shapes of paper Sec. 4.1 (next-token prediction:
  * few rows of A against large weight matrices, "large k" and "large n" cases).  Such a problem has too few output
- * tiles to occupy the GPU, so K is cut into slices (split-K): every SM streams a part of B, FP32 partial tiles go
- * to the workspace and a second small kernel sums them in a fixed order and rounds once to BF16.  Same operation,
- * arguments, layouts and errors as mlt_gemm; the result can differ from mlt_gemm's in the last BF16 bit (the FP32
- * partial sums are added in a different order).
+ * tiles to occupy the GPU, so K is cut into slices (split-K) and every SM streams a part of B.  With at most one
+ * 128 x 128 tile per two SMs the slices of a tile run as a thread-block cluster that sums its FP32 partial tiles
+ * through distributed shared memory; this needs no scratch and mlt_gemm does the same.  With more tiles than that
+ * the FP32 partial tiles go to the workspace and a second small kernel sums them.  Either way the sum runs in a
+ * fixed order and is rounded once to BF16.  Same operation, arguments, layouts and errors as mlt_gemm; the result
+ * can differ from an uncut sum in the last BF16 bit (the FP32 partial sums are added in a different order).
  *
  *   workspace        device scratch, 16-byte aligned, or NULL (then this is mlt_gemm)
- *   workspace_bytes  its size; mlt_gemm_workspace_bytes(M, N, K) is always enough (0 when no split would be
- *                    used); with less, fewer slices are used.  Calls that overlap on the GPU must not share it.
+ *   workspace_bytes  its size; mlt_gemm_workspace_bytes(M, N, K) is always enough (0 when K would not be cut; an
+ *                    upper bound that does not depend on the device); with less, fewer slices are used.  Calls
+ *                    that overlap on the GPU must not share it.
  */
 size_t mlt_gemm_workspace_bytes(int64_t M, int64_t N, int64_t K);
 int mlt_gemm_ex(const void* A, const void* B, void* C,
@@ -179,6 +182,17 @@ int mlt_paged_attn_decode_static(const void* Q, const void* K_cache, const void*
  * if no such kernel has run yet.  Concurrent launches of the same kind overwrite each other's notes.
  */
 int mlt_debug_last_clock_mhz(int which, double* mhz);
+
+/*
+ * The launch plan of mlt_gemm / mlt_gemm_ex for an M x N x K problem with BF16 output on a device of sm_count SMs
+ * (host arithmetic only, no CUDA call; no counterpart in the paper; lets tests pin which kernel a shape reaches):
+ *   out4[0]  tile shape: 0 = CTA pairs on 256 x 256 tiles, 1 = 128 x 256 tiles, 2 = 128 x 128 tiles
+ *   out4[1]  K slices through the workspace (1 = none);  workspace_bytes = 0 stands for no workspace
+ *   out4[2]  CTAs per cluster that cut K for one tile (1 = none)
+ *   out4[3]  K blocks of 64 per slice
+ * MLT_ERR_INVALID_ARG for a null pointer, a non-positive size or sm_count < 2.
+ */
+int mlt_debug_gemm_plan(int64_t M, int64_t N, int64_t K, size_t workspace_bytes, int sm_count, int* out4);
 
 /*
  * Device-side health word.  Kernels never trap: a wait that exceeds its bound

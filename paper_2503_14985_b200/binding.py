@@ -20,7 +20,7 @@ PAGED_STATIC_SCRATCH_BYTES = 16 * 1024 * 1024
 
 EXPORTS = ("mlt_gemm", "mlt_gemm_f16", "mlt_gemm_ex", "mlt_gemm_workspace_bytes", "mlt_mha_fwd", "mlt_paged_attn_decode", "mlt_paged_attn_decode_static",
            "mlt_paged_attn_workspace_bytes",
-           "mlt_last_device_error", "mlt_debug_wait_timeout_selftest", "mlt_debug_last_clock_mhz", "mlt_status_string",
+           "mlt_last_device_error", "mlt_debug_wait_timeout_selftest", "mlt_debug_last_clock_mhz", "mlt_debug_gemm_plan", "mlt_status_string",
            "mlt_version")
 
 _lib = None
@@ -46,6 +46,8 @@ def load() -> ctypes.CDLL:
         lib.mlt_debug_wait_timeout_selftest.restype = i32
         lib.mlt_debug_last_clock_mhz.argtypes = [i32, ctypes.POINTER(ctypes.c_double)]
         lib.mlt_debug_last_clock_mhz.restype = i32
+        lib.mlt_debug_gemm_plan.argtypes = [i64, i64, i64, ctypes.c_size_t, i32, ctypes.POINTER(ctypes.c_int)]
+        lib.mlt_debug_gemm_plan.restype = i32
         lib.mlt_gemm_f16.argtypes = [p, p, p, i64, i64, i64, i64, i64, i64, i32, p]
         lib.mlt_gemm_f16.restype = i32
         lib.mlt_gemm_ex.argtypes = [p, p, p, i64, i64, i64, i64, i64, i64, p, ctypes.c_size_t, p]
@@ -146,6 +148,16 @@ def last_clock_mhz(which: int) -> float:
     if rc != MLT_OK:
         raise MltError(rc, "mlt_debug_last_clock_mhz")
     return float(mhz.value)
+
+
+def gemm_plan(M: int, N: int, K: int, workspace_bytes: int = 0, sm_count: int = 148) -> dict:
+    """Launch plan of gemm / gemm_ex for a shape (host arithmetic, no GPU): tile variant, K slices through the
+    workspace, CTAs per K-cutting cluster, K blocks of 64 per slice."""
+    out = (ctypes.c_int * 4)()
+    rc = int(load().mlt_debug_gemm_plan(M, N, K, workspace_bytes, sm_count, out))
+    if rc != MLT_OK:
+        raise MltError(rc, "mlt_debug_gemm_plan")
+    return {"variant": out[0], "split_k": out[1], "cluster": out[2], "kb_per_split": out[3]}
 
 
 def _stream(stream) -> int:

@@ -527,6 +527,186 @@ gemm_bf16_pair_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_c
     }
 }
 
+// ---------------------------------------------------------------------------
+// Split-K inside a thread-block cluster, for skinny problems without caller scratch (paper Sec. 4.1, next-token
+// shapes): the S CTAs of a cluster own one 128 x 128 output tile, CTA r accumulates K slice r in its own tensor
+// memory, writes the FP32 tile into its own shared memory (the pipeline stages are free by then), and after a
+// cluster barrier CTA r sums columns [r * 128 / S, (r + 1) * 128 / S) over all S CTAs' shared memory (plain
+// distributed-shared-memory loads, ascending slice order: deterministic) and stores BF16.  One kernel, no partial
+// tiles in global memory, no second launch.  One tile per cluster.
+// ---------------------------------------------------------------------------
+constexpr int kClusterKPartPitch = 132;  // floats per row of the FP32 tile in shared memory (528 B: conflict-free 16-byte rows)
+
+__device__ __forceinline__ float4 ld_shared_cluster_f32x4(uint32_t cluster_addr) {
+    float4 v;
+    asm volatile("ld.shared::cluster.v4.f32 {%0, %1, %2, %3}, [%4];" : "=f"(v.x), "=f"(v.y), "=f"(v.z), "=f"(v.w) : "r"(cluster_addr));
+    return v;
+}
+__device__ __forceinline__ uint32_t cluster_nctarank() {
+    uint32_t r;
+    asm volatile("mov.u32 %0, %%cluster_nctarank;" : "=r"(r));
+    return r;
+}
+
+template <int kStages>
+__global__ void __launch_bounds__(kGemmThreads, 1)
+gemm_bf16_clusterk_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_constant__ CUtensorMap tmap_b,
+                          const GemmParams p) {
+    constexpr int BN = 128;
+    using L = GemmSmem<BN, kStages>;
+    static_assert(kGemmBM * kClusterKPartPitch * 4 <= kStages * L::kStageBytes, "the FP32 tile fits the pipeline stages");
+    extern __shared__ uint8_t smem_raw[];
+    uint8_t* smem = reinterpret_cast<uint8_t*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~uintptr_t(1023));
+    uint64_t* bars = reinterpret_cast<uint64_t*>(smem + kStages * L::kStageBytes);
+    uint64_t* full = bars;
+    uint64_t* empty = bars + kStages;
+    uint64_t* acc_full = bars + 2 * kStages;
+    uint32_t* tmem_base_slot = reinterpret_cast<uint32_t*>(acc_full + 1);
+    volatile uint32_t* abort_flag = tmem_base_slot + 1;
+
+    const int warp = threadIdx.x >> 5;
+    if (blockIdx.x == 0 && threadIdx.x == 0) clock_probe(0, 0);
+    const int lane = threadIdx.x & 31;
+    const int S = static_cast<int>(cluster_nctarank());
+    const int slice = static_cast<int>(cluster_ctarank());
+    const int tile = static_cast<int>(blockIdx.x) / S;
+    const int num_kb = (p.K + kGemmBK - 1) / kGemmBK;
+    const int kb0 = slice * p.kb_per_split, kb1 = min(num_kb, kb0 + p.kb_per_split);  // no slice is empty (host)
+    int tm, tn;
+    gemm_tile_coords(p, tile, tm, tn);
+    const int m0 = tm * kGemmBM, n0 = tn * BN;
+    constexpr uint32_t kTmemCols = BN;
+
+    if (threadIdx.x == 0) {
+        for (int s = 0; s < kStages; ++s) {
+            mbar_init(&full[s], 1);
+            mbar_init(&empty[s], 1);
+        }
+        mbar_init(acc_full, 1);
+        *abort_flag = 0;
+        fence_mbar_init();
+    }
+    if (warp == 0 && lane == 0) {
+        prefetch_tensormap(&tmap_a);
+        prefetch_tensormap(&tmap_b);
+    }
+    if (warp == 1) {
+        tmem_alloc(tmem_base_slot, kTmemCols);
+        tmem_relinquish();
+    }
+    tc_fence_before();
+    __syncthreads();
+    tc_fence_after();
+    const uint32_t tmem_base = *tmem_base_slot;
+    float* part = reinterpret_cast<float*>(smem);  // [128][kClusterKPartPitch], written after the main loop
+
+    if (warp == 0) {
+        if (lane == 0) {
+            int stage = 0;
+            uint32_t phase = 0;
+            bool ok = true;
+            for (int kb = kb0; kb < kb1 && ok; ++kb) {
+                ok = mbar_wait(&empty[stage], phase ^ 1, abort_flag, 0x100 + stage);
+                if (!ok) break;
+                uint8_t* sa = smem + stage * L::kStageBytes;
+                uint8_t* sb = sa + L::kABytes;
+                mbar_arrive_expect_tx(&full[stage], L::kStageBytes);
+                tma_load_2d(sa, &tmap_a, &full[stage], kb * kGemmBK, m0);
+#pragma unroll
+                for (int c = 0; c < BN / 64; ++c)
+                    tma_load_2d(sb + c * (kGemmBK * 128), &tmap_b, &full[stage], n0 + c * 64, kb * kGemmBK);
+                if (++stage == kStages) { stage = 0; phase ^= 1; }
+            }
+        }
+    } else if (warp == 1) {
+        const bool leader = elect_one();
+        const uint32_t idesc = gemm_idesc(kGemmBM, BN, p.f16_inputs);
+        const uint32_t a_lo0 = sdesc_lo(smem_u32(smem), 16);
+        const uint32_t b_lo0 = sdesc_lo(smem_u32(smem + L::kABytes), kGemmBK * 128);
+        int stage = 0;
+        uint32_t phase = 0;
+        bool ok = true;
+        for (int kb = kb0; kb < kb1; ++kb) {
+            ok = __all_sync(0xffffffffu, mbar_wait(&full[stage], phase, abort_flag, 0x200 + stage));
+            if (!ok) break;
+            tc_fence_after();
+            const uint32_t a_lo = a_lo0 + stage * (L::kStageBytes >> 4);
+            const uint32_t b_lo = b_lo0 + stage * (L::kStageBytes >> 4);
+            if (leader) {
+                umma_ss_lo_dyn(tmem_base, a_lo, b_lo, idesc, kb != kb0);
+#pragma unroll
+                for (int k = 1; k < kGemmBK / 16; ++k)
+                    umma_ss_lo<true>(tmem_base, a_lo + k * (32 >> 4), b_lo + k * (2048 >> 4), idesc);
+                umma_commit(&empty[stage]);
+            }
+            __syncwarp();
+            if (++stage == kStages) { stage = 0; phase ^= 1; }
+        }
+        if (ok && leader) umma_commit(acc_full);
+        __syncwarp();
+    } else {
+        // accumulator -> this CTA's FP32 tile in shared memory; acc_full also says that every UMMA has read its
+        // operands, and the producer issued no load beyond them: the stages are free
+        const int quarter = warp & 3;
+        const int r = quarter * 32 + lane;  // row inside the tile
+        if (__all_sync(0xffffffffu, mbar_wait(acc_full, 0, abort_flag, 0x400))) {
+            tc_fence_after();
+            const uint32_t t_row = tmem_base + (static_cast<uint32_t>(quarter * 32) << 16);
+#pragma unroll 1
+            for (int c = 0; c < BN / 32; ++c) {
+                uint32_t v[32];
+                tmem_ld_32x32b_x32(t_row + c * 32, v);
+                tmem_wait_ld();
+                if (m0 + r < p.M) {
+                    float4* dst = reinterpret_cast<float4*>(part + r * kClusterKPartPitch + c * 32);
+#pragma unroll
+                    for (int q = 0; q < 8; ++q)
+                        dst[q] = make_float4(__uint_as_float(v[q * 4]), __uint_as_float(v[q * 4 + 1]), __uint_as_float(v[q * 4 + 2]),
+                                             __uint_as_float(v[q * 4 + 3]));
+                }
+            }
+        }
+    }
+
+    // every CTA's tile is in its shared memory (or a wait expired there: its rows are then garbage and the status
+    // word says so); sum this CTA's share of the columns over the cluster
+    tc_fence_before();
+    cluster_sync_all();
+    {
+        const int cols = BN / S;  // S in {2, 4, 8}: 64, 32 or 16 columns, in groups of 4
+        const int groups = cols / 4;
+        const int rows = min(kGemmBM, p.M - m0);
+        const uint32_t part_addr = smem_u32(part);
+        for (int idx = threadIdx.x; idx < rows * groups; idx += kGemmThreads) {
+            const int r = idx / groups, c = slice * cols + (idx % groups) * 4;
+            float4 acc = make_float4(0.0f, 0.0f, 0.0f, 0.0f);
+            for (int s2 = 0; s2 < S; ++s2) {
+                const float4 v = ld_shared_cluster_f32x4(map_to_cta(part_addr + (r * kClusterKPartPitch + c) * 4, s2));
+                acc.x += v.x; acc.y += v.y; acc.z += v.z; acc.w += v.w;
+            }
+            const int col = n0 + c;
+            __nv_bfloat16* dst = p.C + static_cast<int64_t>(m0 + r) * p.ldc + col;
+            if (col + 4 <= p.N) {
+                uint2 out;
+                out.x = pack_bf16x2(acc.x, acc.y);
+                out.y = pack_bf16x2(acc.z, acc.w);
+                *reinterpret_cast<uint2*>(dst) = out;
+            } else {
+                const float a[4] = {acc.x, acc.y, acc.z, acc.w};
+                for (int j = 0; j < 4 && col + j < p.N; ++j) dst[j] = __float2bfloat16(a[j]);
+            }
+        }
+    }
+    // common exit: no CTA leaves while a peer may still read its shared memory
+    cluster_sync_all();
+    if (blockIdx.x == 0 && threadIdx.x == 0) clock_probe(0, 1);
+    if (warp == 1) {
+        __syncwarp();
+        tc_fence_after();
+        tmem_dealloc(tmem_base, kTmemCols);
+    }
+}
+
 // Split-K second step: C[i][j] = RNE_bf16(sum over slices of partial[slice][i][j]); 8 columns per thread.
 __global__ void gemm_splitk_reduce_kernel(const float* partial, __nv_bfloat16* C, int64_t ldc, int M, int N, int split_k) {
     const int64_t groups_per_row = (N + 7) / 8;

@@ -68,6 +68,7 @@ int get_device(DeviceInfo* out) {
         if (set_smem(gemm_bf16_kernel<256, 4, false>, GemmSmem<256, 4>::kNoStaging) != MLT_OK ||
             set_smem(gemm_bf16_kernel<128, 6, false>, GemmSmem<128, 6>::kNoStaging) != MLT_OK ||
             set_smem(gemm_bf16_pair_kernel<6, false>, GemmPairSmem<6>::kNoStaging) != MLT_OK ||
+            set_smem(gemm_bf16_clusterk_kernel<6>, GemmSmem<128, 6>::kNoStaging) != MLT_OK ||
             set_smem(gemm_bf16_kernel<256, 4, true>, GemmSmem<256, 4>::kTotal) != MLT_OK ||
             set_smem(gemm_bf16_kernel<128, 6, true>, GemmSmem<128, 6>::kTotal) != MLT_OK ||
             set_smem(gemm_bf16_pair_kernel<6, true>, GemmPairSmem<6>::kTotal) != MLT_OK)
@@ -216,12 +217,112 @@ int mlt_last_device_error(uint32_t* detail) {
     return MLT_OK;
 }
 
-// K slices a skinny problem may be cut into: enough work items for two per SM, at least 4 blocks of 64 per slice
+// K slices a skinny problem may be cut into through scratch: enough work items for two per SM, at least 4 blocks of
+// 64 per slice; none with 512 rows or more (compute-bound: the second launch costs more than the cut saves, measured
+// on 512^3)
 static int gemm_max_split(int64_t M, int64_t N, int64_t K) {
     const int64_t tiles = ((M + 127) / 128) * ((N + 127) / 128);
     const int64_t num_kb = (K + kGemmBK - 1) / kGemmBK;
-    if (tiles >= 1024 || num_kb < 8) return 1;
+    if (tiles >= 1024 || num_kb < 8 || M >= 512) return 1;
     return static_cast<int>(std::min<int64_t>(32, num_kb / 4));
+}
+
+// CTAs per cluster (1, 2, 4 or 8) that cut K for one 128 x 128 tile of a skinny problem: the count that minimises
+// rounds x (K blocks per CTA + fill, drain and the reduction), every slice at least 4 blocks of 64.
+static int gemm_cluster_split(int64_t tiles, int num_kb, int sm_count) {
+    if (tiles * 2 > sm_count) return 1;  // enough tiles to occupy the GPU without cutting K
+    int best_s = 1;
+    int64_t best = (num_kb + 4);
+    for (int S = 2; S <= 8; S *= 2) {
+        if (num_kb / S < 4 || S > sm_count) break;
+        const int kbps = (num_kb + S - 1) / S;
+        if (static_cast<int64_t>(kbps) * (S - 1) >= num_kb) continue;  // an empty slice
+        const int64_t slots = sm_count / S * S;
+        const int64_t rounds = (tiles * S + slots - 1) / slots;
+        const int64_t cost = rounds * (kbps + 10);  // cluster launch, two cluster barriers and the reduction: about 6 blocks more
+        if (cost < best) { best = cost; best_s = S; }
+    }
+    return best_s;
+}
+
+// What gemm_run launches for a problem: the tile shape, and for skinny problems how K is cut.
+struct GemmPlan {
+    int variant;       // 0: CTA pairs on 256 x 256 tiles, 1: 128 x 256 tiles, 2: 128 x 128 tiles
+    int split_k;       // > 1: K slices with FP32 partials in caller scratch, summed by a second kernel
+    int cluster;       // > 1: CTAs per cluster that cut K for one tile and reduce through distributed shared memory
+    int kb_per_split;  // K blocks of 64 per slice (per CTA of a cluster)
+};
+
+static GemmPlan gemm_plan(int64_t M, int64_t N, int64_t K, bool has_workspace, size_t workspace_bytes, bool f32_out,
+                          int sm_count, int forced) {
+    // Tile shape by problem size.  Problems with at least 512 rows are compute-bound: the variant with the least
+    // (waves x work per tile / efficiency) wins, with the measured relative efficiencies 1 : 0.8 : 0.62 of the three
+    // kernels (the smaller tiles are bound by the shared-memory operand path).  Shorter problems stream B once and
+    // are bound by memory: pairs when there is at least one tile per pair of SMs, else 128 x 256 tiles, else (most
+    // SMs would idle) 128 x 128 tiles, which can also be cut along K.
+    const int64_t pair_tiles = ((M + kPairBM - 1) / kPairBM) * ((N + kPairBN - 1) / kPairBN);
+    const int64_t tiles_m128 = (M + kGemmBM - 1) / kGemmBM;
+    const int64_t tiles1 = tiles_m128 * ((N + 255) / 256);
+    const int64_t tiles2 = tiles_m128 * ((N + 127) / 128);
+    const int num_kb = static_cast<int>((K + kGemmBK - 1) / kGemmBK);
+    GemmPlan plan = {2, 1, 1, num_kb};
+    if (M >= 512) {
+        const int64_t pairs = sm_count / 2;
+        const double c0 = static_cast<double>((pair_tiles + pairs - 1) / pairs);
+        const double c1 = static_cast<double>((tiles1 + sm_count - 1) / sm_count) / 0.8;
+        const double c2 = static_cast<double>((tiles2 + sm_count - 1) / sm_count) * 0.5 / 0.62;
+        plan.variant = (c0 <= c1 && c0 <= c2) ? 0 : (c1 <= c2 ? 1 : 2);
+    } else if (!f32_out && (gemm_cluster_split(tiles2, num_kb, sm_count) > 1 ||
+                            (has_workspace && gemm_max_split(M, N, K) > 1))) {
+        plan.variant = 2;  // memory-bound and K can be cut: small tiles spread the stream of B evenly over the SMs
+    } else if (pair_tiles >= sm_count / 2) {
+        plan.variant = 0;
+    } else if (tiles1 >= sm_count) {
+        plan.variant = 1;
+    } else {
+        plan.variant = 2;
+    }
+    if (forced >= 0 && forced <= 2) plan.variant = forced;
+    if (plan.variant != 2 || f32_out) return plan;
+
+    // Few tiles: clusters of S CTAs per tile when at most half the SMs would have a tile (measured equal to or faster
+    // than partial tiles in scratch plus a second kernel, so it is used with or without a workspace) ...
+    plan.cluster = gemm_cluster_split(tiles2, num_kb, sm_count);
+    if (plan.cluster > 1) {
+        plan.kb_per_split = (num_kb + plan.cluster - 1) / plan.cluster;
+        return plan;
+    }
+    if (!has_workspace) return plan;
+    // ... else slices through scratch: the count that minimises rounds x (K blocks per slice + fill/drain of an item)
+    // plus the time to write and re-read the FP32 partials, in units of one K block of one tile (16 KB of B per SM).
+    int max_split = gemm_max_split(M, N, K);
+    while (max_split > 1 && static_cast<size_t>(max_split) * M * N * sizeof(float) > workspace_bytes) --max_split;
+    int split = 1;
+    double best = 1e300;
+    for (int sl = 1; sl <= max_split; ++sl) {
+        const int kbps = (num_kb + sl - 1) / sl;
+        const int slices = (num_kb + kbps - 1) / kbps;
+        if (slices != sl) continue;  // the same slicing as a smaller count
+        const int64_t rounds = (tiles2 * slices + sm_count - 1) / sm_count;
+        const double partial = sl > 1 ? static_cast<double>(sl) * M * N * 8.0 / (16384.0 * sm_count) : 0.0;
+        const double cost = static_cast<double>(rounds) * (kbps + 4) + partial;
+        if (cost < best) { best = cost; split = sl; }
+    }
+    if (split > 1) {
+        plan.kb_per_split = (num_kb + split - 1) / split;
+        plan.split_k = (num_kb + plan.kb_per_split - 1) / plan.kb_per_split;  // no empty slice
+    }
+    return plan;
+}
+
+int mlt_debug_gemm_plan(int64_t M, int64_t N, int64_t K, size_t workspace_bytes, int sm_count, int* out4) {
+    if (!out4 || M <= 0 || N <= 0 || K <= 0 || sm_count < 2) return MLT_ERR_INVALID_ARG;
+    const GemmPlan plan = gemm_plan(M, N, K, workspace_bytes > 0, workspace_bytes, false, sm_count, -1);
+    out4[0] = plan.variant;
+    out4[1] = plan.split_k;
+    out4[2] = plan.cluster;
+    out4[3] = plan.kb_per_split;
+    return MLT_OK;
 }
 
 size_t mlt_gemm_workspace_bytes(int64_t M, int64_t N, int64_t K) {
@@ -262,33 +363,8 @@ static int gemm_run(const void* A, const void* B, void* C, int64_t M, int64_t N,
         return cudaGetLastError() == cudaSuccess ? MLT_OK : MLT_ERR_CUDA;
     }
 
-    // Tile shape by problem size.  0: CTA pairs on 256 x 256 tiles, 1: 128 x 256 tiles, 2: 128 x 128 tiles.
-    // Problems with at least 512 rows are compute-bound: the variant with the least (waves x work per tile /
-    // efficiency) wins, with the measured relative efficiencies 1 : 0.8 : 0.62 of the three kernels (the smaller
-    // tiles are bound by the shared-memory operand path).  Shorter problems stream B once and are bound by memory:
-    // pairs when there is at least one tile per pair of SMs, else 128 x 256 tiles, else (most SMs would idle)
-    // 128 x 128 tiles, which can also be cut along K.
-    const int64_t pair_tiles = ((M + kPairBM - 1) / kPairBM) * ((N + kPairBN - 1) / kPairBN);
-    const int64_t tiles_m128 = (M + kGemmBM - 1) / kGemmBM;
-    const int64_t tiles1 = tiles_m128 * ((N + 255) / 256);
-    const int64_t tiles2 = tiles_m128 * ((N + 127) / 128);
-    int variant;
-    if (M >= 512) {
-        const int64_t pairs = dev.sm_count / 2;
-        const double c0 = static_cast<double>((pair_tiles + pairs - 1) / pairs);
-        const double c1 = static_cast<double>((tiles1 + dev.sm_count - 1) / dev.sm_count) / 0.8;
-        const double c2 = static_cast<double>((tiles2 + dev.sm_count - 1) / dev.sm_count) * 0.5 / 0.62;
-        variant = (c0 <= c1 && c0 <= c2) ? 0 : (c1 <= c2 ? 1 : 2);
-    } else if (workspace && !f32_out && gemm_max_split(M, N, K) > 1) {
-        variant = 2;  // memory-bound with scratch: small tiles cut along K spread the stream of B evenly over the SMs
-    } else if (pair_tiles >= dev.sm_count / 2) {
-        variant = 0;
-    } else if (tiles1 >= dev.sm_count) {
-        variant = 1;
-    } else {
-        variant = 2;
-    }
-    if (forced_variant() >= 0 && forced_variant() <= 2) variant = forced_variant();
+    const GemmPlan plan = gemm_plan(M, N, K, workspace != nullptr, workspace_bytes, f32_out, dev.sm_count, forced_variant());
+    const int variant = plan.variant;
     const int bm = variant == 0 ? kPairBM : kGemmBM;
     const int bn = variant == 2 ? 128 : 256;
     const int64_t tiles_m = (M + bm - 1) / bm;
@@ -338,31 +414,12 @@ static int gemm_run(const void* A, const void* B, void* C, int64_t M, int64_t N,
     p.accumulate = accumulate ? 1 : 0;
     p.f16_inputs = f16_in ? 1u : 0u;
     p.full_items = p.num_items = 0;
-    if (variant == 2 && workspace && !f32_out) {
-        // Few tiles (skinny or small problem): cut K into slices so that about two work items per SM exist; the
-        // weights are then streamed by all SMs at once.  FP32 partials go to the caller's scratch.
-        const int num_kb = p.kb_per_split;
-        // Slices: the count that minimises rounds x (K blocks per slice + fill/drain of an item) plus the time to
-        // write and re-read the FP32 partials, all in units of one K block of one tile (16 KB of B per SM).
-        const int64_t tiles = tiles_m * tiles_n;
-        int max_split = gemm_max_split(M, N, K);
-        while (max_split > 1 && static_cast<size_t>(max_split) * M * N * sizeof(float) > workspace_bytes) --max_split;
-        int split = 1;
-        double best = 1e300;
-        for (int sl = 1; sl <= max_split; ++sl) {
-            const int kbps = (num_kb + sl - 1) / sl;
-            const int slices = (num_kb + kbps - 1) / kbps;
-            if (slices != sl) continue;  // the same slicing as a smaller count
-            const int64_t rounds = (tiles * slices + dev.sm_count - 1) / dev.sm_count;
-            const double partial = sl > 1 ? static_cast<double>(sl) * M * N * 8.0 / (16384.0 * dev.sm_count) : 0.0;
-            const double cost = static_cast<double>(rounds) * (kbps + 4) + partial;
-            if (cost < best) { best = cost; split = sl; }
-        }
-        if (split > 1) {
-            p.kb_per_split = (num_kb + split - 1) / split;
-            p.split_k = (num_kb + p.kb_per_split - 1) / p.kb_per_split;  // no empty slice
-            p.partial = static_cast<float*>(workspace);
-        }
+    const int cluster_s = plan.cluster;
+    if (plan.split_k > 1) {
+        // Few tiles and more than half an SM count of them: K is cut into slices, FP32 partials go to the caller's scratch
+        p.kb_per_split = plan.kb_per_split;
+        p.split_k = plan.split_k;
+        p.partial = static_cast<float*>(workspace);
     }
     if (variant == 0) {
         // M-tiles per raster group: wide problems re-read B once per group, so fewer, taller groups pay
@@ -378,6 +435,26 @@ static int gemm_run(const void* A, const void* B, void* C, int64_t M, int64_t N,
             gemm_bf16_pair_kernel<6, true><<<2 * clusters, kGemmThreads, GemmPairSmem<6>::kTotal, st>>>(ta, tb, tc, p);
         else
             gemm_bf16_pair_kernel<6, false><<<2 * clusters, kGemmThreads, GemmPairSmem<6>::kNoStaging, st>>>(ta, tb, tc, p);
+    } else if (cluster_s > 1) {
+        // Skinny problem with few tiles: K is cut inside clusters of S CTAs per tile, which reduce through
+        // distributed shared memory (gemm_bf16_clusterk_kernel)
+        const int S = cluster_s;
+        p.group_m = 16;
+        p.kb_per_split = plan.kb_per_split;
+        if (static_cast<int64_t>(p.kb_per_split) * (S - 1) >= (K + kGemmBK - 1) / kGemmBK) return MLT_ERR_UNSUPPORTED;  // an empty slice: the plan never makes one
+        cudaLaunchConfig_t cfg = {};
+        cfg.gridDim = dim3(static_cast<unsigned>(tiles_m * tiles_n * S));
+        cfg.blockDim = dim3(kGemmThreads);
+        cfg.dynamicSmemBytes = GemmSmem<128, 6>::kNoStaging;
+        cfg.stream = st;
+        cudaLaunchAttribute attr;
+        attr.id = cudaLaunchAttributeClusterDimension;
+        attr.val.clusterDim.x = static_cast<unsigned>(S);
+        attr.val.clusterDim.y = 1;
+        attr.val.clusterDim.z = 1;
+        cfg.attrs = &attr;
+        cfg.numAttrs = 1;
+        if (cudaLaunchKernelEx(&cfg, gemm_bf16_clusterk_kernel<6>, ta, tb, p) != cudaSuccess) return MLT_ERR_CUDA;
     } else {
         p.group_m = 16;
         const int grid = static_cast<int>(std::min<int64_t>(tiles_m * tiles_n * p.split_k, dev.sm_count));

@@ -1,0 +1,63 @@
+"""Host logic of the GEMM launch plan (no GPU): which tile shape a problem gets and how K is cut for the memory-bound
+shapes of Sec. 4.1.  The plan is plain integer arithmetic behind mlt_debug_gemm_plan."""
+import itertools
+
+import pytest
+
+import paper_2503_14985_b200 as mlt
+
+
+def kb(K):
+    return (K + 63) // 64
+
+
+@pytest.mark.parametrize("sm_count", [148, 132, 64, 2])
+def test_plan_invariants(sm_count):
+    Ms = [1, 16, 100, 130, 511, 512, 2000]
+    Ns = [8, 128, 520, 4096, 9600, 28672]
+    Ks = [8, 64, 520, 2048, 4100, 28672]
+    for M, N, K in itertools.product(Ms, Ns, Ks):
+        need = mlt.gemm_workspace_bytes(M, N, K)
+        for ws in {0, need // 3 // 16 * 16, need}:
+            pl = mlt.gemm_plan(M, N, K, ws, sm_count)
+            what = f"{M}x{N}x{K} ws={ws} sms={sm_count}: {pl}"
+            assert pl["variant"] in (0, 1, 2), what
+            assert pl["cluster"] in (1, 2, 4, 8) and pl["split_k"] >= 1, what
+            assert pl["cluster"] == 1 or pl["split_k"] == 1, what
+            slices = max(pl["cluster"], pl["split_k"])
+            if slices == 1:
+                assert pl["kb_per_split"] == kb(K), what
+                continue
+            assert pl["variant"] == 2, what
+            # every slice has work, the slices cover K, none is shorter than 4 blocks by design of the cut
+            assert pl["kb_per_split"] * (slices - 1) < kb(K) <= pl["kb_per_split"] * slices, what
+            assert kb(K) // slices >= 4, what
+            if pl["split_k"] > 1:
+                assert pl["split_k"] * M * N * 4 <= ws, what
+            else:
+                tiles = ((M + 127) // 128) * ((N + 127) // 128)
+                assert 2 * tiles <= sm_count, what
+
+
+def test_plan_known_cases_on_148_sms():
+    full = lambda M, N, K: mlt.gemm_plan(M, N, K, mlt.gemm_workspace_bytes(M, N, K), 148)
+    assert mlt.gemm_plan(8192, 8192, 8192)["variant"] == 0 and full(8192, 28672, 4096)["variant"] == 0
+    assert full(8192, 8192, 8192)["split_k"] == 1 and full(8192, 8192, 8192)["cluster"] == 1
+    # next-token shapes: 32 tiles -> 4 CTAs per tile; 64 tiles -> 2; 8 tiles -> 8
+    assert full(16, 4096, 4096)["cluster"] == 4 and mlt.gemm_plan(16, 4096, 4096)["cluster"] == 4
+    assert full(16, 4096, 28672)["cluster"] == 4 and full(16, 4096, 28672)["kb_per_split"] == 112
+    assert full(16, 8192, 4096)["cluster"] == 2
+    assert full(16, 1024, 4096)["cluster"] == 8
+    # 224 tiles: clusters would need more than one round; with scratch K goes through the workspace, without it whole
+    assert full(16, 28672, 4096)["cluster"] == 1 and full(16, 28672, 4096)["split_k"] > 1
+    assert mlt.gemm_plan(16, 28672, 4096) == {"variant": 0, "split_k": 1, "cluster": 1, "kb_per_split": 64}
+    # a short K is not cut
+    assert full(16, 4096, 192)["cluster"] == 1 and full(16, 4096, 192)["split_k"] == 1
+    assert full(512, 512, 512)["cluster"] == 1
+
+
+def test_plan_rejects_bad_arguments():
+    with pytest.raises(mlt.MltError):
+        mlt.gemm_plan(0, 8, 8)
+    with pytest.raises(mlt.MltError):
+        mlt.gemm_plan(8, 8, 8, 0, 1)

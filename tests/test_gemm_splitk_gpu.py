@@ -1,4 +1,5 @@
-"""GPU parity of mlt_gemm_ex (split-K with caller scratch, for the memory-bound shapes of Sec. 4.1) against the oracle."""
+"""GPU parity of the K-cutting GEMM paths for the memory-bound shapes of Sec. 4.1 against the oracle: slices through
+caller scratch (mlt_gemm_ex) and slices inside thread-block clusters (no scratch; mlt_gemm and mlt_gemm_ex)."""
 import numpy as np
 import pytest
 
@@ -32,8 +33,13 @@ def run_ex(A, B, M, N, K, ldc, workspace_bytes):
     return inputs.bf16_bits_to_f64(bits[:M, :N]).reshape(M, N)
 
 
+def plan(M, N, K, workspace_bytes=0):
+    return mlt.gemm_plan(M, N, K, workspace_bytes, torch.cuda.get_device_properties(0).multi_processor_count)
+
+
+# the last three have more than one 128 x 128 tile per two SMs: with scratch they take the two-kernel path
 SHAPES = [(1, 4096, 4096), (16, 4096, 4096), (7, 1000, 2056), (64, 520, 8192), (130, 264, 4100), (16, 4096, 520),
-          (512, 512, 512), (33, 6, 1024)]
+          (512, 512, 512), (33, 6, 1024), (16, 9600, 2048), (40, 10008, 2064), (200, 5000, 4100)]
 
 
 @pytest.mark.parametrize("M,N,K", SHAPES)
@@ -45,24 +51,58 @@ def test_parity_skinny_and_ragged(M, N, K):
     check_gemm(C, oracle.gemm(A, B, M, N, K), f"{M}x{N}x{K}")
 
 
+@pytest.mark.parametrize("M,N,K", [(16, 1024, 4096), (16, 9600, 4096)])     # clusters / scratch
 @pytest.mark.parametrize("fraction", [0.0, 0.26, 1.0])
-def test_any_workspace_size_is_correct(fraction):
-    M, N, K = 16, 1024, 4096
+def test_any_workspace_size_is_correct(fraction, M, N, K):
     A, B = inputs.gemm_inputs(M, N, K, seed=510)
     need = mlt.gemm_workspace_bytes(M, N, K)
     assert need == 16 * M * N * 4           # 64 blocks of 64 -> at most 16 slices of 4
-    C = run_ex(A, B, M, N, K, N, int(need * fraction) // 16 * 16)
+    given = int(need * fraction) // 16 * 16
+    if N == 9600:
+        assert plan(M, N, K, need)["split_k"] > 1 and plan(M, N, K, need)["split_k"] * M * N * 4 <= need
+        assert plan(M, N, K, given)["split_k"] * M * N * 4 <= max(given, M * N * 4)
+    C = run_ex(A, B, M, N, K, N, given)
     check_gemm(C, oracle.gemm(A, B, M, N, K), f"fraction {fraction}")
 
 
-def test_bit_exact_on_small_integers_and_deterministic():
-    M, N, K = 24, 776, 2048
+@pytest.mark.parametrize("M,N,K", [(24, 776, 2048), (24, 9736, 2048)])       # clusters / scratch
+def test_bit_exact_on_small_integers_and_deterministic(M, N, K):
     A, B = inputs.gemm_inputs(M, N, K, seed=7, kind="ternary")
     need = mlt.gemm_workspace_bytes(M, N, K)
+    pl = plan(M, N, K, need)
+    assert (pl["cluster"] > 1) if N == 776 else (pl["split_k"] > 1)
     C1 = run_ex(A, B, M, N, K, N, need)
     ref = oracle.gemm(A, B, M, N, K)
     assert np.abs(ref).max() <= 256 and np.array_equal(C1, ref)      # exact partial sums, exact final sum
     assert np.array_equal(C1, run_ex(A, B, M, N, K, N, need))
+
+
+# Clusters of 2, 4 and 8 CTAs per tile (on 148 SMs), ragged M, N and K, one and two tile rows, a last slice shorter
+# than the others, a K tail that is not a whole block; no scratch is given
+CLUSTER_SHAPES = [(16, 8192, 4096, 2), (48, 8000, 4104, 2), (16, 4096, 4096, 4), (5, 2056, 3000, 8),
+                  (16, 1024, 4096, 8), (130, 264, 4100, 8), (256, 520, 2048 + 24, 4), (1, 128, 4096, 8),
+                  (128, 136, 36 * 64, 8)]
+
+
+@pytest.mark.parametrize("M,N,K,S148", CLUSTER_SHAPES)
+def test_cluster_split_parity(M, N, K, S148):
+    pl = plan(M, N, K)
+    assert pl["cluster"] > 1 and pl["split_k"] == 1
+    if torch.cuda.get_device_properties(0).multi_processor_count == 148:
+        assert pl["cluster"] == S148
+    lda, ldb, ldc = (K + 7) // 8 * 8, (N + 7) // 8 * 8 + 8, (N + 7) // 8 * 8 + 16
+    A, B = inputs.gemm_inputs(M, N, K, seed=900 + M + N, kind="uniform", lda=lda, ldb=ldb)
+    C = run_ex(A, B, M, N, K, ldc, 0)
+    ref = oracle.gemm(A, B, M, N, K)
+    check_gemm(C, ref, f"cluster {M}x{N}x{K}")
+    assert np.array_equal(C, run_ex(A, B, M, N, K, ldc, 0))          # fixed summation order
+    # the public entry point without scratch takes the same path and gives the same bits
+    dA, dB = to_dev(A), to_dev(B)
+    out = torch.empty((M, ldc), dtype=torch.bfloat16, device="cuda")
+    rc = mlt.gemm_raw(dA.data_ptr(), dB.data_ptr(), out.data_ptr(), M, N, K, lda, ldb, ldc,
+                      torch.cuda.current_stream().cuda_stream)
+    assert rc == 0
+    assert np.array_equal(inputs.bf16_bits_to_f64(to_bits(out)[:, :N]).reshape(M, N), C)
 
 
 @pytest.mark.parametrize("name", list(inputs.GEMM_DECODE_CONFIGS))
