@@ -184,13 +184,15 @@ int mlt_paged_attn_decode_static(const void* Q, const void* K_cache, const void*
 int mlt_debug_last_clock_mhz(int which, double* mhz);
 
 /*
- * The launch plan of mlt_gemm / mlt_gemm_ex for an M x N x K problem with BF16 output on a device of sm_count SMs
- * (host arithmetic only, no CUDA call; no counterpart in the paper; lets tests pin which kernel a shape reaches):
+ * The launch plan of mlt_gemm / mlt_gemm_ex for an M x N x K problem with BF16 output (no counterpart in the paper;
+ * lets tests pin which kernel a shape reaches).  sm_count >= 2: a device of that many SMs on which clusters can use
+ * every SM (host arithmetic only, no CUDA call).  sm_count == 0: the current device, with the number of resident
+ * clusters it reports (a cluster must fit one GPC); configures the device on first use like any other call.
  *   out4[0]  tile shape: 0 = CTA pairs on 256 x 256 tiles, 1 = 128 x 256 tiles, 2 = 128 x 128 tiles
  *   out4[1]  K slices through the workspace (1 = none);  workspace_bytes = 0 stands for no workspace
  *   out4[2]  CTAs per cluster that cut K for one tile (1 = none)
  *   out4[3]  K blocks of 64 per slice
- * MLT_ERR_INVALID_ARG for a null pointer, a non-positive size or sm_count < 2.
+ * MLT_ERR_INVALID_ARG for a null pointer, a non-positive size, sm_count 1 or negative.
  */
 int mlt_debug_gemm_plan(int64_t M, int64_t N, int64_t K, size_t workspace_bytes, int sm_count, int* out4);
 

@@ -151,8 +151,8 @@ def last_clock_mhz(which: int) -> float:
 
 
 def gemm_plan(M: int, N: int, K: int, workspace_bytes: int = 0, sm_count: int = 148) -> dict:
-    """Launch plan of gemm / gemm_ex for a shape (host arithmetic, no GPU): tile variant, K slices through the
-    workspace, CTAs per K-cutting cluster, K blocks of 64 per slice."""
+    """Launch plan of gemm / gemm_ex for a shape: tile variant, K slices through the workspace, CTAs per K-cutting
+    cluster, K blocks of 64 per slice.  sm_count >= 2: host arithmetic for such a device, no GPU; 0: the current device."""
     out = (ctypes.c_int * 4)()
     rc = int(load().mlt_debug_gemm_plan(M, N, K, workspace_bytes, sm_count, out))
     if rc != MLT_OK:

@@ -29,6 +29,10 @@ constexpr int kGemmThreads = 192;
 // FP32 output goes through shared memory and TMA: two 4 KB boxes (32 rows x 32 FP32 columns) per epilogue warp
 constexpr int kGemmStagingBytes = 4 * 2 * 4096;
 
+// BF16 output of the 128 x 128 kernel: each epilogue warp stages 32 rows x 64 columns (128 bytes per row, pitch 144:
+// the 16-byte row writes of 8 lanes and the 128-byte row reads of 8 lanes both touch every bank once)
+constexpr int kGemmBf16StagePitch = 144;
+
 template <int BN, int kStages>
 struct GemmSmem {
     static constexpr int kABytes = kGemmBM * kGemmBK * 2;  // 16 KB
@@ -38,6 +42,8 @@ struct GemmSmem {
     // stages | barriers (padded to 1 KB) | staging for FP32 output (only requested by launches that write FP32 C)
     static constexpr int kNoStaging = kStages * kStageBytes + 1024 + 1024;  // + alignment slack
     static constexpr int kTotal = kNoStaging + kGemmStagingBytes;
+    // BF16 output of the 128-wide kernel goes through a small staging area (see gemm_store_half_coalesced)
+    static constexpr int kBf16Staging = kNoStaging + 4 * 32 * kGemmBf16StagePitch;
 };
 
 struct GemmParams {
@@ -115,6 +121,34 @@ __device__ __forceinline__ void gemm_store_chunk(const GemmParams& p, const uint
     }
 }
 
+// 32 rows x 64 accumulator columns of one epilogue warp to BF16 C through shared memory: lane = row writes its 128
+// bytes into the staging row, then 8 lanes per row copy 4 rows per instruction to C, so a store instruction covers
+// 4 lines of 128 bytes instead of 32 lines of 16 bytes (the per-row stores of gemm_store_chunk take about 2000
+// clocks per 128 x 128 tile in the load/store unit, which shows when the epilogue is not hidden behind a next tile).
+// Whole tiles only: the caller keeps ragged right edges on the per-row path.
+__device__ __forceinline__ void gemm_store_half_coalesced(const GemmParams& p, uint8_t* stg, const uint32_t (&v)[2][32],
+                                                          int lane, int row0, int col0) {
+    uint4* mine = reinterpret_cast<uint4*>(stg + lane * kGemmBf16StagePitch);
+#pragma unroll
+    for (int q = 0; q < 8; ++q) {
+        const uint32_t* w = &v[q >> 2][(q & 3) * 8];
+        mine[q] = make_uint4(pack_bf16x2(__uint_as_float(w[0]), __uint_as_float(w[1])),
+                             pack_bf16x2(__uint_as_float(w[2]), __uint_as_float(w[3])),
+                             pack_bf16x2(__uint_as_float(w[4]), __uint_as_float(w[5])),
+                             pack_bf16x2(__uint_as_float(w[6]), __uint_as_float(w[7])));
+    }
+    __syncwarp();
+    const int sub = lane >> 3, unit = lane & 7;
+#pragma unroll
+    for (int i = 0; i < 8; ++i) {
+        const int r = i * 4 + sub;
+        const uint4 x = *reinterpret_cast<const uint4*>(stg + r * kGemmBf16StagePitch + unit * 16);
+        if (row0 + r < p.M)
+            *reinterpret_cast<uint4*>(p.C + static_cast<int64_t>(row0 + r) * p.ldc + col0 + unit * 8) = x;
+    }
+    __syncwarp();  // the staging rows are rewritten by the next call
+}
+
 // The same segment for a whole warp when C is FP32 and reached through a tensor map (p.c_tma): the warp's 32 rows
 // x 32 columns go into a 4 KB staging box (128-byte rows, 16-byte chunk k of row r at chunk k ^ (r & 7): the
 // 128-byte swizzle of the map) and one lane issues a TMA store, or a TMA add-reduction for C += A * B, which adds
@@ -178,6 +212,16 @@ __device__ __forceinline__ void gemm_tile_coords(const GemmParams& p, int tile, 
     tn = r / rows;
 }
 
+#ifdef MLT_TRACE
+// development builds: SM clock at a few points of CTA 0 of gemm_bf16_kernel
+__device__ long long g_gemm_trace[16];
+#define MLT_GT(i) do { if (blockIdx.x == 0 && (threadIdx.x & 31) == 0) g_gemm_trace[i] = clock64(); } while (0)
+#define MLT_GT_NS(i) do { if (blockIdx.x == 0 && threadIdx.x == 0) { unsigned long long ns_; asm volatile("mov.u64 %0, %%globaltimer;" : "=l"(ns_)); g_gemm_trace[i] = static_cast<long long>(ns_); } } while (0)
+#else
+#define MLT_GT_NS(i) do { } while (0)
+#define MLT_GT(i) do { } while (0)
+#endif
+
 template <int BN, int kStages, bool kCTma>
 __global__ void __launch_bounds__(kGemmThreads, 1)
 gemm_bf16_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_constant__ CUtensorMap tmap_b,
@@ -197,6 +241,8 @@ gemm_bf16_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_consta
 
     const int warp = threadIdx.x >> 5;
     if (blockIdx.x == 0 && threadIdx.x == 0) clock_probe(0, 0);
+    if (threadIdx.x == 0) MLT_GT(0);
+    MLT_GT_NS(6);
     const int lane = threadIdx.x & 31;
     const int num_items = p.tiles_m * p.tiles_n * p.split_k;
     const int num_kb = (p.K + kGemmBK - 1) / kGemmBK;
@@ -226,6 +272,7 @@ gemm_bf16_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_consta
     __syncthreads();
     tc_fence_after();
     const uint32_t tmem_base = *tmem_base_slot;
+    if (threadIdx.x == 0) MLT_GT(1);
 
     if (warp == 0) {
         // ----------------------------- producer -----------------------------
@@ -275,6 +322,7 @@ gemm_bf16_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_consta
                 for (int kb = kb0; kb < kb1; ++kb) {
                     ok = __all_sync(0xffffffffu, mbar_wait(&full[stage], phase, abort_flag, 0x200 + stage));
                     if (!ok) break;
+                    if (kb == kb0) MLT_GT(2);
                     tc_fence_after();
                     const uint32_t a_lo = a_lo0 + stage * (L::kStageBytes >> 4);
                     const uint32_t b_lo = b_lo0 + stage * (L::kStageBytes >> 4);
@@ -289,6 +337,7 @@ gemm_bf16_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_consta
                     if (++stage == kStages) { stage = 0; phase ^= 1; }
                 }
                 if (ok && leader) umma_commit(&acc_full[acc]);
+                MLT_GT(3);
                 __syncwarp();
                 if (++acc == 2) { acc = 0; acc_phase ^= 1; }
             }
@@ -306,18 +355,33 @@ gemm_bf16_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_consta
             const int n0 = tn * BN;
             ok = __all_sync(0xffffffffu, mbar_wait(&acc_full[acc], acc_phase, abort_flag, 0x400 + acc));
             if (!ok) break;
+            if (warp == 2) MLT_GT(4);
             tc_fence_after();
             const uint32_t t_row = tmem_base + (static_cast<uint32_t>(quarter * 32) << 16) + acc * BN;
+            if (!kCTma && BN == 128 && !p.partial && !p.Cf && n0 + BN <= p.N) {
+                // BF16 C, whole tile: through the staging rows, 64 columns at a time (on a problem of one wave the
+                // epilogue is on the critical path)
+                uint8_t* stg = smem_staging + quarter * (32 * kGemmBf16StagePitch);
+#pragma unroll
+                for (int h = 0; h < 2; ++h) {
+                    uint32_t v[2][32];
+                    tmem_ld_32x32b_x32(t_row + h * 64, v[0]);
+                    tmem_ld_32x32b_x32(t_row + h * 64 + 32, v[1]);
+                    tmem_wait_ld();
+                    gemm_store_half_coalesced(p, stg, v, lane, tm * kGemmBM + quarter * 32, n0 + h * 64);
+                }
+            } else {
 #pragma unroll 1
-            for (int c = 0; c < BN / 32; ++c) {
-                uint32_t v[32];
-                tmem_ld_32x32b_x32(t_row + c * 32, v);
-                tmem_wait_ld();
-                if constexpr (kCTma)
-                    gemm_store_chunk_tma(p, &tmap_c, smem_staging + quarter * 8192 + (c & 1) * 4096, v, lane,
-                                         tm * kGemmBM + quarter * 32, n0 + c * 32);
-                else
-                    gemm_store_chunk(p, v, row, n0 + c * 32, item % p.split_k);
+                for (int c = 0; c < BN / 32; ++c) {
+                    uint32_t v[32];
+                    tmem_ld_32x32b_x32(t_row + c * 32, v);
+                    tmem_wait_ld();
+                    if constexpr (kCTma)
+                        gemm_store_chunk_tma(p, &tmap_c, smem_staging + quarter * 8192 + (c & 1) * 4096, v, lane,
+                                             tm * kGemmBM + quarter * 32, n0 + c * 32);
+                    else
+                        gemm_store_chunk(p, v, row, n0 + c * 32, item % p.split_k);
+                }
             }
             tc_fence_before();
             __syncwarp();
@@ -331,6 +395,8 @@ gemm_bf16_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_consta
     tc_fence_before();
     __syncthreads();
     if (blockIdx.x == 0 && threadIdx.x == 0) clock_probe(0, 1);
+    if (threadIdx.x == 0) MLT_GT(5);
+    MLT_GT_NS(7);
     if (warp == 1) {
         __syncwarp();
         tc_fence_after();
@@ -360,6 +426,8 @@ struct GemmPairSmem {
     static constexpr int kStageBytes = kABytes + kBBytes;
     static constexpr int kNoStaging = kStages * kStageBytes + 1024 + 1024;
     static constexpr int kTotal = kNoStaging + kGemmStagingBytes;
+    // BF16 output of the 128-wide kernel goes through a small staging area (see gemm_store_half_coalesced)
+    static constexpr int kBf16Staging = kNoStaging + 4 * 32 * kGemmBf16StagePitch;
 };
 
 template <int kStages, bool kCTma>
@@ -652,17 +720,18 @@ gemm_bf16_clusterk_kernel(const __grid_constant__ CUtensorMap tmap_a, const __gr
         if (__all_sync(0xffffffffu, mbar_wait(acc_full, 0, abort_flag, 0x400))) {
             tc_fence_after();
             const uint32_t t_row = tmem_base + (static_cast<uint32_t>(quarter * 32) << 16);
-#pragma unroll 1
-            for (int c = 0; c < BN / 32; ++c) {
-                uint32_t v[32];
-                tmem_ld_32x32b_x32(t_row + c * 32, v);
-                tmem_wait_ld();
-                if (m0 + r < p.M) {
+            uint32_t v[BN / 32][32];  // all loads in flight before the one wait: the epilogue is on the critical path
+#pragma unroll
+            for (int c = 0; c < BN / 32; ++c) tmem_ld_32x32b_x32(t_row + c * 32, v[c]);
+            tmem_wait_ld();
+            if (m0 + r < p.M) {
+#pragma unroll
+                for (int c = 0; c < BN / 32; ++c) {
                     float4* dst = reinterpret_cast<float4*>(part + r * kClusterKPartPitch + c * 32);
 #pragma unroll
                     for (int q = 0; q < 8; ++q)
-                        dst[q] = make_float4(__uint_as_float(v[q * 4]), __uint_as_float(v[q * 4 + 1]), __uint_as_float(v[q * 4 + 2]),
-                                             __uint_as_float(v[q * 4 + 3]));
+                        dst[q] = make_float4(__uint_as_float(v[c][q * 4]), __uint_as_float(v[c][q * 4 + 1]),
+                                             __uint_as_float(v[c][q * 4 + 2]), __uint_as_float(v[c][q * 4 + 3]));
                 }
             }
         }

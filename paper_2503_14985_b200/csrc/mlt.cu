@@ -28,6 +28,9 @@ struct DeviceInfo {
     int cc_major = 0;
     bool configured = false;
     bool mha_ok = false;  // the attention kernels' compiled register count covers their in-kernel register hand-over
+    // CTAs that can be resident at once as clusters of 2, 4 and 8 of the K-cutting GEMM kernel (a cluster must fit
+    // one GPC, so this can be less than the SM count rounded down to a multiple of the cluster size)
+    int cluster_slots[3] = {0, 0, 0};
 };
 
 std::mutex g_mutex;
@@ -66,13 +69,32 @@ int get_device(DeviceInfo* out) {
             return MLT_ERR_CUDA;
         if (d.cc_major != 10) return MLT_ERR_ARCH;
         if (set_smem(gemm_bf16_kernel<256, 4, false>, GemmSmem<256, 4>::kNoStaging) != MLT_OK ||
-            set_smem(gemm_bf16_kernel<128, 6, false>, GemmSmem<128, 6>::kNoStaging) != MLT_OK ||
+            set_smem(gemm_bf16_kernel<128, 6, false>, GemmSmem<128, 6>::kBf16Staging) != MLT_OK ||
             set_smem(gemm_bf16_pair_kernel<6, false>, GemmPairSmem<6>::kNoStaging) != MLT_OK ||
             set_smem(gemm_bf16_clusterk_kernel<6>, GemmSmem<128, 6>::kNoStaging) != MLT_OK ||
             set_smem(gemm_bf16_kernel<256, 4, true>, GemmSmem<256, 4>::kTotal) != MLT_OK ||
             set_smem(gemm_bf16_kernel<128, 6, true>, GemmSmem<128, 6>::kTotal) != MLT_OK ||
             set_smem(gemm_bf16_pair_kernel<6, true>, GemmPairSmem<6>::kTotal) != MLT_OK)
             return MLT_ERR_CUDA;
+        for (int i = 0; i < 3; ++i) {
+            const int S = 2 << i;
+            cudaLaunchConfig_t cfg = {};
+            cfg.gridDim = dim3(static_cast<unsigned>(d.sm_count / S * S));
+            cfg.blockDim = dim3(kGemmThreads);
+            cfg.dynamicSmemBytes = GemmSmem<128, 6>::kNoStaging;
+            cudaLaunchAttribute attr;
+            attr.id = cudaLaunchAttributeClusterDimension;
+            attr.val.clusterDim.x = static_cast<unsigned>(S);
+            attr.val.clusterDim.y = attr.val.clusterDim.z = 1;
+            cfg.attrs = &attr;
+            cfg.numAttrs = 1;
+            int clusters = 0;
+            if (cudaOccupancyMaxActiveClusters(&clusters, gemm_bf16_clusterk_kernel<6>, &cfg) != cudaSuccess) {
+                cudaGetLastError();
+                clusters = 0;  // unknown: this cluster size is not used
+            }
+            d.cluster_slots[i] = clusters * S;
+        }
         if (paged_configure() != 0) return MLT_ERR_CUDA;
         const int mha_rc = mha_configure();
         if (mha_rc == 1) return MLT_ERR_CUDA;
@@ -192,6 +214,10 @@ int mlt_debug_read_trace(unsigned int* host) {  // development builds only: copi
     if (cudaDeviceSynchronize() != cudaSuccess) return MLT_ERR_CUDA;
     return cudaMemcpyFromSymbol(host, g_mha_trace, sizeof(g_mha_trace)) == cudaSuccess ? MLT_OK : MLT_ERR_CUDA;
 }
+int mlt_debug_read_gemm_trace(long long* host) {  // development builds only
+    if (cudaDeviceSynchronize() != cudaSuccess) return MLT_ERR_CUDA;
+    return cudaMemcpyFromSymbol(host, g_gemm_trace, sizeof(g_gemm_trace)) == cudaSuccess ? MLT_OK : MLT_ERR_CUDA;
+}
 #endif
 
 int mlt_debug_last_clock_mhz(int which, double* mhz) {
@@ -229,15 +255,17 @@ static int gemm_max_split(int64_t M, int64_t N, int64_t K) {
 
 // CTAs per cluster (1, 2, 4 or 8) that cut K for one 128 x 128 tile of a skinny problem: the count that minimises
 // rounds x (K blocks per CTA + fill, drain and the reduction), every slice at least 4 blocks of 64.
-static int gemm_cluster_split(int64_t tiles, int num_kb, int sm_count) {
+// cluster_slots: resident CTAs for S = 2, 4, 8 as the device reports them, or null for the SM count rounded down.
+static int gemm_cluster_split(int64_t tiles, int num_kb, int sm_count, const int* cluster_slots) {
     if (tiles * 2 > sm_count) return 1;  // enough tiles to occupy the GPU without cutting K
     int best_s = 1;
     int64_t best = (num_kb + 4);
-    for (int S = 2; S <= 8; S *= 2) {
+    for (int S = 2, i = 0; S <= 8; S *= 2, ++i) {
         if (num_kb / S < 4 || S > sm_count) break;
         const int kbps = (num_kb + S - 1) / S;
         if (static_cast<int64_t>(kbps) * (S - 1) >= num_kb) continue;  // an empty slice
-        const int64_t slots = sm_count / S * S;
+        const int64_t slots = cluster_slots ? cluster_slots[i] : sm_count / S * S;
+        if (slots < S) continue;
         const int64_t rounds = (tiles * S + slots - 1) / slots;
         const int64_t cost = rounds * (kbps + 10);  // cluster launch, two cluster barriers and the reduction: about 6 blocks more
         if (cost < best) { best = cost; best_s = S; }
@@ -254,7 +282,7 @@ struct GemmPlan {
 };
 
 static GemmPlan gemm_plan(int64_t M, int64_t N, int64_t K, bool has_workspace, size_t workspace_bytes, bool f32_out,
-                          int sm_count, int forced) {
+                          int sm_count, const int* cluster_slots, int forced) {
     // Tile shape by problem size.  Problems with at least 512 rows are compute-bound: the variant with the least
     // (waves x work per tile / efficiency) wins, with the measured relative efficiencies 1 : 0.8 : 0.62 of the three
     // kernels (the smaller tiles are bound by the shared-memory operand path).  Shorter problems stream B once and
@@ -272,7 +300,7 @@ static GemmPlan gemm_plan(int64_t M, int64_t N, int64_t K, bool has_workspace, s
         const double c1 = static_cast<double>((tiles1 + sm_count - 1) / sm_count) / 0.8;
         const double c2 = static_cast<double>((tiles2 + sm_count - 1) / sm_count) * 0.5 / 0.62;
         plan.variant = (c0 <= c1 && c0 <= c2) ? 0 : (c1 <= c2 ? 1 : 2);
-    } else if (!f32_out && (gemm_cluster_split(tiles2, num_kb, sm_count) > 1 ||
+    } else if (!f32_out && (gemm_cluster_split(tiles2, num_kb, sm_count, cluster_slots) > 1 ||
                             (has_workspace && gemm_max_split(M, N, K) > 1))) {
         plan.variant = 2;  // memory-bound and K can be cut: small tiles spread the stream of B evenly over the SMs
     } else if (pair_tiles >= sm_count / 2) {
@@ -287,7 +315,7 @@ static GemmPlan gemm_plan(int64_t M, int64_t N, int64_t K, bool has_workspace, s
 
     // Few tiles: clusters of S CTAs per tile when at most half the SMs would have a tile (measured equal to or faster
     // than partial tiles in scratch plus a second kernel, so it is used with or without a workspace) ...
-    plan.cluster = gemm_cluster_split(tiles2, num_kb, sm_count);
+    plan.cluster = gemm_cluster_split(tiles2, num_kb, sm_count, cluster_slots);
     if (plan.cluster > 1) {
         plan.kb_per_split = (num_kb + plan.cluster - 1) / plan.cluster;
         return plan;
@@ -316,8 +344,14 @@ static GemmPlan gemm_plan(int64_t M, int64_t N, int64_t K, bool has_workspace, s
 }
 
 int mlt_debug_gemm_plan(int64_t M, int64_t N, int64_t K, size_t workspace_bytes, int sm_count, int* out4) {
-    if (!out4 || M <= 0 || N <= 0 || K <= 0 || sm_count < 2) return MLT_ERR_INVALID_ARG;
-    const GemmPlan plan = gemm_plan(M, N, K, workspace_bytes > 0, workspace_bytes, false, sm_count, -1);
+    if (!out4 || M <= 0 || N <= 0 || K <= 0 || sm_count == 1 || sm_count < 0) return MLT_ERR_INVALID_ARG;
+    DeviceInfo dev;
+    if (sm_count == 0) {  // the current device, with the cluster occupancy it reports
+        const int rc = get_device(&dev);
+        if (rc != MLT_OK) return rc;
+    }
+    const GemmPlan plan = sm_count == 0 ? gemm_plan(M, N, K, workspace_bytes > 0, workspace_bytes, false, dev.sm_count, dev.cluster_slots, -1)
+                                        : gemm_plan(M, N, K, workspace_bytes > 0, workspace_bytes, false, sm_count, nullptr, -1);
     out4[0] = plan.variant;
     out4[1] = plan.split_k;
     out4[2] = plan.cluster;
@@ -363,7 +397,7 @@ static int gemm_run(const void* A, const void* B, void* C, int64_t M, int64_t N,
         return cudaGetLastError() == cudaSuccess ? MLT_OK : MLT_ERR_CUDA;
     }
 
-    const GemmPlan plan = gemm_plan(M, N, K, workspace != nullptr, workspace_bytes, f32_out, dev.sm_count, forced_variant());
+    const GemmPlan plan = gemm_plan(M, N, K, workspace != nullptr, workspace_bytes, f32_out, dev.sm_count, dev.cluster_slots, forced_variant());
     const int variant = plan.variant;
     const int bm = variant == 0 ? kPairBM : kGemmBM;
     const int bn = variant == 2 ? 128 : 256;
@@ -465,7 +499,7 @@ static int gemm_run(const void* A, const void* B, void* C, int64_t M, int64_t N,
         else if (c_tma)
             gemm_bf16_kernel<128, 6, true><<<grid, kGemmThreads, GemmSmem<128, 6>::kTotal, st>>>(ta, tb, tc, p);
         else
-            gemm_bf16_kernel<128, 6, false><<<grid, kGemmThreads, GemmSmem<128, 6>::kNoStaging, st>>>(ta, tb, tc, p);
+            gemm_bf16_kernel<128, 6, false><<<grid, kGemmThreads, GemmSmem<128, 6>::kBf16Staging, st>>>(ta, tb, tc, p);
         if (p.split_k > 1) {
             if (cudaGetLastError() != cudaSuccess) return MLT_ERR_CUDA;
             const int64_t groups = M * ((N + 7) / 8);
