@@ -239,6 +239,7 @@ gemm_bf16_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_consta
     uint32_t* tmem_base_slot = reinterpret_cast<uint32_t*>(acc_empty + 2);
     volatile uint32_t* abort_flag = tmem_base_slot + 1;
 
+    if (p.split_k > 1) pdl_launch_dependents();  // the reduce kernel's CTAs take the slots this grid's CTAs leave
     const int warp = threadIdx.x >> 5;
     if (blockIdx.x == 0 && threadIdx.x == 0) clock_probe(0, 0);
     if (threadIdx.x == 0) MLT_GT(0);

@@ -117,6 +117,7 @@ __device__ __forceinline__ int paged_head_sub(int g) {  // the lowest `sub` that
 template <int D, int G, int BS>
 __global__ void __launch_bounds__(kPagedThreads)
 paged_decode_kernel(const PagedParams p) {
+    pdl_launch_dependents();  // the combine kernel's CTAs take the slots this grid's CTAs leave, and do their prologue early
     constexpr int LPT = D / 8;         // lanes per token
     constexpr int TPS = 32 / LPT;      // tokens per load instruction of a warp
     constexpr int STEPS = BS / TPS;    // load instructions per block and tensor
@@ -371,6 +372,7 @@ __device__ __forceinline__ int paged_quota(long long n, int max_row, int ctas) {
 template <int D, int G, int BS>
 __global__ void __launch_bounds__(kPagedThreads, kPagedMmaCtasPerSm)
 paged_decode_mma_kernel(const PagedParams p) {
+    pdl_launch_dependents();  // the combine kernel's CTAs take the slots this grid's CTAs leave, and do their prologue early
     static_assert(G == 4 || G == 8, "rows of the MMA: 4 or 8 query heads");
     constexpr int PP = D / 32;  // pairs of 16-element steps of Q K^T
     constexpr int HV = D / 64;  // halves of D in the P V output mapping
