@@ -53,14 +53,29 @@ namespace mlt {
 
 // In-kernel clock trace (development builds only, -DMLT_TRACE): CTA 0 records the SM clock at fixed points of K/V
 // blocks 32..47 of its first work item; role 0 / 1 = first softmax warp of tile 0 / 1, role 2 = UMMA issuer.
-#ifdef MLT_TRACE
+#ifdef MLT_TRACE_ITEMS
+// second form (-DMLT_TRACE -DMLT_TRACE_ITEMS): per work item r < 16 of CTA 0, the first 8 blocks' "S seen" and
+// "P handed over" times (slots 2j, 2j + 1) and the item's start, "O complete seen" and "epilogue done" (18, 16, 17)
+__device__ unsigned int g_mha_trace[3][16][24];
+#define MLT_TR(role, j, ev)                                                                                  \
+    do {                                                                                                     \
+        if (blockIdx.x == 0 && r < 16 && (j) >= 0 && (j) < 8 && ((ev) == 1 || (ev) == 4))                     \
+            g_mha_trace[role][r][(j) * 2 + ((ev) == 4)] = static_cast<unsigned int>(clock64());              \
+    } while (0)
+#define MLT_TRI(role, ev)                                                                                    \
+    do {                                                                                                     \
+        if (blockIdx.x == 0 && r < 16) g_mha_trace[role][r][ev] = static_cast<unsigned int>(clock64());      \
+    } while (0)
+#elif defined(MLT_TRACE)
 __device__ unsigned int g_mha_trace[3][16][24];
 #define MLT_TR(role, j, ev)                                                                                  \
     do {                                                                                                     \
         if (blockIdx.x == 0 && r == 0 && (j) >= 32 && (j) < 48) g_mha_trace[role][(j) - 32][ev] = static_cast<unsigned int>(clock64()); \
     } while (0)
+#define MLT_TRI(role, ev) do { } while (0)
 #else
 #define MLT_TR(role, j, ev) do { } while (0)
+#define MLT_TRI(role, ev) do { } while (0)
 #endif
 
 constexpr int kMhaBlock = 128;   // query rows per tile and keys per K/V block
@@ -557,6 +572,7 @@ mha_fwd_kernel(const __grid_constant__ CUtensorMap tmap_q, const __grid_constant
         const int limit = p.causal ? min(p.Nk - 1, qi + shift) : p.Nk - 1;  // last visible key of this row
         float m_run = -INFINITY;  // reference max (raw score units), taken from the row's first block
         float l_run = 0.0f;
+        if (quarter == 0 && lane == 0) MLT_TRI(t, 18);
 
         for (int j = 0; j < Jt; ++j) {
             if (quarter == 0 && lane == 0) MLT_TR(t, j, 0);
@@ -684,6 +700,7 @@ mha_fwd_kernel(const __grid_constant__ CUtensorMap tmap_q, const __grid_constant
         if (!ok) break;
         ++n_o;
         tc_fence_after();
+        if (quarter == 0 && lane == 0) MLT_TRI(t, 16);
         {
             // Once the loads from tensor memory have completed the next item's first P V may overwrite O_t: the
             // softmax of that item, and with it P_t(0), comes after this point in program order.
@@ -722,6 +739,7 @@ mha_fwd_kernel(const __grid_constant__ CUtensorMap tmap_q, const __grid_constant
             if (valid && p.LSE)
                 p.LSE[static_cast<int64_t>(it.bh) * p.Nq + qi] = m_run * p.scale + __log2f(l_run) * 0.6931471805599453f;
         }
+        if (quarter == 0 && lane == 0) MLT_TRI(t, 17);
         }  // items
         if (lane == 0) tma_store_wait_all<0>();  // shared memory must outlive the stores that read it
     }

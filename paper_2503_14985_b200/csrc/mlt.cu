@@ -209,7 +209,7 @@ int mlt_debug_wait_timeout_selftest(uint64_t budget_cycles, void* stream) {
     return cudaGetLastError() == cudaSuccess ? MLT_OK : MLT_ERR_CUDA;
 }
 
-#ifdef MLT_TRACE
+#if defined(MLT_TRACE) || defined(MLT_TRACE_ITEMS)
 int mlt_debug_read_trace(unsigned int* host) {  // development builds only: copies the attention kernel's clock trace
     if (cudaDeviceSynchronize() != cudaSuccess) return MLT_ERR_CUDA;
     return cudaMemcpyFromSymbol(host, g_mha_trace, sizeof(g_mha_trace)) == cudaSuccess ? MLT_OK : MLT_ERR_CUDA;
