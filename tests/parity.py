@@ -46,7 +46,7 @@ def check_mha(o, lse, o_ref, lse_ref, what="", unit=1.0):
 
 def log_line(text: str) -> None:
     """Appends one line to the parity log of this run (full-output comparisons are recorded there): the file named
-    by MLT_PARITY_LOG, else gpurun_out/parity_full_configs.log under the repository root.  Never fails a test."""
+    by MLT_PARITY_LOG, else parity_full_configs.log in the repository's untracked output folder.  Never fails a test."""
     import os
     path = os.environ.get("MLT_PARITY_LOG")
     if not path:
