@@ -47,6 +47,8 @@
 
 #include <math.h>
 
+#include <cstdlib>
+
 #include "ptx.cuh"
 
 namespace mlt {
@@ -110,7 +112,12 @@ struct MhaParams {
     float scale;
     int num_pairs;   // 256-row query groups per head
     int head_group;  // heads that share a span of consecutive item indices
-    int num_items;   // num_pairs * BH
+    int num_items;   // entries of the work list
+    // Entries below full_items are whole items (both 128-row tiles of a 256-row group).  The entries after them are
+    // single tiles, two entries per remaining item: a last round that would occupy at most half of the CTAs is
+    // handed out tile by tile, so twice as many CTAs share it (a CTA with one tile runs its blocks in 0.8-0.9 of
+    // the time of a CTA with two).
+    int full_items;
 };
 
 // item index -> (pair, bh).  Heads are taken in groups; inside a group the query
@@ -210,13 +217,18 @@ mha_fwd_kernel(const __grid_constant__ CUtensorMap tmap_q, const __grid_constant
     auto decode_item = [&](int r, Item& it) -> bool {
         const int idx = r * G + ((r & 1) ? G - 1 - static_cast<int>(blockIdx.x) : static_cast<int>(blockIdx.x));
         if (r >= rounds || idx >= p.num_items) return false;
-        int pair;
-        mha_item(p, idx, pair, it.bh);
+        int pair, only = -1;  // only: the one tile a single-tile entry stands for
+        int item = idx;
+        if (idx >= p.full_items) {
+            item = p.full_items + ((idx - p.full_items) >> 1);
+            only = (idx - p.full_items) & 1;
+        }
+        mha_item(p, item, pair, it.bh);
         it.q_base = pair * 2 * kMhaBlock;
 #pragma unroll
         for (int t = 0; t < 2; ++t) {  // number of K/V blocks each tile needs
             const int q0 = it.q_base + t * kMhaBlock;
-            if (q0 >= p.Nq) {
+            if (q0 >= p.Nq || (only >= 0 && t != only)) {
                 it.J[t] = 0;
             } else {
                 int last_key = p.Nk - 1;
@@ -776,6 +788,12 @@ inline int mha_configure() {
     return 0;
 }
 
+// Development switch (environment variable MLT_MHA_NO_HALF_ITEMS): hand the last round out as whole items.
+inline bool debug_no_half_items() {
+    static const bool off = std::getenv("MLT_MHA_NO_HALF_ITEMS") != nullptr;
+    return off;
+}
+
 inline int mha_launch(const CUtensorMap& tq, const CUtensorMap& tk, const CUtensorMap& tv, const CUtensorMap& to, float* LSE,
                       int B, int H, int Nq, int Nk, int D, bool causal, float scale, int sm_count, cudaStream_t st,
                       int head_group_override = 0, int grid_override = 0) {
@@ -789,7 +807,7 @@ inline int mha_launch(const CUtensorMap& tq, const CUtensorMap& tk, const CUtens
     p.num_pairs = (Nq + 2 * kMhaBlock - 1) / (2 * kMhaBlock);
     const int64_t items = static_cast<int64_t>(p.num_pairs) * p.BH;
     if (items > INT32_MAX - 1024) return 2;
-    p.num_items = static_cast<int>(items);
+    p.num_items = p.full_items = static_cast<int>(items);
     // Items of equal length (no mask), or many short ones under a causal mask: persistent CTAs, one per SM, which
     // hide each item's fill and drain behind its neighbours.  Causal list order: all heads' last query rows first
     // (longest first over the whole problem), so that the static hand-out balances; otherwise heads go in groups
@@ -803,6 +821,19 @@ inline int mha_launch(const CUtensorMap& tq, const CUtensorMap& tk, const CUtens
     if (head_group_override > 0) p.head_group = head_group_override;
     int grid = static_cast<int>(persistent ? std::min<int64_t>(items, sm_count) : items);
     if (grid_override > 0) grid = static_cast<int>(std::min<int64_t>(items, grid_override));
+    if (persistent) {
+        // a last round of at most half the CTAs goes out tile by tile (only when every item has two real tiles, so
+        // that no entry is empty)
+        const int ctas = grid_override > 0 ? grid_override : sm_count;
+        const int rem = static_cast<int>(items % ctas);
+        const bool two_tiles_each = ((Nq + kMhaBlock - 1) / kMhaBlock) % 2 == 0;
+        // (not when the whole problem is one round: 68 items ran 4 % slower as 136 single tiles)
+        if (items > ctas && rem > 0 && 2 * rem <= ctas && two_tiles_each && !debug_no_half_items()) {
+            p.full_items = static_cast<int>(items) - rem;
+            p.num_items = static_cast<int>(items) + rem;
+            grid = std::min(p.num_items, ctas);
+        }
+    }
     if (D == 64)
         mha_fwd_kernel<64><<<grid, kMhaThreads, MhaSmem<64>::kTotal, st>>>(tq, tk, tv, to, p);
     else

@@ -54,7 +54,9 @@ CASES = [(1, 1, 128, 128, 64, 0), (1, 1, 128, 128, 128, 1), (1, 2, 1, 1, 64, 0),
          # more work items than SMs: a CTA runs several items one after another (ragged last pairs among them)
          (3, 70, 300, 300, 64, 1), (2, 80, 300, 420, 128, 1), (5, 40, 520, 260, 128, 0), (2, 90, 257, 257, 64, 0),
          # ... with a single K/V block per item, and with the second 128-row tile absent in every item
-         (2, 100, 256, 128, 64, 0), (2, 100, 256, 100, 128, 0), (3, 60, 128, 128, 64, 1), (3, 60, 100, 228, 128, 1)]
+         (2, 100, 256, 128, 64, 0), (2, 100, 256, 100, 128, 0), (3, 60, 128, 128, 64, 1), (3, 60, 100, 228, 128, 1),
+         # a last round of at most half the CTAs (on 148 SMs: 2, 8 and 52 items left over), handed out as single tiles
+         (1, 150, 256, 300, 128, 1), (1, 75, 512, 512, 64, 1), (2, 76, 512, 640, 64, 0), (1, 100, 512, 384, 128, 0)]
 
 
 @pytest.mark.parametrize("B,H,Nq,Nk,D,causal", CASES)
