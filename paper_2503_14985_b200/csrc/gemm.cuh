@@ -604,7 +604,7 @@ gemm_bf16_pair_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_c
 // distributed-shared-memory loads, ascending slice order: deterministic) and stores BF16.  One kernel, no partial
 // tiles in global memory, no second launch.  One tile per cluster.
 // ---------------------------------------------------------------------------
-constexpr int kClusterKPartPitch = 132;  // floats per row of the FP32 tile in shared memory (528 B: conflict-free 16-byte rows)
+constexpr int kClusterKPartPad = 4;  // floats added to a row of the FP32 tile in shared memory (pitch 528 or 1040 B: conflict-free 16-byte rows)
 
 __device__ __forceinline__ float4 ld_shared_cluster_f32x4(uint32_t cluster_addr) {
     float4 v;
@@ -617,13 +617,14 @@ __device__ __forceinline__ uint32_t cluster_nctarank() {
     return r;
 }
 
-template <int kStages>
+template <int BN, int kStages>
 __global__ void __launch_bounds__(kGemmThreads, 1)
 gemm_bf16_clusterk_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_constant__ CUtensorMap tmap_b,
                           const GemmParams p) {
-    constexpr int BN = 128;
+    static_assert(BN == 128 || BN == 256, "tile widths of the single-CTA kernels");
+    constexpr int kPartPitch = BN + kClusterKPartPad;
     using L = GemmSmem<BN, kStages>;
-    static_assert(kGemmBM * kClusterKPartPitch * 4 <= kStages * L::kStageBytes, "the FP32 tile fits the pipeline stages");
+    static_assert(kGemmBM * kPartPitch * 4 <= kStages * L::kStageBytes, "the FP32 tile fits the pipeline stages");
     extern __shared__ uint8_t smem_raw[];
     uint8_t* smem = reinterpret_cast<uint8_t*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~uintptr_t(1023));
     uint64_t* bars = reinterpret_cast<uint64_t*>(smem + kStages * L::kStageBytes);
@@ -667,7 +668,7 @@ gemm_bf16_clusterk_kernel(const __grid_constant__ CUtensorMap tmap_a, const __gr
     __syncthreads();
     tc_fence_after();
     const uint32_t tmem_base = *tmem_base_slot;
-    float* part = reinterpret_cast<float*>(smem);  // [128][kClusterKPartPitch], written after the main loop
+    float* part = reinterpret_cast<float*>(smem);  // [128][kPartPitch], written after the main loop
 
     if (warp == 0) {
         if (lane == 0) {
@@ -721,18 +722,21 @@ gemm_bf16_clusterk_kernel(const __grid_constant__ CUtensorMap tmap_a, const __gr
         if (__all_sync(0xffffffffu, mbar_wait(acc_full, 0, abort_flag, 0x400))) {
             tc_fence_after();
             const uint32_t t_row = tmem_base + (static_cast<uint32_t>(quarter * 32) << 16);
-            uint32_t v[BN / 32][32];  // all loads in flight before the one wait: the epilogue is on the critical path
+#pragma unroll 1
+            for (int h = 0; h < BN / 128; ++h) {  // 128 columns at a time: four loads in flight before the one wait
+                uint32_t v[4][32];
 #pragma unroll
-            for (int c = 0; c < BN / 32; ++c) tmem_ld_32x32b_x32(t_row + c * 32, v[c]);
-            tmem_wait_ld();
-            if (m0 + r < p.M) {
+                for (int c = 0; c < 4; ++c) tmem_ld_32x32b_x32(t_row + h * 128 + c * 32, v[c]);
+                tmem_wait_ld();
+                if (m0 + r < p.M) {
 #pragma unroll
-                for (int c = 0; c < BN / 32; ++c) {
-                    float4* dst = reinterpret_cast<float4*>(part + r * kClusterKPartPitch + c * 32);
+                    for (int c = 0; c < 4; ++c) {
+                        float4* dst = reinterpret_cast<float4*>(part + r * kPartPitch + h * 128 + c * 32);
 #pragma unroll
-                    for (int q = 0; q < 8; ++q)
-                        dst[q] = make_float4(__uint_as_float(v[c][q * 4]), __uint_as_float(v[c][q * 4 + 1]),
-                                             __uint_as_float(v[c][q * 4 + 2]), __uint_as_float(v[c][q * 4 + 3]));
+                        for (int q = 0; q < 8; ++q)
+                            dst[q] = make_float4(__uint_as_float(v[c][q * 4]), __uint_as_float(v[c][q * 4 + 1]),
+                                                 __uint_as_float(v[c][q * 4 + 2]), __uint_as_float(v[c][q * 4 + 3]));
+                    }
                 }
             }
         }
@@ -743,7 +747,7 @@ gemm_bf16_clusterk_kernel(const __grid_constant__ CUtensorMap tmap_a, const __gr
     tc_fence_before();
     cluster_sync_all();
     {
-        const int cols = BN / S;  // S in {2, 4, 8}: 64, 32 or 16 columns, in groups of 4
+        const int cols = BN / S;  // S in {2, 4, 8}: 16 to 128 columns, in groups of 4
         const int groups = cols / 4;
         const int rows = min(kGemmBM, p.M - m0);
         const uint32_t part_addr = smem_u32(part);
@@ -751,7 +755,7 @@ gemm_bf16_clusterk_kernel(const __grid_constant__ CUtensorMap tmap_a, const __gr
             const int r = idx / groups, c = slice * cols + (idx % groups) * 4;
             float4 acc = make_float4(0.0f, 0.0f, 0.0f, 0.0f);
             for (int s2 = 0; s2 < S; ++s2) {
-                const float4 v = ld_shared_cluster_f32x4(map_to_cta(part_addr + (r * kClusterKPartPitch + c) * 4, s2));
+                const float4 v = ld_shared_cluster_f32x4(map_to_cta(part_addr + (r * kPartPitch + c) * 4, s2));
                 acc.x += v.x; acc.y += v.y; acc.z += v.z; acc.w += v.w;
             }
             const int col = n0 + c;

@@ -71,7 +71,8 @@ int get_device(DeviceInfo* out) {
         if (set_smem(gemm_bf16_kernel<256, 4, false>, GemmSmem<256, 4>::kNoStaging) != MLT_OK ||
             set_smem(gemm_bf16_kernel<128, 6, false>, GemmSmem<128, 6>::kBf16Staging) != MLT_OK ||
             set_smem(gemm_bf16_pair_kernel<6, false>, GemmPairSmem<6>::kNoStaging) != MLT_OK ||
-            set_smem(gemm_bf16_clusterk_kernel<6>, GemmSmem<128, 6>::kNoStaging) != MLT_OK ||
+            set_smem(gemm_bf16_clusterk_kernel<128, 6>, GemmSmem<128, 6>::kNoStaging) != MLT_OK ||
+            set_smem(gemm_bf16_clusterk_kernel<256, 4>, GemmSmem<256, 4>::kNoStaging) != MLT_OK ||
             set_smem(gemm_bf16_kernel<256, 4, true>, GemmSmem<256, 4>::kTotal) != MLT_OK ||
             set_smem(gemm_bf16_kernel<128, 6, true>, GemmSmem<128, 6>::kTotal) != MLT_OK ||
             set_smem(gemm_bf16_pair_kernel<6, true>, GemmPairSmem<6>::kTotal) != MLT_OK)
@@ -89,7 +90,7 @@ int get_device(DeviceInfo* out) {
             cfg.attrs = &attr;
             cfg.numAttrs = 1;
             int clusters = 0;
-            if (cudaOccupancyMaxActiveClusters(&clusters, gemm_bf16_clusterk_kernel<6>, &cfg) != cudaSuccess) {
+            if (cudaOccupancyMaxActiveClusters(&clusters, gemm_bf16_clusterk_kernel<128, 6>, &cfg) != cudaSuccess) {
                 cudaGetLastError();
                 clusters = 0;  // unknown: this cluster size is not used
             }
@@ -145,9 +146,10 @@ int forced_variant() {
 
 // Debug only: tuning overrides read once from the environment (0 = not set).  MLT_GEMM_GROUP_M: M-tiles per raster
 // group of the pair kernel; MLT_GEMM_NO_HALF: no half tiles in the last wave; MLT_MHA_HEAD_GROUP / MLT_MHA_GRID: item
-// list grouping and CTA count of the attention kernel; MLT_PAGED_SPLITS: CTAs per (sequence, KV head).
+// list grouping and CTA count of the attention kernel; MLT_PAGED_SPLITS: CTAs per (sequence, KV head);
+// MLT_GEMM_WIDE_RATIO: per cent of the current plan's cost below which 128 x 256 tiles in clusters are taken (1: never).
 struct DebugEnv {
-    int gemm_group_m, gemm_no_half, mha_head_group, mha_grid, paged_splits;
+    int gemm_group_m, gemm_no_half, mha_head_group, mha_grid, paged_splits, gemm_wide_ratio;
 };
 const DebugEnv& debug_env() {
     static const DebugEnv env = [] {
@@ -157,7 +159,7 @@ const DebugEnv& debug_env() {
             return v > 0 ? v : 0;
         };
         return DebugEnv{get("MLT_GEMM_GROUP_M"), get("MLT_GEMM_NO_HALF"), get("MLT_MHA_HEAD_GROUP"), get("MLT_MHA_GRID"),
-                        get("MLT_PAGED_SPLITS")};
+                        get("MLT_PAGED_SPLITS"), get("MLT_GEMM_WIDE_RATIO")};
     }();
     return env;
 }
@@ -277,12 +279,12 @@ static int gemm_cluster_split(int64_t tiles, int num_kb, int sm_count, const int
 struct GemmPlan {
     int variant;       // 0: CTA pairs on 256 x 256 tiles, 1: 128 x 256 tiles, 2: 128 x 128 tiles
     int split_k;       // > 1: K slices with FP32 partials in caller scratch, summed by a second kernel
-    int cluster;       // > 1: CTAs per cluster that cut K for one tile and reduce through distributed shared memory
+    int cluster;       // > 1: CTAs per cluster that cut K for one tile (128 x 128, or 128 x 256 with variant 1) and reduce through distributed shared memory
     int kb_per_split;  // K blocks of 64 per slice (per CTA of a cluster)
 };
 
-static GemmPlan gemm_plan(int64_t M, int64_t N, int64_t K, bool has_workspace, size_t workspace_bytes, bool f32_out,
-                          int sm_count, const int* cluster_slots, int forced) {
+static GemmPlan gemm_plan_base(int64_t M, int64_t N, int64_t K, bool has_workspace, size_t workspace_bytes, bool f32_out,
+                               int sm_count, const int* cluster_slots, int forced) {
     // Tile shape by problem size.  Problems with at least 512 rows are compute-bound: the variant with the least
     // (waves x work per tile / efficiency) wins, with the measured relative efficiencies 1 : 0.8 : 0.62 of the three
     // kernels (the smaller tiles are bound by the shared-memory operand path).  Shorter problems stream B once and
@@ -340,6 +342,52 @@ static GemmPlan gemm_plan(int64_t M, int64_t N, int64_t K, bool has_workspace, s
         plan.kb_per_split = (num_kb + split - 1) / split;
         plan.split_k = (num_kb + plan.kb_per_split - 1) / plan.kb_per_split;  // no empty slice
     }
+    return plan;
+}
+
+// The plan above, or for problems of 129 to 640 rows 128 x 256 tiles with K cut inside clusters, when that moves
+// clearly fewer bytes through the busiest SM.  These problems are bound by what one SM can pull from L2 (about 110
+// GB/s): a 128 x 128 tile pulls 32 KB per K block for 2 MFLOP, a 128 x 256 tile 48 KB for 4 MFLOP, and cutting K
+// inside a cluster puts the narrower problem on all SMs all the same.  Cost of a plan = rounds x (K blocks per CTA +
+// fixed blocks) x KB per block.
+static GemmPlan gemm_plan(int64_t M, int64_t N, int64_t K, bool has_workspace, size_t workspace_bytes, bool f32_out,
+                          int sm_count, const int* cluster_slots, int forced) {
+    GemmPlan plan = gemm_plan_base(M, N, K, has_workspace, workspace_bytes, f32_out, sm_count, cluster_slots, forced);
+    const int ratio = debug_env().gemm_wide_ratio ? debug_env().gemm_wide_ratio : 90;  // per cent; 1: never
+    if (f32_out || M <= 128 || M > 640 || (forced >= 0 && forced <= 2) || sm_count < 8) return plan;
+    const int64_t pair_tiles = ((M + kPairBM - 1) / kPairBM) * ((N + kPairBN - 1) / kPairBN);
+    const int64_t tiles_m128 = (M + kGemmBM - 1) / kGemmBM;
+    const int64_t tiles1 = tiles_m128 * ((N + 255) / 256);
+    const int64_t tiles2 = tiles_m128 * ((N + 127) / 128);
+    const int num_kb = static_cast<int>((K + kGemmBK - 1) / kGemmBK);
+    auto slots_of = [&](int S) {
+        const int i = S == 2 ? 0 : (S == 4 ? 1 : 2);
+        return static_cast<int64_t>(cluster_slots ? cluster_slots[i] : sm_count / S * S);
+    };
+    auto rounds_of = [](int64_t items, int64_t slots) { return (items + slots - 1) / slots; };
+    double cur;
+    if (plan.variant == 0)
+        cur = static_cast<double>(rounds_of(pair_tiles, sm_count / 2)) * (num_kb + 4) * 32.0;
+    else if (plan.variant == 1)
+        cur = static_cast<double>(rounds_of(tiles1, sm_count)) * (num_kb + 4) * 48.0;
+    else if (plan.cluster > 1)
+        cur = static_cast<double>(rounds_of(tiles2 * plan.cluster, std::max<int64_t>(slots_of(plan.cluster), plan.cluster))) *
+              (plan.kb_per_split + 10) * 32.0;
+    else
+        cur = static_cast<double>(rounds_of(tiles2 * plan.split_k, sm_count)) * (plan.kb_per_split + 4) * 32.0 +
+              (plan.split_k > 1 ? static_cast<double>(plan.split_k) * M * N * 8.0 / (1024.0 * sm_count) : 0.0);
+    int best_s = 1, best_kbps = num_kb;
+    double best = 1e300;
+    for (int S = 2; S <= 8; S *= 2) {
+        if (num_kb / S < 4) break;
+        const int kbps = (num_kb + S - 1) / S;
+        if (static_cast<int64_t>(kbps) * (S - 1) >= num_kb) continue;  // an empty slice
+        const int64_t slots = slots_of(S);
+        if (slots < S) continue;
+        const double cost = static_cast<double>(rounds_of(tiles1 * S, slots)) * (kbps + 10) * 48.0;
+        if (cost < best) { best = cost; best_s = S; best_kbps = kbps; }
+    }
+    if (best_s > 1 && best * 100.0 < cur * ratio) plan = GemmPlan{1, 1, best_s, best_kbps};
     return plan;
 }
 
@@ -479,7 +527,7 @@ static int gemm_run(const void* A, const void* B, void* C, int64_t M, int64_t N,
         cudaLaunchConfig_t cfg = {};
         cfg.gridDim = dim3(static_cast<unsigned>(tiles_m * tiles_n * S));
         cfg.blockDim = dim3(kGemmThreads);
-        cfg.dynamicSmemBytes = GemmSmem<128, 6>::kNoStaging;
+        cfg.dynamicSmemBytes = variant == 1 ? GemmSmem<256, 4>::kNoStaging : GemmSmem<128, 6>::kNoStaging;
         cfg.stream = st;
         cudaLaunchAttribute attr;
         attr.id = cudaLaunchAttributeClusterDimension;
@@ -488,7 +536,9 @@ static int gemm_run(const void* A, const void* B, void* C, int64_t M, int64_t N,
         attr.val.clusterDim.z = 1;
         cfg.attrs = &attr;
         cfg.numAttrs = 1;
-        if (cudaLaunchKernelEx(&cfg, gemm_bf16_clusterk_kernel<6>, ta, tb, p) != cudaSuccess) return MLT_ERR_CUDA;
+        const cudaError_t e = variant == 1 ? cudaLaunchKernelEx(&cfg, gemm_bf16_clusterk_kernel<256, 4>, ta, tb, p)
+                                           : cudaLaunchKernelEx(&cfg, gemm_bf16_clusterk_kernel<128, 6>, ta, tb, p);
+        if (e != cudaSuccess) return MLT_ERR_CUDA;
     } else {
         p.group_m = 16;
         const int grid = static_cast<int>(std::min<int64_t>(tiles_m * tiles_n * p.split_k, dev.sm_count));

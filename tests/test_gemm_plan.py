@@ -13,7 +13,7 @@ def kb(K):
 
 @pytest.mark.parametrize("sm_count", [148, 132, 64, 2])
 def test_plan_invariants(sm_count):
-    Ms = [1, 16, 100, 130, 511, 512, 2000]
+    Ms = [1, 16, 100, 130, 300, 511, 512, 640, 2000]
     Ns = [8, 128, 520, 4096, 9600, 28672]
     Ks = [8, 64, 520, 2048, 4100, 28672]
     for M, N, K in itertools.product(Ms, Ns, Ks):
@@ -28,13 +28,13 @@ def test_plan_invariants(sm_count):
             if slices == 1:
                 assert pl["kb_per_split"] == kb(K), what
                 continue
-            assert pl["variant"] == 2, what
+            assert pl["variant"] == 2 or (pl["variant"] == 1 and pl["cluster"] > 1 and 128 < M <= 640), what
             # every slice has work, the slices cover K, none is shorter than 4 blocks by design of the cut
             assert pl["kb_per_split"] * (slices - 1) < kb(K) <= pl["kb_per_split"] * slices, what
             assert kb(K) // slices >= 4, what
             if pl["split_k"] > 1:
                 assert pl["split_k"] * M * N * 4 <= ws, what
-            else:
+            elif pl["variant"] == 2:
                 tiles = ((M + 127) // 128) * ((N + 127) // 128)
                 assert 2 * tiles <= sm_count, what
 
@@ -54,6 +54,9 @@ def test_plan_known_cases_on_148_sms():
     # a short K is not cut
     assert full(16, 4096, 192)["cluster"] == 1 and full(16, 4096, 192)["split_k"] == 1
     assert full(512, 512, 512)["cluster"] == 1
+    # 129 to 640 rows: 128 x 256 tiles with K cut in clusters when that moves clearly fewer bytes per SM
+    assert mlt.gemm_plan(256, 8192, 8192) == {"variant": 1, "split_k": 1, "cluster": 2, "kb_per_split": 64}
+    assert mlt.gemm_plan(128, 8192, 8192)["variant"] == 2
 
 
 def test_plan_rejects_bad_arguments():

@@ -121,3 +121,22 @@ def test_argument_errors():
     assert mlt.gemm_ex_raw(p, p, p, 8, 8, 8, 8, 8, 8, p + 4, 1024) == 3       # misaligned workspace
     assert mlt.gemm_workspace_bytes(8192, 8192, 8192) == 0                     # plenty of tiles: no split
     assert mlt.gemm_workspace_bytes(16, 4096, 256) == 0                        # K too short to cut
+
+
+# 129 to 640 rows: 128 x 256 tiles with K cut inside clusters (two tile rows and more, ragged edges, a short last slice)
+WIDE_CLUSTER_SHAPES = [(384, 4096, 14336), (160, 4104, 28672 + 40), (256, 8192, 8192), (300, 2056, 16000), (640, 1000, 12000 + 8)]
+
+
+@pytest.mark.parametrize("M,N,K", WIDE_CLUSTER_SHAPES)
+def test_wide_tiles_in_clusters(M, N, K):
+    pl = plan(M, N, K)
+    print(f"{M}x{N}x{K}: {pl}")
+    if mlt.gemm_plan(M, N, K, 0, 148)["variant"] == 1:   # what a device of 148 SMs with every SM usable would do
+        assert mlt.gemm_plan(M, N, K, 0, 148)["cluster"] > 1
+    lda, ldb, ldc = (K + 7) // 8 * 8, (N + 7) // 8 * 8 + 8, (N + 7) // 8 * 8 + 8
+    A, B = inputs.gemm_inputs(M, N, K, seed=950 + M, kind="uniform", lda=lda, ldb=ldb)
+    C = run_ex(A, B, M, N, K, ldc, 0)
+    rows = np.unique(np.concatenate([np.arange(0, M, 37), [0, 127, 128, M - 1]])).astype(np.int64)
+    check_gemm(C[rows], oracle.gemm(A, B, M, N, K, rows=rows), f"wide cluster {M}x{N}x{K}")
+    assert np.array_equal(C, run_ex(A, B, M, N, K, ldc, 0))          # fixed summation order
+
