@@ -566,6 +566,21 @@ gemm_bf16_pair_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_c
             if (!ok) break;
             tc_fence_after();
             const uint32_t t_row = tmem_base + (static_cast<uint32_t>(quarter * 32) << 16) + acc * kPairBN;
+            // The last item of a CTA has no main loop behind it to hide its epilogue, and all CTAs reach theirs at about
+            // the same time: there BF16 C goes through the staging rows in whole lines (half the time of the per-row
+            // stores; not in steady state, where the extra shared-memory traffic would slow the operand reads).
+            if (!kCTma && !p.Cf && item + num_clusters >= p.num_items && n0 + bn <= p.N) {
+                uint8_t* stg = smem_staging + quarter * (32 * kGemmBf16StagePitch);
+#pragma unroll 1
+                for (int h = 0; h < bn / 64; ++h) {
+                    uint32_t v[2][32];
+                    tmem_ld_32x32b_x32(t_row + h * 64, v[0]);
+                    tmem_ld_32x32b_x32(t_row + h * 64 + 32, v[1]);
+                    tmem_wait_ld();
+                    gemm_store_half_coalesced(p, stg, v, lane, tm * kPairBM + static_cast<int>(rank) * 128 + quarter * 32,
+                                              n0 + h * 64);
+                }
+            } else {
 #pragma unroll 1
             for (int c = 0; c < bn / 32; ++c) {
                 uint32_t v[32];
@@ -576,6 +591,7 @@ gemm_bf16_pair_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_c
                                          tm * kPairBM + static_cast<int>(rank) * 128 + quarter * 32, n0 + c * 32);
                 else
                     gemm_store_chunk(p, v, row, n0 + c * 32, 0);
+            }
             }
             tc_fence_before();
             __syncwarp();

@@ -70,7 +70,7 @@ int get_device(DeviceInfo* out) {
         if (d.cc_major != 10) return MLT_ERR_ARCH;
         if (set_smem(gemm_bf16_kernel<256, 4, false>, GemmSmem<256, 4>::kNoStaging) != MLT_OK ||
             set_smem(gemm_bf16_kernel<128, 6, false>, GemmSmem<128, 6>::kBf16Staging) != MLT_OK ||
-            set_smem(gemm_bf16_pair_kernel<6, false>, GemmPairSmem<6>::kNoStaging) != MLT_OK ||
+            set_smem(gemm_bf16_pair_kernel<6, false>, GemmPairSmem<6>::kBf16Staging) != MLT_OK ||
             set_smem(gemm_bf16_clusterk_kernel<128, 6>, GemmSmem<128, 6>::kNoStaging) != MLT_OK ||
             set_smem(gemm_bf16_clusterk_kernel<256, 4>, GemmSmem<256, 4>::kNoStaging) != MLT_OK ||
             set_smem(gemm_bf16_kernel<256, 4, true>, GemmSmem<256, 4>::kTotal) != MLT_OK ||
@@ -516,7 +516,7 @@ static int gemm_run(const void* A, const void* B, void* C, int64_t M, int64_t N,
         if (c_tma)
             gemm_bf16_pair_kernel<6, true><<<2 * clusters, kGemmThreads, GemmPairSmem<6>::kTotal, st>>>(ta, tb, tc, p);
         else
-            gemm_bf16_pair_kernel<6, false><<<2 * clusters, kGemmThreads, GemmPairSmem<6>::kNoStaging, st>>>(ta, tb, tc, p);
+            gemm_bf16_pair_kernel<6, false><<<2 * clusters, kGemmThreads, GemmPairSmem<6>::kBf16Staging, st>>>(ta, tb, tc, p);
     } else if (cluster_s > 1) {
         // Skinny problem with few tiles: K is cut inside clusters of S CTAs per tile, which reduce through
         // distributed shared memory (gemm_bf16_clusterk_kernel)
