@@ -188,7 +188,9 @@ int mlt_debug_last_clock_mhz(int which, double* mhz);
  * lets tests pin which kernel a shape reaches).  sm_count >= 2: a device of that many SMs on which clusters can use
  * every SM (host arithmetic only, no CUDA call).  sm_count == 0: the current device, with the number of resident
  * clusters it reports (a cluster must fit one GPC); configures the device on first use like any other call.
- *   out4[0]  tile shape: 0 = CTA pairs on 256 x 256 tiles, 1 = 128 x 256 tiles, 2 = 128 x 128 tiles
+ *   out4[0]  tile shape: 0 = CTA pairs on 256 x 256 tiles, 1 = 128 x 256 tiles, 2 = 128 x 128 tiles, 3 = 128 x 128
+ *            tiles with the even K hand-out through the workspace (every CTA the same number of (tile, K block)
+ *            units; then out4[1] = the most partial tiles one output tile can get, out4[3] = units per CTA)
  *   out4[1]  K slices through the workspace (1 = none);  workspace_bytes = 0 stands for no workspace
  *   out4[2]  CTAs per cluster that cut K for one tile (1 = none)
  *   out4[3]  K blocks of 64 per slice

@@ -57,6 +57,10 @@ struct GemmParams {
     int split_k;       // 1: no split, the epilogue writes BF16 C
     int kb_per_split;
     float* partial;
+    // Even K hand-out (single-CTA kernel, with scratch): all (tile, K block) units in tile order are cut into one
+    // contiguous share of `even_units` per CTA, whatever tiles a share touches; a CTA writes one FP32 partial per tile
+    // it touches, into slot (its index) - (index of the first CTA that touches the tile).  0: off.
+    int even_units;
     // FP16-input / FP32-output variant (the dtypes of the paper's Listing 2) and its accumulate form C += A*B
     float* Cf;         // non-null: FP32 output with pitch ldcf instead of BF16 C
     int64_t ldcf;
@@ -212,6 +216,41 @@ __device__ __forceinline__ void gemm_tile_coords(const GemmParams& p, int tile, 
     tn = r / rows;
 }
 
+// The pieces of work of one CTA of the single-CTA kernel, in the order every role walks them: (tile, K slice) items
+// handed out with a stride of the grid, or (even K hand-out) the pieces of the CTA's contiguous share of all
+// (tile, K block) units.
+struct GemmWork {
+    int tile, kb0, kb1, slot;
+};
+struct GemmWorkIter {
+    long long u, u_end;  // even hand-out: next unit, end of the share
+    int item;            // strided hand-out: next item
+    __device__ __forceinline__ GemmWorkIter(const GemmParams& p, int num_kb) {
+        item = static_cast<int>(blockIdx.x);
+        const long long total = static_cast<long long>(p.tiles_m) * p.tiles_n * num_kb;
+        u = static_cast<long long>(blockIdx.x) * p.even_units;
+        u_end = min(total, u + p.even_units);
+    }
+    __device__ __forceinline__ bool next(const GemmParams& p, int num_kb, GemmWork& w) {
+        if (p.even_units > 0) {
+            if (u >= u_end) return false;
+            w.tile = static_cast<int>(u / num_kb);
+            w.kb0 = static_cast<int>(u - static_cast<long long>(w.tile) * num_kb);
+            w.kb1 = static_cast<int>(min(static_cast<long long>(num_kb), w.kb0 + (u_end - u)));
+            w.slot = static_cast<int>(blockIdx.x) - static_cast<int>(static_cast<long long>(w.tile) * num_kb / p.even_units);
+            u += w.kb1 - w.kb0;
+            return true;
+        }
+        if (item >= p.tiles_m * p.tiles_n * p.split_k) return false;
+        w.tile = item / p.split_k;
+        w.slot = item % p.split_k;
+        w.kb0 = w.slot * p.kb_per_split;
+        w.kb1 = min(num_kb, w.kb0 + p.kb_per_split);
+        item += static_cast<int>(gridDim.x);
+        return true;
+    }
+};
+
 #ifdef MLT_TRACE
 // development builds: SM clock at a few points of CTA 0 of gemm_bf16_kernel
 __device__ long long g_gemm_trace[16];
@@ -245,7 +284,6 @@ gemm_bf16_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_consta
     if (threadIdx.x == 0) MLT_GT(0);
     MLT_GT_NS(6);
     const int lane = threadIdx.x & 31;
-    const int num_items = p.tiles_m * p.tiles_n * p.split_k;
     const int num_kb = (p.K + kGemmBK - 1) / kGemmBK;
     constexpr uint32_t kTmemCols = 2 * BN;  // 512 for BN = 256, 256 for BN = 128
 
@@ -281,12 +319,13 @@ gemm_bf16_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_consta
             int stage = 0;
             uint32_t phase = 0;
             bool ok = true;
-            for (int item = blockIdx.x; item < num_items && ok; item += gridDim.x) {
+            GemmWorkIter work(p, num_kb);
+            GemmWork w;
+            while (ok && work.next(p, num_kb, w)) {
                 int tm, tn;
-                gemm_tile_coords(p, item / p.split_k, tm, tn);
+                gemm_tile_coords(p, w.tile, tm, tn);
                 const int m0 = tm * kGemmBM, n0 = tn * BN;
-                const int kb0 = (item % p.split_k) * p.kb_per_split, kb1 = min(num_kb, kb0 + p.kb_per_split);
-                for (int kb = kb0; kb < kb1; ++kb) {
+                for (int kb = w.kb0; kb < w.kb1; ++kb) {
                     ok = mbar_wait(&empty[stage], phase ^ 1, abort_flag, 0x100 + stage);
                     if (!ok) break;
                     uint8_t* sa = smem + stage * L::kStageBytes;
@@ -314,12 +353,14 @@ gemm_bf16_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_consta
             int acc = 0;
             uint32_t acc_phase = 0;
             bool ok = true;
-            for (int item = blockIdx.x; item < num_items && ok; item += gridDim.x) {
+            GemmWorkIter work(p, num_kb);
+            GemmWork w;
+            while (ok && work.next(p, num_kb, w)) {
                 ok = __all_sync(0xffffffffu, mbar_wait(&acc_empty[acc], acc_phase ^ 1, abort_flag, 0x300 + acc));
                 if (!ok) break;
                 tc_fence_after();
                 const uint32_t d_tmem = tmem_base + acc * BN;
-                const int kb0 = (item % p.split_k) * p.kb_per_split, kb1 = min(num_kb, kb0 + p.kb_per_split);
+                const int kb0 = w.kb0, kb1 = w.kb1;
                 for (int kb = kb0; kb < kb1; ++kb) {
                     ok = __all_sync(0xffffffffu, mbar_wait(&full[stage], phase, abort_flag, 0x200 + stage));
                     if (!ok) break;
@@ -349,9 +390,11 @@ gemm_bf16_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_consta
         int acc = 0;
         uint32_t acc_phase = 0;
         bool ok = true;
-        for (int item = blockIdx.x; item < num_items && ok; item += gridDim.x) {
+        GemmWorkIter work(p, num_kb);
+        GemmWork w;
+        while (ok && work.next(p, num_kb, w)) {
             int tm, tn;
-            gemm_tile_coords(p, item / p.split_k, tm, tn);
+            gemm_tile_coords(p, w.tile, tm, tn);
             const int row = tm * kGemmBM + quarter * 32 + lane;
             const int n0 = tn * BN;
             ok = __all_sync(0xffffffffu, mbar_wait(&acc_full[acc], acc_phase, abort_flag, 0x400 + acc));
@@ -381,7 +424,7 @@ gemm_bf16_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_consta
                         gemm_store_chunk_tma(p, &tmap_c, smem_staging + quarter * 8192 + (c & 1) * 4096, v, lane,
                                              tm * kGemmBM + quarter * 32, n0 + c * 32);
                     else
-                        gemm_store_chunk(p, v, row, n0 + c * 32, item % p.split_k);
+                        gemm_store_chunk(p, v, row, n0 + c * 32, w.slot);
                 }
             }
             tc_fence_before();
@@ -797,8 +840,10 @@ gemm_bf16_clusterk_kernel(const __grid_constant__ CUtensorMap tmap_a, const __gr
     }
 }
 
-// Split-K second step: C[i][j] = RNE_bf16(sum over slices of partial[slice][i][j]); 8 columns per thread.
-__global__ void gemm_splitk_reduce_kernel(const float* partial, __nv_bfloat16* C, int64_t ldc, int M, int N, int split_k) {
+// Split-K second step: C[i][j] = RNE_bf16(sum over slices of partial[slice][i][j]); 8 columns per thread.  With the
+// even K hand-out the number of partials differs from tile to tile and follows from the same arithmetic as in the kernel.
+__global__ void gemm_splitk_reduce_kernel(const float* partial, __nv_bfloat16* C, int64_t ldc, int M, int N, int split_k,
+                                          int even_units, int num_kb, int tiles_m) {
     const int64_t groups_per_row = (N + 7) / 8;
     const int64_t total = static_cast<int64_t>(M) * groups_per_row;
     // Launched with programmatic stream serialisation: the CTAs may start while the GEMM kernel is still running
@@ -809,13 +854,18 @@ __global__ void gemm_splitk_reduce_kernel(const float* partial, __nv_bfloat16* C
         const int row = static_cast<int>(i / groups_per_row);
         const int col = static_cast<int>(i % groups_per_row) * 8;
         float acc[8] = {0, 0, 0, 0, 0, 0, 0, 0};
+        int parts = split_k;
+        if (even_units > 0) {  // even K hand-out: the CTAs whose shares touch this element's tile, one partial each
+            const long long t = static_cast<long long>(col / 128) * tiles_m + row / kGemmBM;  // one raster group: M fastest
+            parts = static_cast<int>(((t + 1) * num_kb - 1) / even_units - t * num_kb / even_units) + 1;
+        }
         const bool full = col + 8 <= N && (N & 3) == 0;
         const int64_t slice_pitch = static_cast<int64_t>(M) * N;
         const float* src0 = partial + static_cast<int64_t>(row) * N + col;
         int s = 0;
         if (full) {
             // four slices' loads in flight before the first addition (the additions keep the ascending slice order)
-            for (; s + 4 <= split_k; s += 4) {
+            for (; s + 4 <= parts; s += 4) {
                 float4 a[4], b[4];
 #pragma unroll
                 for (int u = 0; u < 4; ++u) {
@@ -829,7 +879,7 @@ __global__ void gemm_splitk_reduce_kernel(const float* partial, __nv_bfloat16* C
                 }
             }
         }
-        for (; s < split_k; ++s) {
+        for (; s < parts; ++s) {
             const float* src = src0 + s * slice_pitch;
             if (full) {
                 const float4 a = *reinterpret_cast<const float4*>(src), b = *reinterpret_cast<const float4*>(src + 4);

@@ -147,9 +147,10 @@ int forced_variant() {
 // Debug only: tuning overrides read once from the environment (0 = not set).  MLT_GEMM_GROUP_M: M-tiles per raster
 // group of the pair kernel; MLT_GEMM_NO_HALF: no half tiles in the last wave; MLT_MHA_HEAD_GROUP / MLT_MHA_GRID: item
 // list grouping and CTA count of the attention kernel; MLT_PAGED_SPLITS: CTAs per (sequence, KV head);
-// MLT_GEMM_WIDE_RATIO: per cent of the current plan's cost below which 128 x 256 tiles in clusters are taken (1: never).
+// MLT_GEMM_WIDE_RATIO: per cent of the current plan's cost below which 128 x 256 tiles in clusters are taken (1: never);
+// MLT_GEMM_NO_EVEN: uniform K slices through scratch instead of the even hand-out.
 struct DebugEnv {
-    int gemm_group_m, gemm_no_half, mha_head_group, mha_grid, paged_splits, gemm_wide_ratio;
+    int gemm_group_m, gemm_no_half, mha_head_group, mha_grid, paged_splits, gemm_wide_ratio, gemm_no_even;
 };
 const DebugEnv& debug_env() {
     static const DebugEnv env = [] {
@@ -159,7 +160,7 @@ const DebugEnv& debug_env() {
             return v > 0 ? v : 0;
         };
         return DebugEnv{get("MLT_GEMM_GROUP_M"), get("MLT_GEMM_NO_HALF"), get("MLT_MHA_HEAD_GROUP"), get("MLT_MHA_GRID"),
-                        get("MLT_PAGED_SPLITS"), get("MLT_GEMM_WIDE_RATIO")};
+                        get("MLT_PAGED_SPLITS"), get("MLT_GEMM_WIDE_RATIO"), get("MLT_GEMM_NO_EVEN")};
     }();
     return env;
 }
@@ -280,7 +281,9 @@ struct GemmPlan {
     int variant;       // 0: CTA pairs on 256 x 256 tiles, 1: 128 x 256 tiles, 2: 128 x 128 tiles
     int split_k;       // > 1: K slices with FP32 partials in caller scratch, summed by a second kernel
     int cluster;       // > 1: CTAs per cluster that cut K for one tile (128 x 128, or 128 x 256 with variant 1) and reduce through distributed shared memory
-    int kb_per_split;  // K blocks of 64 per slice (per CTA of a cluster)
+    int kb_per_split;  // K blocks of 64 per slice (per CTA of a cluster; per CTA's share with the even hand-out)
+    int even;          // 1: even K hand-out through scratch (variant 2): every CTA the same number of (tile, K block)
+                       //    units, split_k = the most partials a tile can get
 };
 
 static GemmPlan gemm_plan_base(int64_t M, int64_t N, int64_t K, bool has_workspace, size_t workspace_bytes, bool f32_out,
@@ -295,7 +298,7 @@ static GemmPlan gemm_plan_base(int64_t M, int64_t N, int64_t K, bool has_workspa
     const int64_t tiles1 = tiles_m128 * ((N + 255) / 256);
     const int64_t tiles2 = tiles_m128 * ((N + 127) / 128);
     const int num_kb = static_cast<int>((K + kGemmBK - 1) / kGemmBK);
-    GemmPlan plan = {2, 1, 1, num_kb};
+    GemmPlan plan = {2, 1, 1, num_kb, 0};
     if (M >= 512) {
         const int64_t pairs = sm_count / 2;
         const double c0 = static_cast<double>((pair_tiles + pairs - 1) / pairs);
@@ -342,6 +345,22 @@ static GemmPlan gemm_plan_base(int64_t M, int64_t N, int64_t K, bool has_workspa
         plan.kb_per_split = (num_kb + split - 1) / split;
         plan.split_k = (num_kb + plan.kb_per_split - 1) / plan.kb_per_split;  // no empty slice
     }
+    // ... or the even hand-out: all tiles x K blocks units cut into one contiguous share per SM, whatever tiles a
+    // share touches (uniform slices leave the last round part empty: 672 items on 148 SMs are 4.5 rounds, paid as 5).
+    // One raster group only (the reduce kernel recomputes a tile's index from its coordinates).
+    if (max_split > 1 && tiles_m128 <= 16 && !debug_env().gemm_no_even) {
+        const int64_t total = tiles2 * num_kb;
+        const int64_t units = (total + sm_count - 1) / sm_count;
+        const int parts = static_cast<int>((num_kb + units - 1) / units) + 1;  // CTAs that can touch one tile
+        const double partial = 2.0 * M * N * 8.0 / (16384.0 * sm_count);        // about two partials per element
+        const double cost = static_cast<double>(units) + 2 * 4 + partial;        // two pieces per share: fill and drain twice
+        if (units >= 8 && units <= INT32_MAX && static_cast<size_t>(parts) * M * N * sizeof(float) <= workspace_bytes &&
+            cost < (split > 1 ? best : static_cast<double>((tiles2 + sm_count - 1) / sm_count) * (num_kb + 4))) {
+            plan.even = 1;
+            plan.split_k = parts;
+            plan.kb_per_split = static_cast<int>(units);
+        }
+    }
     return plan;
 }
 
@@ -373,6 +392,8 @@ static GemmPlan gemm_plan(int64_t M, int64_t N, int64_t K, bool has_workspace, s
     else if (plan.cluster > 1)
         cur = static_cast<double>(rounds_of(tiles2 * plan.cluster, std::max<int64_t>(slots_of(plan.cluster), plan.cluster))) *
               (plan.kb_per_split + 10) * 32.0;
+    else if (plan.even)
+        cur = static_cast<double>(plan.kb_per_split + 8) * 32.0 + 2.0 * M * N * 8.0 / (1024.0 * sm_count);
     else
         cur = static_cast<double>(rounds_of(tiles2 * plan.split_k, sm_count)) * (plan.kb_per_split + 4) * 32.0 +
               (plan.split_k > 1 ? static_cast<double>(plan.split_k) * M * N * 8.0 / (1024.0 * sm_count) : 0.0);
@@ -387,7 +408,7 @@ static GemmPlan gemm_plan(int64_t M, int64_t N, int64_t K, bool has_workspace, s
         const double cost = static_cast<double>(rounds_of(tiles1 * S, slots)) * (kbps + 10) * 48.0;
         if (cost < best) { best = cost; best_s = S; best_kbps = kbps; }
     }
-    if (best_s > 1 && best * 100.0 < cur * ratio) plan = GemmPlan{1, 1, best_s, best_kbps};
+    if (best_s > 1 && best * 100.0 < cur * ratio) plan = GemmPlan{1, 1, best_s, best_kbps, 0};
     return plan;
 }
 
@@ -400,7 +421,7 @@ int mlt_debug_gemm_plan(int64_t M, int64_t N, int64_t K, size_t workspace_bytes,
     }
     const GemmPlan plan = sm_count == 0 ? gemm_plan(M, N, K, workspace_bytes > 0, workspace_bytes, false, dev.sm_count, dev.cluster_slots, -1)
                                         : gemm_plan(M, N, K, workspace_bytes > 0, workspace_bytes, false, sm_count, nullptr, -1);
-    out4[0] = plan.variant;
+    out4[0] = plan.even ? 3 : plan.variant;
     out4[1] = plan.split_k;
     out4[2] = plan.cluster;
     out4[3] = plan.kb_per_split;
@@ -497,11 +518,13 @@ static int gemm_run(const void* A, const void* B, void* C, int64_t M, int64_t N,
     p.f16_inputs = f16_in ? 1u : 0u;
     p.full_items = p.num_items = 0;
     const int cluster_s = plan.cluster;
+    p.even_units = 0;
     if (plan.split_k > 1) {
         // Few tiles and more than half an SM count of them: K is cut into slices, FP32 partials go to the caller's scratch
         p.kb_per_split = plan.kb_per_split;
         p.split_k = plan.split_k;
         p.partial = static_cast<float*>(workspace);
+        if (plan.even) p.even_units = plan.kb_per_split;
     }
     if (variant == 0) {
         // M-tiles per raster group: wide problems re-read B once per group, so fewer, taller groups pay
@@ -541,7 +564,10 @@ static int gemm_run(const void* A, const void* B, void* C, int64_t M, int64_t N,
         if (e != cudaSuccess) return MLT_ERR_CUDA;
     } else {
         p.group_m = 16;
-        const int grid = static_cast<int>(std::min<int64_t>(tiles_m * tiles_n * p.split_k, dev.sm_count));
+        const int64_t work_items = p.even_units > 0
+                                       ? (tiles_m * tiles_n * ((K + kGemmBK - 1) / kGemmBK) + p.even_units - 1) / p.even_units
+                                       : tiles_m * tiles_n * p.split_k;
+        const int grid = static_cast<int>(std::min<int64_t>(work_items, dev.sm_count));
         if (variant == 1 && c_tma)
             gemm_bf16_kernel<256, 4, true><<<grid, kGemmThreads, GemmSmem<256, 4>::kTotal, st>>>(ta, tb, tc, p);
         else if (variant == 1)
@@ -564,7 +590,7 @@ static int gemm_run(const void* A, const void* B, void* C, int64_t M, int64_t N,
             cfg.attrs = &attr;
             cfg.numAttrs = 1;
             if (cudaLaunchKernelEx(&cfg, gemm_splitk_reduce_kernel, static_cast<const float*>(p.partial), p.C, ldc, p.M, p.N,
-                                   p.split_k) != cudaSuccess)
+                                   p.split_k, p.even_units, static_cast<int>((K + kGemmBK - 1) / kGemmBK), p.tiles_m) != cudaSuccess)
                 return MLT_ERR_CUDA;
         }
     }

@@ -21,7 +21,13 @@ def test_plan_invariants(sm_count):
         for ws in {0, need // 3 // 16 * 16, need}:
             pl = mlt.gemm_plan(M, N, K, ws, sm_count)
             what = f"{M}x{N}x{K} ws={ws} sms={sm_count}: {pl}"
-            assert pl["variant"] in (0, 1, 2), what
+            assert pl["variant"] in (0, 1, 2, 3), what
+            if pl["variant"] == 3:   # even K hand-out: shares cover all units, the partial tiles fit the scratch
+                tiles = ((M + 127) // 128) * ((N + 127) // 128)
+                assert pl["cluster"] == 1 and M < 512 and ws > 0, what
+                assert pl["kb_per_split"] * sm_count >= tiles * kb(K) > pl["kb_per_split"] * (sm_count - 1) - sm_count, what
+                assert pl["split_k"] == -(-kb(K) // pl["kb_per_split"]) + 1 and pl["split_k"] * M * N * 4 <= ws, what
+                continue
             assert pl["cluster"] in (1, 2, 4, 8) and pl["split_k"] >= 1, what
             assert pl["cluster"] == 1 or pl["split_k"] == 1, what
             slices = max(pl["cluster"], pl["split_k"])
@@ -49,7 +55,7 @@ def test_plan_known_cases_on_148_sms():
     assert full(16, 8192, 4096)["cluster"] == 2
     assert full(16, 1024, 4096)["cluster"] == 8
     # 224 tiles: clusters would need more than one round; with scratch K goes through the workspace, without it whole
-    assert full(16, 28672, 4096)["cluster"] == 1 and full(16, 28672, 4096)["split_k"] > 1
+    assert full(16, 28672, 4096) == {"variant": 3, "split_k": 2, "cluster": 1, "kb_per_split": 97}   # 224 x 64 units / 148
     assert mlt.gemm_plan(16, 28672, 4096) == {"variant": 0, "split_k": 1, "cluster": 1, "kb_per_split": 64}
     # a short K is not cut
     assert full(16, 4096, 192)["cluster"] == 1 and full(16, 4096, 192)["split_k"] == 1
