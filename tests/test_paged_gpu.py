@@ -29,7 +29,7 @@ def run_paged(Q, Kc, Vc, table, lens, scale, workspace_bytes=None, with_lse=True
     L = Lbuf[guard:guard + S * H]
     if workspace_bytes is None:
         workspace_bytes = mlt.paged_attn_workspace_bytes(S, H, D)
-    ws = torch.full((workspace_bytes + 64,), 0xAB, dtype=torch.uint8, device="cuda") if workspace_bytes else None
+    ws = torch.full((workspace_bytes + 64,), 0xFF, dtype=torch.uint8, device="cuda") if workspace_bytes else None  # NaN patterns: an unwritten partial that is read shows
     dQ, dK, dV = to_dev(Q), to_dev(Kc), to_dev(Vc)
     dT = torch.from_numpy(np.ascontiguousarray(table, dtype=np.int32)).cuda()
     dL = torch.from_numpy(np.ascontiguousarray(lens, dtype=np.int32)).cuda()
@@ -44,7 +44,7 @@ def run_paged(Q, Kc, Vc, table, lens, scale, workspace_bytes=None, with_lse=True
     lb = Lbuf.cpu().numpy()
     assert np.isnan(lb[:guard]).all() and np.isnan(lb[-guard:]).all(), "LSE guard band was written"
     if ws is not None:
-        assert (ws[workspace_bytes:].cpu().numpy() == 0xAB).all(), "workspace overrun"
+        assert (ws[workspace_bytes:].cpu().numpy() == 0xFF).all(), "workspace overrun"
     body = ob[guard:-guard]
     assert not (body == SENTINEL).any(), "unwritten O elements"
     return inputs.bf16_bits_to_f64(body).reshape(S * H, D), (lb[guard:-guard].astype(np.float64) if with_lse else None)
