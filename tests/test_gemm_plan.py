@@ -70,3 +70,33 @@ def test_plan_rejects_bad_arguments():
         mlt.gemm_plan(0, 8, 8)
     with pytest.raises(mlt.MltError):
         mlt.gemm_plan(8, 8, 8, 0, 1)
+
+
+def test_even_hand_out_slots_fit_the_plan():
+    """Even K hand-out (plan variant 3): CTA c takes units [c U, (c + 1) U) of all tiles x K blocks in tile order and
+    writes, per tile it touches, partial slot c - (first CTA of the tile).  The plan's split_k is the number of partial
+    tiles the scratch must hold per output tile: no slot may reach it, and the reduce kernel's count formula must be
+    the number of CTAs that really touch the tile."""
+    seen = 0
+    for sm_count in (148, 132, 64):
+        for M, N, K in [(16, 28672, 4096), (16, 9600, 2048), (200, 5000, 4100), (1, 9600, 4100), (100, 20000, 1700),
+                        (300, 12000, 3000), (511, 9000, 2500), (64, 30000, 8192)]:
+            pl = mlt.gemm_plan(M, N, K, mlt.gemm_workspace_bytes(M, N, K), sm_count)
+            if pl["variant"] != 3:
+                continue
+            seen += 1
+            U, nkb = pl["kb_per_split"], kb(K)
+            tiles = ((M + 127) // 128) * ((N + 127) // 128)
+            total = tiles * nkb
+            ctas = -(-total // U)
+            assert ctas <= sm_count
+            touched = {}
+            for c in range(ctas):
+                for t in range(c * U // nkb, (min(total, (c + 1) * U) - 1) // nkb + 1):
+                    touched.setdefault(t, []).append(c)
+            assert sorted(touched) == list(range(tiles))
+            for t, cs in touched.items():
+                assert cs == list(range(cs[0], cs[-1] + 1)) and cs[0] == t * nkb // U      # slot = c - cs[0]
+                assert len(cs) == ((t + 1) * nkb - 1) // U - t * nkb // U + 1               # the reduce kernel's count
+                assert len(cs) <= pl["split_k"], (M, N, K, sm_count, pl, t, cs)
+    assert seen >= 6
