@@ -148,9 +148,10 @@ int forced_variant() {
 // group of the pair kernel; MLT_GEMM_NO_HALF: no half tiles in the last wave; MLT_MHA_HEAD_GROUP / MLT_MHA_GRID: item
 // list grouping and CTA count of the attention kernel; MLT_PAGED_SPLITS: CTAs per (sequence, KV head);
 // MLT_GEMM_WIDE_RATIO: per cent of the current plan's cost below which 128 x 256 tiles in clusters are taken (1: never);
-// MLT_GEMM_NO_EVEN: uniform K slices through scratch instead of the even hand-out.
+// MLT_GEMM_NO_EVEN: uniform K slices through scratch instead of the even hand-out; MLT_GEMM_NO_SKINNY_MODEL: the
+// rule-based plan for problems of one tile row instead of the time model.
 struct DebugEnv {
-    int gemm_group_m, gemm_no_half, mha_head_group, mha_grid, paged_splits, gemm_wide_ratio, gemm_no_even;
+    int gemm_group_m, gemm_no_half, mha_head_group, mha_grid, paged_splits, gemm_wide_ratio, gemm_no_even, gemm_no_skinny_model;
 };
 const DebugEnv& debug_env() {
     static const DebugEnv env = [] {
@@ -160,7 +161,7 @@ const DebugEnv& debug_env() {
             return v > 0 ? v : 0;
         };
         return DebugEnv{get("MLT_GEMM_GROUP_M"), get("MLT_GEMM_NO_HALF"), get("MLT_MHA_HEAD_GROUP"), get("MLT_MHA_GRID"),
-                        get("MLT_PAGED_SPLITS"), get("MLT_GEMM_WIDE_RATIO"), get("MLT_GEMM_NO_EVEN")};
+                        get("MLT_PAGED_SPLITS"), get("MLT_GEMM_WIDE_RATIO"), get("MLT_GEMM_NO_EVEN"), get("MLT_GEMM_NO_SKINNY_MODEL")};
     }();
     return env;
 }
@@ -299,6 +300,48 @@ static GemmPlan gemm_plan_base(int64_t M, int64_t N, int64_t K, bool has_workspa
     const int64_t tiles2 = tiles_m128 * ((N + 127) / 128);
     const int num_kb = static_cast<int>((K + kGemmBK - 1) / kGemmBK);
     GemmPlan plan = {2, 1, 1, num_kb, 0};
+    if (M <= kGemmBM && !f32_out && !(forced >= 0 && forced <= 2) && !debug_env().gemm_no_skinny_model &&
+        gemm_cluster_split(tiles2, num_kb, sm_count, cluster_slots) == 1) {
+        // One row of tiles, too many of them to cut K inside clusters: B streams once and the question is only which
+        // launch keeps HBM busiest.  Time model in microseconds, fitted to CUDA-event timings on M = 16..128,
+        // N = 14k..115k, K = 2k..8k: 5 us of launch and fill, then the larger of the stream at the copy bandwidth
+        // (6.5 TB/s) and the busiest SM's bytes at what one SM pulls (67 GB/s in 512-byte rows of a 128 x 256 tile,
+        // 56 GB/s in the 256-byte rows of a 128 x 128 tile; the rows of A come from L2 and count 0.3); a second kernel
+        // costs 5 us more and the even hand-out's short end pieces about 2.  The CTA-pair kernel never won here (half
+        // of each pair has no rows).
+        const double a_bytes = 0.3 * static_cast<double>(M) * 128.0;
+        const double fill = (num_kb + 4.0) / num_kb;
+        const double hbm_us = 2.0 * (static_cast<double>(M) * K + static_cast<double>(K) * N + static_cast<double>(M) * N) / 6.5e6;
+        auto rounds_of = [&](int64_t items) { return static_cast<double>((items + sm_count - 1) / sm_count); };
+        const double t1 = 5.0 + std::max(hbm_us, rounds_of(tiles1) * num_kb * (a_bytes + 32768.0) * fill / 67e3);
+        const double t2 = 5.0 + std::max(hbm_us, rounds_of(tiles2) * num_kb * (a_bytes + 16384.0) * fill / 56e3);
+        plan.variant = t1 < t2 ? 1 : 2;
+        double best_t = std::min(t1, t2);
+        int max_split = has_workspace ? gemm_max_split(M, N, K) : 1;
+        while (max_split > 1 && static_cast<size_t>(max_split) * M * N * sizeof(float) > workspace_bytes) --max_split;
+        const double partial_us = static_cast<double>(M) * N * 8.0 / 6.5e6;  // one FP32 partial written and read
+        for (int sl = 2; sl <= max_split; ++sl) {  // uniform slices through scratch
+            const int kbps = (num_kb + sl - 1) / sl;
+            const int slices = (num_kb + kbps - 1) / kbps;
+            if (slices != sl) continue;
+            const double t = 10.0 + sl * partial_us +
+                             std::max(hbm_us, rounds_of(tiles2 * slices) * (kbps + 4.0) * (a_bytes + 16384.0) / 56e3);
+            if (t < best_t) {
+                best_t = t;
+                plan = GemmPlan{2, slices, 1, kbps, 0};
+            }
+        }
+        if (max_split > 1 && !debug_env().gemm_no_even) {  // the even hand-out through scratch
+            const int64_t units = (tiles2 * num_kb + sm_count - 1) / sm_count;
+            const int parts = static_cast<int>((num_kb + units - 1) / units) + 1;
+            const double t = 12.0 + 2.0 * partial_us + std::max(hbm_us, (units + 8.0) * (a_bytes + 16384.0) / 56e3);
+            if (units >= 8 && units <= INT32_MAX && static_cast<size_t>(parts) * M * N * sizeof(float) <= workspace_bytes && t < best_t) {
+                best_t = t;
+                plan = GemmPlan{2, parts, 1, static_cast<int>(units), 1};
+            }
+        }
+        return plan;
+    }
     if (M >= 512) {
         const int64_t pairs = sm_count / 2;
         const double c0 = static_cast<double>((pair_tiles + pairs - 1) / pairs);

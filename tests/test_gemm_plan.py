@@ -55,8 +55,11 @@ def test_plan_known_cases_on_148_sms():
     assert full(16, 8192, 4096)["cluster"] == 2
     assert full(16, 1024, 4096)["cluster"] == 8
     # 224 tiles: clusters would need more than one round; with scratch K goes through the workspace, without it whole
-    assert full(16, 28672, 4096) == {"variant": 3, "split_k": 2, "cluster": 1, "kb_per_split": 97}   # 224 x 64 units / 148
-    assert mlt.gemm_plan(16, 28672, 4096) == {"variant": 0, "split_k": 1, "cluster": 1, "kb_per_split": 64}
+    # one tile row, many tiles: the time model.  112 tiles of 128 x 256 in one round keep HBM busy without any cut ...
+    assert full(16, 28672, 4096) == mlt.gemm_plan(16, 28672, 4096) == {"variant": 1, "split_k": 1, "cluster": 1, "kb_per_split": 64}
+    # ... 160 of them would be a round and a bit: the even hand-out through scratch (320 x 64 units / 148), else small tiles
+    assert full(16, 40960, 4096) == {"variant": 3, "split_k": 2, "cluster": 1, "kb_per_split": 139}
+    assert mlt.gemm_plan(16, 40960, 4096)["variant"] == 2
     # a short K is not cut
     assert full(16, 4096, 192)["cluster"] == 1 and full(16, 4096, 192)["split_k"] == 1
     assert full(512, 512, 512)["cluster"] == 1
@@ -79,7 +82,7 @@ def test_even_hand_out_slots_fit_the_plan():
     the number of CTAs that really touch the tile."""
     seen = 0
     for sm_count in (148, 132, 64):
-        for M, N, K in [(16, 28672, 4096), (16, 9600, 2048), (200, 5000, 4100), (1, 9600, 4100), (100, 20000, 1700),
+        for M, N, K in [(16, 40960, 4096), (16, 9600, 4096), (200, 5000, 4100), (1, 9600, 4100), (100, 20000, 1700),
                         (300, 12000, 3000), (511, 9000, 2500), (64, 30000, 8192)]:
             pl = mlt.gemm_plan(M, N, K, mlt.gemm_workspace_bytes(M, N, K), sm_count)
             if pl["variant"] != 3:
