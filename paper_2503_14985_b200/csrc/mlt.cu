@@ -342,7 +342,11 @@ static GemmPlan gemm_plan_base(int64_t M, int64_t N, int64_t K, bool has_workspa
         }
         return plan;
     }
-    if (M >= 512) {
+    // (From 129 rows on the same comparison holds as long as there are too many tiles to cut K inside clusters:
+    // measured on 140..400 rows, N = 9600..28672, the model's pick was the fastest launch every time, and K cuts
+    // through scratch were 10-90 % slower than it.)
+    const bool by_waves = M >= 512 || (M > kGemmBM && !f32_out && gemm_cluster_split(tiles2, num_kb, sm_count, cluster_slots) == 1);
+    if (by_waves) {
         const int64_t pairs = sm_count / 2;
         const double c0 = static_cast<double>((pair_tiles + pairs - 1) / pairs);
         const double c1 = static_cast<double>((tiles1 + sm_count - 1) / sm_count) / 0.8;
@@ -368,7 +372,7 @@ static GemmPlan gemm_plan_base(int64_t M, int64_t N, int64_t K, bool has_workspa
         plan.kb_per_split = (num_kb + plan.cluster - 1) / plan.cluster;
         return plan;
     }
-    if (!has_workspace) return plan;
+    if (!has_workspace || M > kGemmBM) return plan;
     // ... else slices through scratch: the count that minimises rounds x (K blocks per slice + fill/drain of an item)
     // plus the time to write and re-read the FP32 partials, in units of one K block of one tile (16 KB of B per SM).
     int max_split = gemm_max_split(M, N, K);
@@ -448,7 +452,8 @@ static GemmPlan gemm_plan(int64_t M, int64_t N, int64_t K, bool has_workspace, s
         if (static_cast<int64_t>(kbps) * (S - 1) >= num_kb) continue;  // an empty slice
         const int64_t slots = slots_of(S);
         if (slots < S) continue;
-        const double cost = static_cast<double>(rounds_of(tiles1 * S, slots)) * (kbps + 10) * 48.0;
+        if (tiles1 * S > slots) continue;  // one round only: with more the model below misjudged (160x9600x4096: 45 against 31 us)
+        const double cost = static_cast<double>(kbps + 10) * 48.0;
         if (cost < best) { best = cost; best_s = S; best_kbps = kbps; }
     }
     if (best_s > 1 && best * 100.0 < cur * ratio) plan = GemmPlan{1, 1, best_s, best_kbps, 0};
