@@ -149,9 +149,9 @@ int forced_variant() {
 // list grouping and CTA count of the attention kernel; MLT_PAGED_SPLITS: CTAs per (sequence, KV head);
 // MLT_GEMM_WIDE_RATIO: per cent of the current plan's cost below which 128 x 256 tiles in clusters are taken (1: never);
 // MLT_GEMM_NO_EVEN: uniform K slices through scratch instead of the even hand-out; MLT_GEMM_NO_SKINNY_MODEL: the
-// rule-based plan for problems of one tile row instead of the time model.
+// rule-based plan for problems of one tile row instead of the time model; MLT_GEMM_NO_CLUSTER: no K cut inside clusters.
 struct DebugEnv {
-    int gemm_group_m, gemm_no_half, mha_head_group, mha_grid, paged_splits, gemm_wide_ratio, gemm_no_even, gemm_no_skinny_model;
+    int gemm_group_m, gemm_no_half, mha_head_group, mha_grid, paged_splits, gemm_wide_ratio, gemm_no_even, gemm_no_skinny_model, gemm_no_cluster;
 };
 const DebugEnv& debug_env() {
     static const DebugEnv env = [] {
@@ -161,7 +161,7 @@ const DebugEnv& debug_env() {
             return v > 0 ? v : 0;
         };
         return DebugEnv{get("MLT_GEMM_GROUP_M"), get("MLT_GEMM_NO_HALF"), get("MLT_MHA_HEAD_GROUP"), get("MLT_MHA_GRID"),
-                        get("MLT_PAGED_SPLITS"), get("MLT_GEMM_WIDE_RATIO"), get("MLT_GEMM_NO_EVEN"), get("MLT_GEMM_NO_SKINNY_MODEL")};
+                        get("MLT_PAGED_SPLITS"), get("MLT_GEMM_WIDE_RATIO"), get("MLT_GEMM_NO_EVEN"), get("MLT_GEMM_NO_SKINNY_MODEL"), get("MLT_GEMM_NO_CLUSTER")};
     }();
     return env;
 }
@@ -261,7 +261,7 @@ static int gemm_max_split(int64_t M, int64_t N, int64_t K) {
 // rounds x (K blocks per CTA + fill, drain and the reduction), every slice at least 4 blocks of 64.
 // cluster_slots: resident CTAs for S = 2, 4, 8 as the device reports them, or null for the SM count rounded down.
 static int gemm_cluster_split(int64_t tiles, int num_kb, int sm_count, const int* cluster_slots) {
-    if (tiles * 2 > sm_count) return 1;  // enough tiles to occupy the GPU without cutting K
+    if (tiles * 2 > sm_count || debug_env().gemm_no_cluster) return 1;  // enough tiles to occupy the GPU without cutting K
     int best_s = 1;
     int64_t best = (num_kb + 4);
     for (int S = 2, i = 0; S <= 8; S *= 2, ++i) {
